@@ -1,0 +1,86 @@
+// Shared device-side definitions of the DMTD decode library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dmtd {
+
+// Device-resident schedule counters (Section 2.2 of the paper); kernels read their row
+// positions from here so that a captured CUDA graph stays valid as the context grows.
+struct DevState {
+  int n_known;    // tokens whose id is known
+  int lo_len;     // positions with KV in the lower layers; first row of a full pass's refill
+  int up_len;     // positions with KV in the decoding layers
+  int cycle;
+  int slot;
+  int n_emitted;
+  int newest;     // n_known - 1: position fed to the decoding layers
+  int scratch;    // row origin for prefill chunks and dmtd_step_layers
+  int error;      // sticky: 1 = token id out of range
+  int tau;
+  int pad[6];
+};
+
+// A weight matrix [N][K] as the kernels read it.
+//  bf16: a stream of 1 KiB "atoms".  An atom holds 16 rows x 32 k in the register order of
+//        the A operand of mma.m16n8k16: two halves (rows g and g+8) of 32 lanes x 16 bytes,
+//        lane (g = lane/4, t = lane%4) owning k = 8t..8t+7 of the atom.  Atoms are ordered
+//        [k-slab][row tile][atom in slab]; a slab is `aps` atoms (KS = 32*aps values of k).
+//  fp32: plain row-major [N][K].
+struct PackedMat {
+  const uint4 *w;     // bf16 atom stream
+  const float *wf;    // fp32 row-major
+  int N, K;
+  int n_tiles;        // ceil(N / 16)
+  int aps;            // atoms per slab
+  int n_slabs;        // K / (32 * aps)
+};
+
+__host__ __device__ inline long long packed_atoms(const PackedMat &m) {
+  return (long long)m.n_slabs * m.n_tiles * m.aps;
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) {
+  return __uint_as_float(bits16 << 16);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Split an fp32 value into two bf16 terms hi + lo (|error| <= 2^-17 |x|): tensor-core
+// operands must be bf16, and a single rounding of the activations would exceed the logit
+// tolerance after 36 layers.
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
+  hi = __float2bfloat16_rn(x);
+  lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+// D += A * B, m16n8k16, bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};\n"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const uint4 *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+}  // namespace dmtd

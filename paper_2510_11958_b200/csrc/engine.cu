@@ -1,0 +1,714 @@
+// Host side of the DMTD decode library: context, weight repacking, the cycle scheduler of
+// Section 2.2 of the paper, and the C ABI declared in include/dmtd.h.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <numeric>
+#include <string>
+#include <vector>
+
+#include "../../include/dmtd.h"
+#include "kernels.cuh"
+
+using namespace dmtd;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+struct LayerDev {
+  PackedMat qkv, o, gu, down;
+  float *w_in, *w_post, *w_qn, *w_kn;
+};
+
+}  // namespace
+
+struct dmtd_ctx {
+  dmtd_model_shape s{};
+  int L_d = 0, tau = 0, max_batch = 0, max_seq = 0;
+  int device = 0, n_sms = 0;
+  cudaStream_t stream = nullptr;
+  std::string err;
+  std::vector<void *> allocs;
+
+  // model
+  std::vector<LayerDev> layers;
+  PackedMat embed{};
+  float *w_final = nullptr;
+  double *inv_freq = nullptr;
+
+  // sequence state
+  void *kc = nullptr, *vc = nullptr;        // [L][max_batch][nkv][max_seq][D]
+  size_t kv_layer_elems = 0;
+  int *tokens = nullptr;                    // [max_batch][max_seq]
+  DevState *dstate = nullptr;
+  dmtd_state h{};                           // host mirror
+  bool prefilled = false;
+  int B = 0;
+
+  // workspace
+  int ws_rows = 0, lda = 0, ldqkv = 0, ldgu = 0, ldl = 0, CH = 0, nsplit_max = 0;
+  float *x_lo = nullptr, *x_up = nullptr, *act = nullptr, *qkv = nullptr, *gu = nullptr,
+        *logits = nullptr, *part_o = nullptr, *part_ml = nullptr;
+  float2 *rope_tab = nullptr;
+
+  // options
+  bool use_graph = true, literal_sum = false;
+
+  // graphs: [kind 1 = full, 2 = upper-only]
+  cudaGraphExec_t graph_exec[3] = {nullptr, nullptr, nullptr};
+  int graph_nodes[3] = {0, 0, 0};
+  int graph_B = 0, graph_tau = 0;
+  bool capturing = false;
+
+  int64_t launches = 0;
+};
+
+namespace {
+
+dmtd_status fail(dmtd_ctx *c, dmtd_status st, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (c) c->err = buf; else g_create_error = buf;
+  return st;
+}
+
+#define CUDA_TRY(c, expr)                                                                   \
+  do {                                                                                      \
+    cudaError_t e_ = (expr);                                                                \
+    if (e_ != cudaSuccess)                                                                  \
+      return fail((c), DMTD_ERR_CUDA, "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e_), \
+                  __FILE__, __LINE__);                                                      \
+  } while (0)
+
+template <typename T>
+dmtd_status dev_alloc(dmtd_ctx *c, T **p, size_t n) {
+  void *q = nullptr;
+  CUDA_TRY(c, cudaMalloc(&q, std::max<size_t>(n, 1) * sizeof(T)));
+  c->allocs.push_back(q);
+  *p = static_cast<T *>(q);
+  return DMTD_OK;
+}
+
+dmtd_status check_launch(dmtd_ctx *c, const char *what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(c, DMTD_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
+  c->launches += 1;
+  return DMTD_OK;
+}
+#define LAUNCH_OK(c, what)                          \
+  do {                                              \
+    dmtd_status s_ = check_launch((c), (what));     \
+    if (s_ != DMTD_OK) return s_;                   \
+  } while (0)
+#define TRY(expr)                                   \
+  do {                                              \
+    dmtd_status s_ = (expr);                        \
+    if (s_ != DMTD_OK) return s_;                   \
+  } while (0)
+
+bool is_bf16(const dmtd_ctx *c) { return c->s.weight_dtype == DMTD_BF16; }
+size_t wbytes(const dmtd_ctx *c) { return is_bf16(c) ? 2 : 4; }
+
+// Largest divisor of the atom count per row that keeps a k-slab at or below 40 atoms.
+int choose_aps(int K) {
+  int atoms = K / 32, best = 1;
+  for (int d = 1; d <= std::min(atoms, 40); ++d)
+    if (atoms % d == 0) best = d;
+  return best;
+}
+
+// Build one packed matrix from up to three row blocks (e.g. q, k, v) of equal K.
+dmtd_status pack_matrix(dmtd_ctx *c, PackedMat *out, int K, const void *const *srcs, const int *Ns, int n_src) {
+  int N = 0;
+  for (int i = 0; i < n_src; ++i) N += Ns[i];
+  PackedMat m{};
+  m.N = N; m.K = K; m.n_tiles = (N + 15) / 16;
+  if (is_bf16(c)) {
+    m.aps = choose_aps(K);
+    m.n_slabs = K / 32 / m.aps;
+    uint4 *dst = nullptr;
+    TRY(dev_alloc(c, &dst, (size_t)packed_atoms(m) * 64));
+    int tile0 = 0;
+    for (int i = 0; i < n_src; ++i) {
+      if (tile0 * 16 != (int)std::accumulate(Ns, Ns + i, 0))
+        return fail(c, DMTD_ERR_SHAPE, "row blocks of a fused matrix must be multiples of 16 rows");
+      long long chunks = (long long)m.n_slabs * ((Ns[i] + 15) / 16) * m.aps * 64;
+      int grid = (int)std::min<long long>((chunks + 255) / 256, 65535);
+      pack_bf16_kernel<<<grid, 256, 0, c->stream>>>(static_cast<const __nv_bfloat16 *>(srcs[i]), Ns[i], K, dst,
+                                                    tile0, m.n_tiles, m.aps, m.n_slabs);
+      LAUNCH_OK(c, "pack_bf16_kernel");
+      tile0 += (Ns[i] + 15) / 16;
+    }
+    m.w = dst;
+  } else {
+    float *dst = nullptr;
+    TRY(dev_alloc(c, &dst, (size_t)N * K));
+    size_t off = 0;
+    for (int i = 0; i < n_src; ++i) {
+      CUDA_TRY(c, cudaMemcpyAsync(dst + off, srcs[i], (size_t)Ns[i] * K * 4, cudaMemcpyDeviceToDevice, c->stream));
+      off += (size_t)Ns[i] * K;
+    }
+    m.wf = dst;
+  }
+  *out = m;
+  return DMTD_OK;
+}
+
+dmtd_status vec_to_float(dmtd_ctx *c, float **out, const void *src, int n) {
+  TRY(dev_alloc(c, out, (size_t)n));
+  if (is_bf16(c))
+    to_float_kernel<__nv_bfloat16><<<(n + 255) / 256, 256, 0, c->stream>>>(static_cast<const __nv_bfloat16 *>(src), *out, n);
+  else
+    to_float_kernel<float><<<(n + 255) / 256, 256, 0, c->stream>>>(static_cast<const float *>(src), *out, n);
+  LAUNCH_OK(c, "to_float_kernel");
+  return DMTD_OK;
+}
+
+// ---------------------------------------------------------------------------- launches
+
+int gemv_smem_bytes(const PackedMat &W, int NT) {
+  int KS = W.aps * 32;
+  int row_bytes = ((KS * 2) % 128 == 64) ? KS * 2 : KS * 2 + 64;
+  return 8 * NT * row_bytes;
+}
+
+template <int NT>
+dmtd_status launch_gemv_nt(dmtd_ctx *c, const PackedMat &W, const float *act, int lda, int M, float *out, int ldo) {
+  int smem = gemv_smem_bytes(W, NT);
+  static int configured = 0;
+  if (configured < smem) {
+    CUDA_TRY(c, cudaFuncSetAttribute(gemv_bf16_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+    configured = 100 * 1024;
+  }
+  gemv_bf16_kernel<NT><<<2 * c->n_sms, GEMV_THREADS, smem, c->stream>>>(W, act, lda, M, out, ldo);
+  LAUNCH_OK(c, "gemv_bf16_kernel");
+  return DMTD_OK;
+}
+
+// out[m][n] += sum_k W[n][k] act[m][k]
+dmtd_status launch_gemv(dmtd_ctx *c, const PackedMat &W, const float *act, int lda, int M, float *out, int ldo) {
+  if (W.wf) {
+    gemv_f32_kernel<<<2 * c->n_sms, 256, 0, c->stream>>>(W, act, lda, M, out, ldo);
+    LAUNCH_OK(c, "gemv_f32_kernel");
+    return DMTD_OK;
+  }
+  if (M <= 4) return launch_gemv_nt<1>(c, W, act, lda, M, out, ldo);
+  if (M <= 8) return launch_gemv_nt<2>(c, W, act, lda, M, out, ldo);
+  return launch_gemv_nt<4>(c, W, act, lda, M, out, ldo);
+}
+
+template <int D, typename KVT>
+dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit) {
+  const dmtd_model_shape &s = c->s;
+  int M = B * R, heads = s.n_q_heads + 2 * s.n_kv_heads, G = s.n_q_heads / s.n_kv_heads;
+  KVT *kc = static_cast<KVT *>(c->kc) + (size_t)layer * c->kv_layer_elems;
+  KVT *vc = static_cast<KVT *>(c->vc) + (size_t)layer * c->kv_layer_elems;
+  const LayerDev &lw = c->layers[layer];
+  qk_norm_rope_append_kernel<D, KVT><<<dim3(M, (heads + 3) / 4), 128, 0, c->stream>>>(
+      c->qkv, c->ldqkv, s.n_q_heads, s.n_kv_heads, R, lw.w_qn, lw.w_kn, s.rms_eps, c->rope_tab, pos0, kc, vc,
+      c->max_seq);
+  LAUNCH_OK(c, "qk_norm_rope_append_kernel");
+  int RB = std::max(1, ATTN_QR / G), n_rb = (R + RB - 1) / RB;
+  size_t smem = (size_t)ATTN_WARPS * ATTN_QR * D * sizeof(float);
+  static bool configured = false;
+  if (!configured) {
+    CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<D, KVT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+    configured = true;
+  }
+  attn_partial_kernel<D, KVT><<<dim3(nsplit, s.n_kv_heads * n_rb, B), ATTN_WARPS * 32, smem, c->stream>>>(
+      c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml,
+      nsplit);
+  LAUNCH_OK(c, "attn_partial_kernel");
+  int n_rh = M * s.n_q_heads;
+  attn_merge_kernel<D><<<(n_rh + 3) / 4, 128, 0, c->stream>>>(c->part_o, c->part_ml, nsplit, n_rh, s.n_q_heads,
+                                                             c->act, c->lda);
+  LAUNCH_OK(c, "attn_merge_kernel");
+  return DMTD_OK;
+}
+
+dmtd_status launch_attention(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit) {
+  bool kvbf = c->s.kv_dtype == DMTD_BF16;
+  if (c->s.head_dim == 128)
+    return kvbf ? launch_attention_t<128, __nv_bfloat16>(c, layer, B, R, pos0, nsplit)
+                : launch_attention_t<128, float>(c, layer, B, R, pos0, nsplit);
+  return kvbf ? launch_attention_t<64, __nv_bfloat16>(c, layer, B, R, pos0, nsplit)
+              : launch_attention_t<64, float>(c, layer, B, R, pos0, nsplit);
+}
+
+dmtd_status launch_rope_table(dmtd_ctx *c, const int *pos0, int R) {
+  int half = c->s.head_dim / 2, n = R * half;
+  rope_table_kernel<<<(n + 127) / 128, 128, 0, c->stream>>>(pos0, R, half, c->inv_freq, c->rope_tab);
+  LAUNCH_OK(c, "rope_table_kernel");
+  return DMTD_OK;
+}
+
+dmtd_status launch_embed(dmtd_ctx *c, const int *pos0, int B, int R, float *x, bool accumulate) {
+  embed_kernel<<<B * R, 128, 0, c->stream>>>(c->embed, c->tokens, c->max_seq, pos0, R, x, c->s.hidden,
+                                             accumulate ? 1 : 0, c->dstate);
+  LAUNCH_OK(c, "embed_kernel");
+  return DMTD_OK;
+}
+
+// Number of key slices to launch: all of them while capturing a graph (the graph must stay
+// valid as the context grows), else just enough for keys [0, pos_end).
+int splits_for(const dmtd_ctx *c, int pos_end) {
+  if (c->capturing) return c->nsplit_max;
+  return std::max(1, std::min(c->nsplit_max, (pos_end + c->CH - 1) / c->CH));
+}
+
+// One decoder layer (steps a2-a7) on x [B*R][hidden]; rows of sequence b sit at positions
+// *pos0 .. *pos0+R-1.  pos_end = host's value of *pos0 + R.
+dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos0, int pos_end) {
+  const dmtd_model_shape &s = c->s;
+  const LayerDev &lw = c->layers[l];
+  int M = B * R, H = s.hidden, I = s.intermediate, QD = s.n_q_heads * s.head_dim;
+  prep_norm_kernel<<<M, 256, 0, c->stream>>>(x, H, lw.w_in, H, s.rms_eps, c->act, c->lda, c->qkv, c->ldqkv, c->ldqkv);
+  LAUNCH_OK(c, "prep_norm_kernel");
+  TRY(launch_gemv(c, lw.qkv, c->act, c->lda, M, c->qkv, c->ldqkv));
+  TRY(launch_attention(c, l, B, R, pos0, splits_for(c, pos_end)));
+  (void)QD;
+  TRY(launch_gemv(c, lw.o, c->act, c->lda, M, x, H));
+  prep_norm_kernel<<<M, 256, 0, c->stream>>>(x, H, lw.w_post, H, s.rms_eps, c->act, c->lda, c->gu, c->ldgu, c->ldgu);
+  LAUNCH_OK(c, "prep_norm_kernel");
+  TRY(launch_gemv(c, lw.gu, c->act, c->lda, M, c->gu, c->ldgu));
+  prep_swiglu_kernel<<<dim3((I + 255) / 256, M), 256, 0, c->stream>>>(c->gu, c->ldgu, I, c->act, c->lda);
+  LAUNCH_OK(c, "prep_swiglu_kernel");
+  TRY(launch_gemv(c, lw.down, c->act, c->lda, M, x, H));
+  return DMTD_OK;
+}
+
+// Step a9/a10: final norm, tied LM head, greedy pick, token feedback.
+dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, float *out_logits) {
+  const dmtd_model_shape &s = c->s;
+  prep_norm_kernel<<<B, 256, 0, c->stream>>>(c->x_up, s.hidden, c->w_final, s.hidden, s.rms_eps, c->act, c->lda,
+                                             c->logits, c->ldl, c->ldl);
+  LAUNCH_OK(c, "prep_norm_kernel");
+  TRY(launch_gemv(c, c->embed, c->act, c->lda, B, c->logits, c->ldl));
+  if (out_logits)
+    CUDA_TRY(c, cudaMemcpy2DAsync(out_logits, (size_t)s.vocab * 4, c->logits, (size_t)c->ldl * 4, (size_t)s.vocab * 4, B,
+                                  cudaMemcpyDeviceToDevice, c->stream));
+  argmax_kernel<<<B, 1024, 0, c->stream>>>(c->logits, c->ldl, s.vocab, c->tokens, c->max_seq, c->dstate,
+                                           write_token ? 1 : 0, out_argmax);
+  LAUNCH_OK(c, "argmax_kernel");
+  return DMTD_OK;
+}
+
+// One pass of the decode stage (Section 2.2).  kind 1: full pass - the R = n_known - lo_len
+// pending rows through the lower layers (refill), the newest row through the decoding
+// layers.  kind 2: the newest token's embedding through the decoding layers only.
+dmtd_status enqueue_pass(dmtd_ctx *c, int kind, int R_lower, bool write_token, int *out_argmax, float *out_logits) {
+  const int B = c->B, L = c->s.n_layers, lo = L - c->L_d, H = c->s.hidden;
+  const int newest = c->h.n_known - 1;
+  if (kind == 1 && lo > 0) {
+    TRY(launch_embed(c, &c->dstate->lo_len, B, R_lower, c->x_lo, false));
+    TRY(launch_rope_table(c, &c->dstate->lo_len, R_lower));
+    for (int l = 0; l < lo; ++l) TRY(run_layer(c, l, c->x_lo, B, R_lower, &c->dstate->lo_len, c->h.n_known));
+    select_last_kernel<<<B, 256, 0, c->stream>>>(c->x_lo, R_lower, H, c->x_up);
+    LAUNCH_OK(c, "select_last_kernel");
+    if (c->literal_sum) TRY(launch_embed(c, &c->dstate->newest, B, 1, c->x_up, true));
+  } else {
+    TRY(launch_embed(c, &c->dstate->newest, B, 1, c->x_up, false));
+  }
+  TRY(launch_rope_table(c, &c->dstate->newest, 1));
+  for (int l = lo; l < L; ++l) TRY(run_layer(c, l, c->x_up, B, 1, &c->dstate->newest, newest + 1));
+  TRY(run_head(c, B, write_token, out_argmax, out_logits));
+  advance_state_kernel<<<1, 1, 0, c->stream>>>(c->dstate, kind, 0);
+  LAUNCH_OK(c, "advance_state_kernel");
+  return DMTD_OK;
+}
+
+void host_advance(dmtd_ctx *c, int kind) {
+  dmtd_state &h = c->h;
+  if (kind == 1) { h.lo_len = h.n_known; h.cycle += 1; }
+  h.up_len = h.n_known;
+  h.n_known += 1;
+  h.slot = (h.slot + 1) % h.tau;
+  h.n_emitted += 1;
+}
+
+void drop_graphs(dmtd_ctx *c) {
+  for (int k = 0; k < 3; ++k)
+    if (c->graph_exec[k]) { cudaGraphExecDestroy(c->graph_exec[k]); c->graph_exec[k] = nullptr; }
+}
+
+// Capture a steady-state pass (R_lower = tau) into a graph.  Positions come from the device
+// counters and the attention grid covers max_seq, so one graph serves the whole generation.
+dmtd_status capture_pass(dmtd_ctx *c, int kind) {
+  cudaGraph_t graph = nullptr;
+  int64_t before = c->launches;
+  c->capturing = true;
+  cudaError_t e = cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal);
+  if (e != cudaSuccess) { c->capturing = false; return fail(c, DMTD_ERR_CUDA, "begin capture: %s", cudaGetErrorString(e)); }
+  dmtd_status st = enqueue_pass(c, kind, c->tau, true, nullptr, nullptr);
+  e = cudaStreamEndCapture(c->stream, &graph);
+  c->capturing = false;
+  int nodes = (int)(c->launches - before);
+  c->launches = before;
+  if (st != DMTD_OK) { if (graph) cudaGraphDestroy(graph); return st; }
+  if (e != cudaSuccess) return fail(c, DMTD_ERR_CUDA, "end capture: %s", cudaGetErrorString(e));
+  e = cudaGraphInstantiate(&c->graph_exec[kind], graph, 0);
+  cudaGraphDestroy(graph);
+  if (e != cudaSuccess) return fail(c, DMTD_ERR_CUDA, "graph instantiate: %s", cudaGetErrorString(e));
+  c->graph_nodes[kind] = nodes;
+  return DMTD_OK;
+}
+
+// Run the next pass of the schedule in greedy mode.
+dmtd_status run_greedy_pass(dmtd_ctx *c) {
+  int kind = c->h.slot == 0 ? 1 : 2;
+  int R_lower = c->h.n_known - c->h.lo_len;
+  bool steady = (kind == 2) || (R_lower == c->tau);
+  if (c->use_graph && steady) {
+    if (c->graph_B != c->B || c->graph_tau != c->tau) { drop_graphs(c); c->graph_B = c->B; c->graph_tau = c->tau; }
+    if (!c->graph_exec[kind]) TRY(capture_pass(c, kind));
+    CUDA_TRY(c, cudaGraphLaunch(c->graph_exec[kind], c->stream));
+    c->launches += c->graph_nodes[kind];
+  } else {
+    TRY(enqueue_pass(c, kind, R_lower, true, nullptr, nullptr));
+  }
+  host_advance(c, kind);
+  return DMTD_OK;
+}
+
+dmtd_status validate_shape(const dmtd_model_shape *s, int L_d, int tau, int max_batch, int max_seq) {
+  if (s->n_layers < 1 || s->hidden < 1 || s->n_q_heads < 1 || s->n_kv_heads < 1 || s->intermediate < 1 || s->vocab < 1)
+    return fail(nullptr, DMTD_ERR_SHAPE, "model dimensions must be positive");
+  if (L_d < 1 || L_d > s->n_layers) return fail(nullptr, DMTD_ERR_SHAPE, "L_d must be in [1, n_layers]");
+  if (tau < 1) return fail(nullptr, DMTD_ERR_SHAPE, "tau must be >= 1");
+  if (max_batch < 1 || max_seq < 2) return fail(nullptr, DMTD_ERR_INVALID_ARG, "max_batch >= 1 and max_seq >= 2 required");
+  if (s->n_q_heads % s->n_kv_heads) return fail(nullptr, DMTD_ERR_SHAPE, "n_q_heads must be a multiple of n_kv_heads");
+  if (s->n_q_heads / s->n_kv_heads > ATTN_QR) return fail(nullptr, DMTD_ERR_SHAPE, "at most 16 query heads per kv head");
+  if (s->head_dim != 64 && s->head_dim != 128) return fail(nullptr, DMTD_ERR_SHAPE, "head_dim must be 64 or 128");
+  if (s->weight_dtype != DMTD_F32 && s->weight_dtype != DMTD_BF16) return fail(nullptr, DMTD_ERR_SHAPE, "weight_dtype");
+  if (s->kv_dtype != DMTD_F32 && s->kv_dtype != DMTD_BF16) return fail(nullptr, DMTD_ERR_SHAPE, "kv_dtype");
+  int mult = s->weight_dtype == DMTD_BF16 ? 32 : 4;
+  if (s->hidden % mult || s->intermediate % mult)
+    return fail(nullptr, DMTD_ERR_SHAPE, "hidden and intermediate must be multiples of %d", mult);
+  if (s->weight_dtype == DMTD_BF16 && ((s->n_q_heads * s->head_dim) % 16 || s->intermediate % 16))
+    return fail(nullptr, DMTD_ERR_SHAPE, "fused row blocks must be multiples of 16");
+  if (!s->tied_lm_head) return fail(nullptr, DMTD_ERR_UNSUPPORTED, "only a tied LM head is supported");
+  if (!(s->rope_theta > 0.f) || !(s->rms_eps >= 0.f)) return fail(nullptr, DMTD_ERR_SHAPE, "rope_theta / rms_eps");
+  return DMTD_OK;
+}
+
+}  // namespace
+
+// ================================================================================ C ABI
+
+extern "C" {
+
+dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau, int32_t max_batch,
+                        int32_t max_seq, const dmtd_weights *w, void *cuda_stream, dmtd_ctx **out) {
+  if (!shape || !w || !out || !w->embed || !w->final_norm || !w->layers)
+    return fail(nullptr, DMTD_ERR_INVALID_ARG, "null argument");
+  if (w->lm_head) return fail(nullptr, DMTD_ERR_UNSUPPORTED, "only a tied LM head is supported (lm_head must be NULL)");
+  dmtd_status vs = validate_shape(shape, L_d, tau, max_batch, max_seq);
+  if (vs != DMTD_OK) return vs;
+
+  dmtd_ctx *c = new dmtd_ctx();
+  auto bail = [&](dmtd_status st) { g_create_error = c->err; dmtd_destroy(c); return st; };
+#define CTRY(expr) do { dmtd_status s__ = (expr); if (s__ != DMTD_OK) return bail(s__); } while (0)
+#define CCUDA(expr) do { cudaError_t e__ = (expr); if (e__ != cudaSuccess) { \
+    fail(c, DMTD_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); return bail(DMTD_ERR_CUDA); } } while (0)
+
+  c->s = *shape; c->L_d = L_d; c->tau = tau; c->max_batch = max_batch; c->max_seq = max_seq;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  CCUDA(cudaGetDevice(&c->device));
+  CCUDA(cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->device));
+  const dmtd_model_shape &s = c->s;
+  const int H = s.hidden, D = s.head_dim, QD = s.n_q_heads * D, KVD = s.n_kv_heads * D, I = s.intermediate;
+
+  // weights
+  c->layers.resize(s.n_layers);
+  for (int l = 0; l < s.n_layers; ++l) {
+    const dmtd_layer_weights &lw = w->layers[l];
+    const void *ptrs[] = {lw.input_norm, lw.q_proj, lw.k_proj, lw.v_proj, lw.q_norm, lw.k_norm, lw.o_proj,
+                          lw.post_norm, lw.gate_proj, lw.up_proj, lw.down_proj};
+    for (const void *p : ptrs)
+      if (!p) { fail(c, DMTD_ERR_INVALID_ARG, "null weight pointer in layer %d", l); return bail(DMTD_ERR_INVALID_ARG); }
+    LayerDev &ld = c->layers[l];
+    const void *qkv_src[3] = {lw.q_proj, lw.k_proj, lw.v_proj};
+    int qkv_n[3] = {QD, KVD, KVD};
+    CTRY(pack_matrix(c, &ld.qkv, H, qkv_src, qkv_n, 3));
+    const void *o_src[1] = {lw.o_proj}; int o_n[1] = {H};
+    CTRY(pack_matrix(c, &ld.o, QD, o_src, o_n, 1));
+    const void *gu_src[2] = {lw.gate_proj, lw.up_proj}; int gu_n[2] = {I, I};
+    CTRY(pack_matrix(c, &ld.gu, H, gu_src, gu_n, 2));
+    const void *d_src[1] = {lw.down_proj}; int d_n[1] = {H};
+    CTRY(pack_matrix(c, &ld.down, I, d_src, d_n, 1));
+    CTRY(vec_to_float(c, &ld.w_in, lw.input_norm, H));
+    CTRY(vec_to_float(c, &ld.w_post, lw.post_norm, H));
+    CTRY(vec_to_float(c, &ld.w_qn, lw.q_norm, D));
+    CTRY(vec_to_float(c, &ld.w_kn, lw.k_norm, D));
+  }
+  {
+    const void *e_src[1] = {w->embed}; int e_n[1] = {s.vocab};
+    CTRY(pack_matrix(c, &c->embed, H, e_src, e_n, 1));
+    CTRY(vec_to_float(c, &c->w_final, w->final_norm, H));
+  }
+  {
+    std::vector<double> f(D / 2);
+    for (int i = 0; i < D / 2; ++i) f[i] = std::pow((double)s.rope_theta, -2.0 * i / (double)D);
+    CTRY(dev_alloc(c, &c->inv_freq, f.size()));
+    CCUDA(cudaMemcpyAsync(c->inv_freq, f.data(), f.size() * sizeof(double), cudaMemcpyHostToDevice, c->stream));
+    CCUDA(cudaStreamSynchronize(c->stream));
+  }
+
+  // sequence state
+  size_t kvb = s.kv_dtype == DMTD_BF16 ? 2 : 4;
+  c->kv_layer_elems = (size_t)max_batch * s.n_kv_heads * max_seq * D;
+  {
+    unsigned char *p = nullptr;
+    CTRY(dev_alloc(c, &p, c->kv_layer_elems * s.n_layers * kvb)); c->kc = p;
+    CTRY(dev_alloc(c, &p, c->kv_layer_elems * s.n_layers * kvb)); c->vc = p;
+  }
+  CTRY(dev_alloc(c, &c->tokens, (size_t)max_batch * max_seq));
+  CTRY(dev_alloc(c, &c->dstate, 1));
+
+  // workspace
+  c->ws_rows = std::max(256, max_batch * std::max(tau, 8));
+  c->lda = std::max(H, std::max(QD, I));
+  c->ldqkv = QD + 2 * KVD; c->ldgu = 2 * I; c->ldl = (s.vocab + 15) / 16 * 16;
+  c->CH = max_seq <= 2048 ? 64 : 256;
+  c->nsplit_max = (max_seq + c->CH - 1) / c->CH;
+  CTRY(dev_alloc(c, &c->x_lo, (size_t)c->ws_rows * H));
+  CTRY(dev_alloc(c, &c->x_up, (size_t)max_batch * H));
+  CTRY(dev_alloc(c, &c->act, (size_t)c->ws_rows * c->lda));
+  CTRY(dev_alloc(c, &c->qkv, (size_t)c->ws_rows * c->ldqkv));
+  CTRY(dev_alloc(c, &c->gu, (size_t)c->ws_rows * c->ldgu));
+  CTRY(dev_alloc(c, &c->logits, (size_t)max_batch * c->ldl));
+  CTRY(dev_alloc(c, &c->part_o, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * D));
+  CTRY(dev_alloc(c, &c->part_ml, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * 2));
+  CTRY(dev_alloc(c, &c->rope_tab, (size_t)c->ws_rows * (D / 2)));
+  CTRY(dmtd_reset(c));
+  CCUDA(cudaStreamSynchronize(c->stream));   // repacking done: the caller may free its weights
+#undef CTRY
+#undef CCUDA
+  *out = c;
+  return DMTD_OK;
+}
+
+void dmtd_destroy(dmtd_ctx *c) {
+  if (!c) return;
+  if (c->stream || true) cudaStreamSynchronize(c->stream);
+  drop_graphs(c);
+  for (void *p : c->allocs) cudaFree(p);
+  delete c;
+}
+
+dmtd_status dmtd_reset(dmtd_ctx *c) {
+  if (!c) return DMTD_ERR_INVALID_ARG;
+  DevState z{};
+  z.tau = c->tau;
+  CUDA_TRY(c, cudaMemcpyAsync(c->dstate, &z, sizeof z, cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  c->h = dmtd_state{};
+  c->h.tau = c->tau; c->h.L_d = c->L_d;
+  c->prefilled = false; c->B = 0;
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_prefill(dmtd_ctx *c, const int32_t *prompt, int32_t B, int32_t P, const int32_t *forced_first,
+                         int32_t *out_token, float *out_logits) {
+  if (!c) return DMTD_ERR_INVALID_ARG;
+  if (!prompt || B < 1 || P < 1) return fail(c, DMTD_ERR_INVALID_ARG, "prefill: null prompt or non-positive size");
+  if (c->prefilled) return fail(c, DMTD_ERR_STATE, "prefill: context already holds a sequence; call dmtd_reset first");
+  if (B > c->max_batch || P + 1 > c->max_seq) return fail(c, DMTD_ERR_CAPACITY, "prefill: B=%d P=%d exceed max_batch=%d max_seq=%d", B, P, c->max_batch, c->max_seq);
+  const int L = c->s.n_layers, lo = L - c->L_d;
+  c->B = B;
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->tokens, (size_t)c->max_seq * 4, prompt, (size_t)P * 4, (size_t)P * 4, B,
+                                cudaMemcpyDeviceToDevice, c->stream));
+  // All prompt rows through all layers (Section 2.2: the prefill is pass 1 of cycle 1), in
+  // causal chunks of rows that fit the workspace.
+  const int Rc_max = std::max(1, c->ws_rows / B);
+  int last_R = 0;
+  for (int p0 = 0; p0 < P; p0 += Rc_max) {
+    int R = std::min(Rc_max, P - p0);
+    set_int_kernel<<<1, 1, 0, c->stream>>>(&c->dstate->scratch, p0);
+    LAUNCH_OK(c, "set_int_kernel");
+    TRY(launch_embed(c, &c->dstate->scratch, B, R, c->x_lo, false));
+    TRY(launch_rope_table(c, &c->dstate->scratch, R));
+    for (int l = 0; l < L; ++l) {
+      if (l == lo && c->literal_sum && lo > 0) TRY(launch_embed(c, &c->dstate->scratch, B, R, c->x_lo, true));
+      TRY(run_layer(c, l, c->x_lo, B, R, &c->dstate->scratch, p0 + R));
+    }
+    last_R = R;
+  }
+  select_last_kernel<<<B, 256, 0, c->stream>>>(c->x_lo, last_R, c->s.hidden, c->x_up);
+  LAUNCH_OK(c, "select_last_kernel");
+  // n_known must read P when the head writes the token
+  set_int_kernel<<<1, 1, 0, c->stream>>>(&c->dstate->n_known, P);
+  LAUNCH_OK(c, "set_int_kernel");
+  TRY(run_head(c, B, forced_first == nullptr, out_token, out_logits));
+  if (forced_first)
+    CUDA_TRY(c, cudaMemcpy2DAsync(c->tokens + P, (size_t)c->max_seq * 4, forced_first, 4, 4, B,
+                                  cudaMemcpyDeviceToDevice, c->stream));
+  advance_state_kernel<<<1, 1, 0, c->stream>>>(c->dstate, 0, P);
+  LAUNCH_OK(c, "advance_state_kernel");
+  c->h.n_known = P + 1; c->h.lo_len = P; c->h.up_len = P; c->h.cycle = 1;
+  c->h.slot = 1 % c->tau; c->h.n_emitted = 1;
+  c->prefilled = true;
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_decode_cycle(dmtd_ctx *c, int32_t max_new, int32_t *out_tokens, int32_t *n_out) {
+  if (!c) return DMTD_ERR_INVALID_ARG;
+  if (!n_out || max_new < 0) return fail(c, DMTD_ERR_INVALID_ARG, "decode_cycle: n_out is null or max_new < 0");
+  *n_out = 0;
+  if (!c->prefilled) return fail(c, DMTD_ERR_STATE, "decode_cycle: no prefill yet");
+  const int first = c->h.n_known;
+  int n = 0;
+  dmtd_status rc = DMTD_OK;
+  while (n < max_new) {
+    if (c->h.n_known + 1 > c->max_seq) { rc = fail(c, DMTD_ERR_CAPACITY, "decode_cycle: position %d does not fit max_seq=%d", c->h.n_known, c->max_seq); break; }
+    TRY(run_greedy_pass(c));
+    ++n;
+    if (c->h.slot == 0) break;     // the cycle is complete
+  }
+  if (out_tokens && n > 0) {
+    gather_tokens_kernel<<<c->B, 32, 0, c->stream>>>(c->tokens, c->max_seq, first, n, c->tau, out_tokens);
+    LAUNCH_OK(c, "gather_tokens_kernel");
+  }
+  *n_out = n;
+  return rc;
+}
+
+dmtd_status dmtd_decode_forced(dmtd_ctx *c, const int32_t *forced, int32_t n, float *out_logits, int32_t *out_argmax) {
+  if (!c) return DMTD_ERR_INVALID_ARG;
+  if (!forced || n < 0) return fail(c, DMTD_ERR_INVALID_ARG, "decode_forced: null forced tokens or n < 0");
+  if (!c->prefilled) return fail(c, DMTD_ERR_STATE, "decode_forced: no prefill yet");
+  if (c->h.n_known + n > c->max_seq) return fail(c, DMTD_ERR_CAPACITY, "decode_forced: %d more positions do not fit max_seq=%d", n, c->max_seq);
+  if (n == 0) return DMTD_OK;
+  // the forced tokens are the sequence's next n tokens: place them, then run the schedule
+  // without letting the head overwrite them
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->tokens + c->h.n_known, (size_t)c->max_seq * 4, forced, (size_t)n * 4, (size_t)n * 4,
+                                c->B, cudaMemcpyDeviceToDevice, c->stream));
+  const size_t BV = (size_t)c->B * c->s.vocab;
+  for (int i = 0; i < n; ++i) {
+    int kind = c->h.slot == 0 ? 1 : 2;
+    TRY(enqueue_pass(c, kind, c->h.n_known - c->h.lo_len, false, out_argmax ? out_argmax + (size_t)i * c->B : nullptr,
+                     out_logits ? out_logits + (size_t)i * BV : nullptr));
+    host_advance(c, kind);
+  }
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_step_layers(dmtd_ctx *c, int32_t l0, int32_t l1, float *hidden, int32_t B, int32_t R, int32_t pos0) {
+  if (!c) return DMTD_ERR_INVALID_ARG;
+  if (!hidden || l0 < 0 || l1 > c->s.n_layers || l0 > l1 || B < 1 || R < 1 || pos0 < 0)
+    return fail(c, DMTD_ERR_INVALID_ARG, "step_layers: bad layer range, sizes or null hidden");
+  if (B > c->max_batch || pos0 + R > c->max_seq || B * R > c->ws_rows)
+    return fail(c, DMTD_ERR_CAPACITY, "step_layers: B=%d R=%d pos0=%d exceed max_batch=%d max_seq=%d rows=%d", B, R, pos0, c->max_batch, c->max_seq, c->ws_rows);
+  set_int_kernel<<<1, 1, 0, c->stream>>>(&c->dstate->scratch, pos0);
+  LAUNCH_OK(c, "set_int_kernel");
+  TRY(launch_rope_table(c, &c->dstate->scratch, R));
+  for (int l = l0; l < l1; ++l) TRY(run_layer(c, l, hidden, B, R, &c->dstate->scratch, pos0 + R));
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_prefill_host(dmtd_ctx *c, const int32_t *prompt_host, int32_t B, int32_t P, int32_t *out_token_host) {
+  if (!c) return DMTD_ERR_INVALID_ARG;
+  if (!prompt_host || B < 1 || P < 1) return fail(c, DMTD_ERR_INVALID_ARG, "prefill_host: null prompt or non-positive size");
+  if (c->prefilled) return fail(c, DMTD_ERR_STATE, "prefill_host: context already holds a sequence; call dmtd_reset first");
+  if (B > c->max_batch || P + 1 > c->max_seq) return fail(c, DMTD_ERR_CAPACITY, "prefill_host: sizes exceed capacity");
+  // stage the prompt at the tail of the act workspace (unused until the first layer runs)
+  int *stage = reinterpret_cast<int *>(c->gu);
+  if ((size_t)B * P > (size_t)c->ws_rows * c->ldgu) return fail(c, DMTD_ERR_CAPACITY, "prefill_host: prompt larger than staging space");
+  CUDA_TRY(c, cudaMemcpyAsync(stage, prompt_host, (size_t)B * P * 4, cudaMemcpyHostToDevice, c->stream));
+  // the token buffer copy inside dmtd_prefill reads `stage` before any layer writes gu
+  TRY(dmtd_prefill(c, stage, B, P, nullptr, nullptr, nullptr));
+  if (out_token_host)
+    CUDA_TRY(c, cudaMemcpy2DAsync(out_token_host, 4, c->tokens + P, (size_t)c->max_seq * 4, 4, B, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_decode_cycle_host(dmtd_ctx *c, int32_t max_new, int32_t *out_tokens_host, int32_t *n_out) {
+  if (!c) return DMTD_ERR_INVALID_ARG;
+  if (!n_out) return fail(c, DMTD_ERR_INVALID_ARG, "decode_cycle_host: n_out is null");
+  const int first = c->h.n_known;
+  dmtd_status rc = dmtd_decode_cycle(c, max_new, nullptr, n_out);
+  if (rc != DMTD_OK && rc != DMTD_ERR_CAPACITY) return rc;
+  if (out_tokens_host && *n_out > 0)
+    CUDA_TRY(c, cudaMemcpy2DAsync(out_tokens_host, (size_t)c->tau * 4, c->tokens + first, (size_t)c->max_seq * 4,
+                                  (size_t)*n_out * 4, c->B, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return rc;
+}
+
+dmtd_status dmtd_get_state(const dmtd_ctx *c, dmtd_state *out) {
+  if (!c || !out) return DMTD_ERR_INVALID_ARG;
+  *out = c->h;
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_get_device_state(dmtd_ctx *c, dmtd_state *out) {
+  if (!c || !out) return DMTD_ERR_INVALID_ARG;
+  DevState d{};
+  CUDA_TRY(c, cudaMemcpyAsync(&d, c->dstate, sizeof d, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (d.error) return fail(c, DMTD_ERR_INVALID_ARG, "a token id outside [0, vocab) reached the embedding gather");
+  out->n_known = d.n_known; out->lo_len = d.lo_len; out->up_len = d.up_len; out->cycle = d.cycle;
+  out->slot = d.slot; out->n_emitted = d.n_emitted; out->tau = d.tau; out->L_d = c->L_d;
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_set_tau(dmtd_ctx *c, int32_t tau) {
+  if (!c) return DMTD_ERR_INVALID_ARG;
+  if (tau < 1) return fail(c, DMTD_ERR_SHAPE, "set_tau: tau must be >= 1");
+  if (c->prefilled && c->h.slot != 0) return fail(c, DMTD_ERR_STATE, "set_tau: only at a cycle boundary");
+  if (c->max_batch * tau > c->ws_rows) return fail(c, DMTD_ERR_CAPACITY, "set_tau: workspace too small for tau=%d", tau);
+  c->tau = tau; c->h.tau = tau;
+  CUDA_TRY(c, cudaMemcpyAsync(&c->dstate->tau, &c->tau, sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_set_option(dmtd_ctx *c, const char *name, int64_t value) {
+  if (!c || !name) return DMTD_ERR_INVALID_ARG;
+  if (value != 0 && value != 1) return fail(c, DMTD_ERR_INVALID_ARG, "option %s takes 0 or 1", name);
+  if (!strcmp(name, "cuda_graph")) { c->use_graph = value != 0; return DMTD_OK; }
+  if (!strcmp(name, "literal_sum")) { c->literal_sum = value != 0; drop_graphs(c); return DMTD_OK; }
+  return fail(c, DMTD_ERR_INVALID_ARG, "unknown option %s", name);
+}
+
+dmtd_status dmtd_get_kv(dmtd_ctx *c, int32_t layer, void **k, void **v) {
+  if (!c || layer < 0 || layer >= c->s.n_layers) return DMTD_ERR_INVALID_ARG;
+  size_t kvb = c->s.kv_dtype == DMTD_BF16 ? 2 : 4;
+  if (k) *k = static_cast<unsigned char *>(c->kc) + (size_t)layer * c->kv_layer_elems * kvb;
+  if (v) *v = static_cast<unsigned char *>(c->vc) + (size_t)layer * c->kv_layer_elems * kvb;
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_get_launch_count(const dmtd_ctx *c, int64_t *out) {
+  if (!c || !out) return DMTD_ERR_INVALID_ARG;
+  *out = c->launches;
+  return DMTD_OK;
+}
+
+const char *dmtd_status_str(dmtd_status s) {
+  switch (s) {
+    case DMTD_OK: return "ok";
+    case DMTD_ERR_INVALID_ARG: return "invalid argument";
+    case DMTD_ERR_SHAPE: return "unsupported shape";
+    case DMTD_ERR_STATE: return "call out of order";
+    case DMTD_ERR_CAPACITY: return "capacity exceeded";
+    case DMTD_ERR_CUDA: return "CUDA error";
+    case DMTD_ERR_TIMEOUT: return "device wait timed out";
+    case DMTD_ERR_UNSUPPORTED: return "unsupported";
+  }
+  return "unknown status";
+}
+
+const char *dmtd_last_error(const dmtd_ctx *c) { return c ? c->err.c_str() : g_create_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,224 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from synthetic import SHAPES, make_prompts, make_weights
+
+from helpers import (LOGIT_ATOL, check_logits, gpu_forced, oracle_forced, oracle_greedy, to_cuda)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dmtd():
+    import paper_2510_11958_b200 as pkg
+    pkg.load_library()
+    return pkg
+
+
+def _engine(dmtd, shape, wc, L_d, tau, max_batch, max_seq, **kw):
+    return dmtd.Dmtd(shape, wc, L_d=L_d, tau=tau, max_batch=max_batch, max_seq=max_seq, **kw)
+
+
+CASES = [
+    # name, shape, dtype, L_d, tau, B, P, n_new
+    ("tiny_f32_tau3", "tiny", "f32", 2, 3, 1, 32, 24),
+    ("tiny_f32_tau1", "tiny", "f32", 2, 1, 1, 32, 24),
+    ("tiny_bf16_tau3", "tiny", "bf16", 2, 3, 1, 32, 24),
+    ("tiny_bf16_b3_tau4", "tiny", "bf16", 1, 4, 3, 7, 14),
+    ("mid_bf16_tau3", "mid", "bf16", 2, 3, 2, 37, 13),
+    ("mid_bf16_tau2_b5", "mid", "bf16", 4, 2, 5, 9, 8),
+    ("mid_bf16_Ld_all", "mid", "bf16", 6, 3, 1, 11, 7),
+]
+
+
+@pytest.mark.parametrize("name,shape_name,dtype,L_d,tau,B,P,n_new", CASES, ids=[c[0] for c in CASES])
+def test_teacher_forced_logits_and_state(dmtd, name, shape_name, dtype, L_d, tau, B, P, n_new):
+    shape = SHAPES[shape_name].with_(dtype=dtype)
+    w = make_weights(shape, seed=0, norm_jitter=0.1)
+    prompts = make_prompts(shape.vocab, B, P, seed=1).numpy()
+    # teacher sequence: what the oracle itself generates greedily
+    toks, _, _, _ = oracle_greedy(shape, w, L_d, tau, prompts, n_new)
+    ref_logits, ref_am, o = oracle_forced(shape, w, L_d, tau, prompts, toks)
+    eng = _engine(dmtd, shape, to_cuda(w), L_d, tau, B, P + n_new + 1)
+    got_logits, got_am = gpu_forced(eng, prompts, toks)
+    err, clear = check_logits(got_logits, ref_logits, got_am, ref_am)
+    assert eng.state() == o.state()
+    assert eng.device_state() == o.state()
+    print(f"{name}: max|dlogit|={err:.2e}, clear-margin steps {clear:.0%}")
+
+
+@pytest.mark.parametrize("graph", [0, 1])
+@pytest.mark.parametrize("shape_name,dtype,L_d,tau,B,P,n_new", [("tiny", "f32", 2, 3, 1, 32, 24),
+                                                               ("mid", "bf16", 2, 3, 2, 20, 17),
+                                                               ("tiny", "bf16", 2, 1, 2, 5, 6)])
+def test_free_running_greedy(dmtd, graph, shape_name, dtype, L_d, tau, B, P, n_new):
+    """Greedy generation call by call: token counts, state after every call (bit-exact), and the
+    tokens themselves up to the first step where the oracle's margin is not clear."""
+    shape = SHAPES[shape_name].with_(dtype=dtype)
+    w = make_weights(shape, seed=0, norm_jitter=0.1)
+    prompts = make_prompts(shape.vocab, B, P, seed=1).numpy()
+    toks, logits, states, _ = oracle_greedy(shape, w, L_d, tau, prompts, n_new)
+    eng = _engine(dmtd, shape, to_cuda(w), L_d, tau, B, P + n_new + 1)
+    eng.set_option("cuda_graph", graph)
+    tok, _ = eng.prefill(torch.from_numpy(prompts).cuda())
+    got = [tok.cpu().numpy()]
+    assert eng.state() == states[0]
+    k = 1
+    while len(got) < n_new:
+        rc, n, out = eng.decode_cycle(n_new - len(got))
+        out = out.cpu().numpy()
+        got += [out[:, i] for i in range(n)]
+        assert eng.state() == states[k]
+        assert eng.device_state() == states[k]
+        k += 1
+    got = np.stack(got, 1)
+    srt = np.sort(logits, -1)
+    clear = (srt[..., -1] - srt[..., -2] > 5e-2).T            # [B, n]
+    for b in range(B):
+        upto = n_new if clear[b].all() else int(np.argmin(clear[b]))
+        assert (got[b, :upto] == toks[b, :upto]).all()
+
+
+def test_graph_replay_matches_plain_launches(dmtd):
+    shape = SHAPES["mid"]
+    w = to_cuda(make_weights(shape, seed=0))
+    prompts = torch.from_numpy(make_prompts(shape.vocab, 2, 16, seed=1).numpy()).cuda()
+    outs = []
+    for graph in (0, 1):
+        eng = _engine(dmtd, shape, w, 2, 3, 2, 64)
+        eng.set_option("cuda_graph", graph)
+        eng.prefill(prompts)
+        toks = []
+        for _ in range(6):
+            rc, n, out = eng.decode_cycle(3)
+            toks.append(out[:, :n].clone())
+        outs.append(torch.cat(toks, 1).cpu())
+        assert eng.launch_count() > 0
+    assert (outs[0] == outs[1]).all()
+
+
+def test_prefill_longer_than_one_chunk(dmtd):
+    """A prompt that does not fit the workspace in one go is fed in causal chunks."""
+    shape = SHAPES["tiny"].with_(dtype="bf16")
+    w = make_weights(shape, seed=0)
+    P = 300                                   # workspace holds 256 rows
+    prompts = make_prompts(shape.vocab, 1, P, seed=1).numpy()
+    forced = make_prompts(shape.vocab, 1, 4, seed=2).numpy()
+    ref_logits, ref_am, o = oracle_forced(shape, w, 2, 3, prompts, forced)
+    eng = _engine(dmtd, shape, to_cuda(w), 2, 3, 1, P + 8)
+    got_logits, got_am = gpu_forced(eng, prompts, forced)
+    check_logits(got_logits, ref_logits, got_am, ref_am)
+    assert eng.device_state() == o.state()
+
+
+@pytest.mark.parametrize("shape_name,dtype,B,R,pos0", [("tiny", "f32", 2, 3, 5), ("mid", "bf16", 3, 3, 17),
+                                                      ("mid", "bf16", 1, 1, 40), ("mid", "bf16", 2, 19, 0)])
+def test_step_layers_hidden_and_kv(dmtd, shape_name, dtype, B, R, pos0):
+    """dmtd_step_layers against the oracle's: output rows and the K/V they append."""
+    import oracle
+    shape = SHAPES[shape_name].with_(dtype=dtype)
+    w = make_weights(shape, seed=3, norm_jitter=0.1)
+    L = shape.n_layers
+    g = torch.Generator().manual_seed(5)
+    max_seq = pos0 + R + 2
+    o = oracle.Oracle(shape, w, L_d=1, tau=1, max_batch=B, max_seq=max_seq)
+    eng = _engine(dmtd, shape, to_cuda(w), 1, 1, B, max_seq)
+    # history: run pos0 earlier rows through both so the caches hold the same past
+    if pos0:
+        h0 = torch.randn(B, pos0, shape.hidden, generator=g) * 0.5
+        o.step_layers(0, L, h0.double().numpy(), 0)
+        eng.step_layers(0, L, h0.cuda().contiguous(), 0)
+    h = torch.randn(B, R, shape.hidden, generator=g) * 0.5
+    ref = o.step_layers(1, L, h.double().numpy(), pos0) if L > 2 else o.step_layers(0, L, h.double().numpy(), pos0)
+    l0 = 1 if L > 2 else 0
+    got = eng.step_layers(l0, L, h.cuda().contiguous(), pos0)
+    torch.cuda.synchronize()
+    scale = np.abs(ref).max()
+    assert np.abs(got.double().cpu().numpy() - ref).max() <= 2e-3 * max(1.0, scale)
+    # appended K/V of the last layer
+    import ctypes
+    kp, vp = eng.kv(L - 1)
+    kvdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    n = B * shape.n_kv_heads * max_seq * shape.head_dim
+    for ptr, which in ((kp, 0), (vp, 1)):
+        buf = torch.empty(n, dtype=kvdt, device="cuda")
+        ctypes.CDLL("libcudart.so").cudaMemcpy(ctypes.c_void_p(buf.data_ptr()), ctypes.c_void_p(ptr),
+                                               ctypes.c_size_t(n * buf.element_size()), 3)
+        dev = buf.view(B, shape.n_kv_heads, max_seq, shape.head_dim).double().cpu().numpy()
+        for b in range(B):
+            refkv = o.kv_cache(L - 1, b, pos0 + R)[which]            # [pos, nkv, d]
+            gotkv = dev[b].transpose(1, 0, 2)[: pos0 + R]
+            tol = 1e-5 if dtype == "f32" else 2.0 ** -8 * max(1.0, np.abs(refkv).max())
+            assert np.abs(gotkv - refkv).max() <= tol
+
+
+def test_batch_rows_are_independent(dmtd):
+    shape = SHAPES["mid"]
+    w = to_cuda(make_weights(shape, seed=0))
+    prompts = make_prompts(shape.vocab, 4, 12, seed=1)
+    forced = make_prompts(shape.vocab, 4, 9, seed=2)
+    eng = _engine(dmtd, shape, w, 2, 3, 4, 32)
+    full, _ = gpu_forced(eng, prompts.numpy(), forced.numpy())
+    for b in (0, 3):
+        e1 = _engine(dmtd, shape, w, 2, 3, 1, 32)
+        one, _ = gpu_forced(e1, prompts[b:b + 1].numpy(), forced[b:b + 1].numpy())
+        assert np.abs(one[:, 0] - full[:, b]).max() < 1e-3
+
+
+def test_literal_sum_option(dmtd):
+    """The literal reading of Eq. 4 (embedding added to the lower-stack output)."""
+    shape = SHAPES["tiny"]
+    w = make_weights(shape, seed=0)
+    prompts = make_prompts(shape.vocab, 1, 9, seed=1).numpy()
+    forced = make_prompts(shape.vocab, 1, 8, seed=2).numpy()
+    ref_logits, ref_am, _ = oracle_forced(shape, w, 2, 3, prompts, forced, literal_sum=True)
+    eng = _engine(dmtd, shape, to_cuda(w), 2, 3, 1, 32)
+    eng.set_option("literal_sum", 1)
+    got_logits, got_am = gpu_forced(eng, prompts, forced)
+    check_logits(got_logits, ref_logits, got_am, ref_am)
+
+
+def test_reset_and_set_tau(dmtd):
+    shape = SHAPES["tiny"]
+    w = make_weights(shape, seed=0)
+    prompts = make_prompts(shape.vocab, 1, 6, seed=1).numpy()
+    forced = make_prompts(shape.vocab, 1, 7, seed=2).numpy()
+    eng = _engine(dmtd, shape, to_cuda(w), 2, 3, 1, 32)
+    gpu_forced(eng, prompts, forced)
+    eng.reset()
+    eng.set_tau(2)
+    ref_logits, ref_am, o = oracle_forced(shape, w, 2, 2, prompts, forced)
+    got_logits, got_am = gpu_forced(eng, prompts, forced)
+    check_logits(got_logits, ref_logits, got_am, ref_am)
+    assert eng.device_state() == o.state()
+
+
+def test_errors(dmtd):
+    shape = SHAPES["tiny"]
+    w = to_cuda(make_weights(shape, seed=0))
+    S = __import__("paper_2510_11958_b200.binding", fromlist=["STATUS"]).STATUS
+    with pytest.raises(dmtd.DmtdError) as e:
+        _engine(dmtd, shape, w, 5, 3, 1, 32)
+    assert e.value.status == S["SHAPE"]
+    with pytest.raises(dmtd.DmtdError) as e:
+        _engine(dmtd, shape, w, 2, 0, 1, 32)
+    assert e.value.status == S["SHAPE"]
+    eng = _engine(dmtd, shape, w, 2, 3, 1, 8)
+    with pytest.raises(dmtd.DmtdError) as e:
+        eng.decode_cycle(3)
+    assert e.value.status == S["STATE"]
+    prompts = torch.from_numpy(make_prompts(shape.vocab, 1, 5, seed=1).numpy()).cuda()
+    with pytest.raises(dmtd.DmtdError) as e:
+        eng.prefill(torch.cat([prompts, prompts], 0))
+    assert e.value.status == S["CAPACITY"]
+    eng.prefill(prompts)
+    with pytest.raises(dmtd.DmtdError) as e:
+        eng.prefill(prompts)
+    assert e.value.status == S["STATE"]
+    rc, n, _ = eng.decode_cycle(3)
+    assert rc == 0 and n == 2
+    rc, n, _ = eng.decode_cycle(3, allow_capacity=True)     # position 8 does not fit max_seq = 8
+    assert rc == S["CAPACITY"] and n == 0
+    assert eng.device_state() == eng.state()
