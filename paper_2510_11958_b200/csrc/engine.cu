@@ -33,6 +33,7 @@ struct dmtd_ctx {
   int L_d = 0, tau = 0, max_batch = 0, max_seq = 0;
   int device = 0, n_sms = 0;
   cudaStream_t stream = nullptr;
+  cudaStream_t capture_stream = nullptr;    // graphs are recorded here (the caller's stream may be the legacy one)
   std::string err;
   std::vector<void *> allocs;
 
@@ -345,12 +346,16 @@ void drop_graphs(dmtd_ctx *c) {
 dmtd_status capture_pass(dmtd_ctx *c, int kind) {
   cudaGraph_t graph = nullptr;
   int64_t before = c->launches;
+  if (!c->capture_stream) CUDA_TRY(c, cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking));
+  cudaError_t e = cudaStreamBeginCapture(c->capture_stream, cudaStreamCaptureModeThreadLocal);
+  if (e != cudaSuccess) return fail(c, DMTD_ERR_CUDA, "begin capture: %s", cudaGetErrorString(e));
+  cudaStream_t user_stream = c->stream;
+  c->stream = c->capture_stream;
   c->capturing = true;
-  cudaError_t e = cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal);
-  if (e != cudaSuccess) { c->capturing = false; return fail(c, DMTD_ERR_CUDA, "begin capture: %s", cudaGetErrorString(e)); }
   dmtd_status st = enqueue_pass(c, kind, c->tau, true, nullptr, nullptr);
-  e = cudaStreamEndCapture(c->stream, &graph);
+  e = cudaStreamEndCapture(c->capture_stream, &graph);
   c->capturing = false;
+  c->stream = user_stream;
   int nodes = (int)(c->launches - before);
   c->launches = before;
   if (st != DMTD_OK) { if (graph) cudaGraphDestroy(graph); return st; }
@@ -501,6 +506,7 @@ void dmtd_destroy(dmtd_ctx *c) {
   if (!c) return;
   if (c->stream || true) cudaStreamSynchronize(c->stream);
   drop_graphs(c);
+  if (c->capture_stream) cudaStreamDestroy(c->capture_stream);
   for (void *p : c->allocs) cudaFree(p);
   delete c;
 }

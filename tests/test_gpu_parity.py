@@ -164,7 +164,10 @@ def test_batch_rows_are_independent(dmtd):
     for b in (0, 3):
         e1 = _engine(dmtd, shape, w, 2, 3, 1, 32)
         one, _ = gpu_forced(e1, prompts[b:b + 1].numpy(), forced[b:b + 1].numpy())
-        assert np.abs(one[:, 0] - full[:, b]).max() < 1e-3
+        # not bit-equal: the fp32 reduction order differs with the batch size, and a last-bit
+        # change in k or v can flip its bf16 rounding in the cache; mixing up sequences would
+        # show as O(0.1)
+        assert np.abs(one[:, 0] - full[:, b]).max() < 5e-3
 
 
 def test_literal_sum_option(dmtd):
