@@ -26,6 +26,7 @@
 #ifndef DMTD_H
 #define DMTD_H
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -133,6 +134,26 @@ dmtd_status dmtd_decode_forced(dmtd_ctx *ctx, const int32_t *forced, int32_t n,
 dmtd_status dmtd_step_layers(dmtd_ctx *ctx, int32_t l0, int32_t l1, float *hidden, int32_t B,
                              int32_t R, int32_t pos0);
 
+/* Step a4 on its own: split-KV attention of R new rows per sequence against a KV cache (the
+ * attention of Section 2.2's passes needs the cached K and V of every earlier token), with the
+ * online-softmax merge of the key slices.  No context is needed.
+ *   q        device float [B][R][n_q_heads][head_dim], already normalised, rotated (not scaled)
+ *   k, v     device [B][n_kv_heads][max_seq][head_dim] in kv_dtype; row r of a sequence sits at
+ *            position pos0 + r and attends to positions [0, pos0 + r]; K and V of the R new
+ *            positions must already be in the cache
+ *   scratch  device memory of at least dmtd_attention_scratch_bytes(...) bytes, 256-byte
+ *            aligned, owned by the caller; holds the per-slice partial results while the call's
+ *            kernels run on `cuda_stream` (calls sharing one scratch must be stream-ordered)
+ *   out      device float [B][R][n_q_heads][head_dim]
+ * Errors: SHAPE for head_dim not 64/128, n_q_heads % n_kv_heads != 0 or more than 16 query
+ * heads per KV head; CAPACITY if pos0 + R > max_seq or scratch_bytes is too small. */
+size_t dmtd_attention_scratch_bytes(int32_t B, int32_t R, int32_t n_q_heads, int32_t head_dim,
+                                    int32_t n_keys);
+dmtd_status dmtd_attention_decode(const float *q, const void *k, const void *v, int32_t kv_dtype,
+                                  int32_t B, int32_t R, int32_t n_q_heads, int32_t n_kv_heads,
+                                  int32_t head_dim, int32_t max_seq, int32_t pos0, void *scratch,
+                                  size_t scratch_bytes, float *out, void *cuda_stream);
+
 /* Host-buffer forms of prefill and decode_cycle (same semantics; the copies to and from the
  * device are part of the call, which returns after the stream has drained).
  *   prompt_host [B][P], out_token_host [B], out_tokens_host [B][tau] */
@@ -166,7 +187,7 @@ dmtd_status dmtd_get_kv(dmtd_ctx *ctx, int32_t layer, void **k, void **v);
 dmtd_status dmtd_get_launch_count(const dmtd_ctx *ctx, int64_t *out);
 
 const char *dmtd_status_str(dmtd_status s);
-const char *dmtd_last_error(const dmtd_ctx *ctx);   /* ctx may be NULL: last create error   */
+const char *dmtd_last_error(const dmtd_ctx *ctx);   /* NULL: last error of a call without a context, on this thread */
 
 #ifdef __cplusplus
 }

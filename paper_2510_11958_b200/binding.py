@@ -89,11 +89,14 @@ def load_library():
         "dmtd_set_option": [vp, C.c_char_p, i64],
         "dmtd_get_kv": [vp, i32, C.POINTER(vp), C.POINTER(vp)],
         "dmtd_get_launch_count": [vp, C.POINTER(i64)],
+        "dmtd_attention_decode": [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp, C.c_size_t, vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(d, name)
         fn.argtypes = args
         fn.restype = C.c_int
+    d.dmtd_attention_scratch_bytes.argtypes = [i32, i32, i32, i32, i32]
+    d.dmtd_attention_scratch_bytes.restype = C.c_size_t
     d.dmtd_destroy.argtypes = [vp]
     d.dmtd_destroy.restype = None
     d.dmtd_status_str.argtypes = [C.c_int]
@@ -241,3 +244,32 @@ class Dmtd:
         n = C.c_int64(0)
         self._check(self.dll.dmtd_get_launch_count(self._ctx, C.byref(n)))
         return n.value
+
+
+def _kv_code(t):
+    return {torch.float32: 0, torch.bfloat16: 1}[t.dtype]
+
+
+def attention_decode(q, k, v, pos0, scratch=None):
+    """Split-KV attention of the R new rows of each sequence (dmtd_attention_decode).
+
+    q: cuda float32 [B, R, nq, D]; k, v: cuda [B, nkv, max_seq, D] float32 or bfloat16, with the
+    new rows' K and V already at positions pos0 .. pos0+R-1.  Returns out [B, R, nq, D] float32.
+    `scratch` is a cuda uint8 tensor of at least attention_scratch_bytes(...) bytes; one is
+    allocated through torch if none is given.
+    """
+    dll = load_library()
+    assert q.is_cuda and q.dtype == torch.float32 and q.is_contiguous()
+    assert k.is_cuda and v.is_cuda and k.is_contiguous() and v.is_contiguous() and k.dtype == v.dtype
+    B, R, nq, D = q.shape
+    _, nkv, max_seq, _ = k.shape
+    need = dll.dmtd_attention_scratch_bytes(B, R, nq, D, pos0 + R)
+    if scratch is None:
+        scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    out = torch.empty_like(q)
+    rc = dll.dmtd_attention_decode(_ptr(q), _ptr(k), _ptr(v), _kv_code(k), B, R, nq, nkv, D, max_seq, pos0,
+                                   _ptr(scratch), scratch.numel(), _ptr(out),
+                                   C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    if rc:
+        raise DmtdError(rc, dll.dmtd_last_error(None).decode())
+    return out

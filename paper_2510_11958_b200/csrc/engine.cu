@@ -718,3 +718,90 @@ const char *dmtd_status_str(dmtd_status s) {
 const char *dmtd_last_error(const dmtd_ctx *c) { return c ? c->err.c_str() : g_create_error.c_str(); }
 
 }  // extern "C"
+
+// ---- step a4 as a context-free call ------------------------------------------------------
+
+namespace {
+
+struct AttnPlan { int CH, nsplit; size_t ml_off, o_off, bytes; };
+
+// Scratch layout: [0, 256) the first position as a device int, then the running (max, sum)
+// pairs, then the unnormalised partial outputs, one set per (row, head, key slice).
+AttnPlan attn_plan(int B, int R, int nq, int D, int n_keys) {
+  AttnPlan p{};
+  p.CH = n_keys <= 2048 ? 64 : 256;
+  p.nsplit = std::max(1, (n_keys + p.CH - 1) / p.CH);
+  size_t slots = (size_t)B * R * nq * p.nsplit;
+  p.ml_off = 256;
+  p.o_off = p.ml_off + (slots * 2 * sizeof(float) + 255) / 256 * 256;
+  p.bytes = p.o_off + slots * D * sizeof(float);
+  return p;
+}
+
+dmtd_status attention_check(const float *q, const void *k, const void *v, int kv_dtype, int B, int R, int nq, int nkv,
+                            int D, int max_seq, int pos0, const float *out) {
+  if (!q || !k || !v || !out || B < 1 || R < 1 || pos0 < 0 || max_seq < 1)
+    return fail(nullptr, DMTD_ERR_INVALID_ARG, "attention: null pointer or non-positive size");
+  if (kv_dtype != DMTD_F32 && kv_dtype != DMTD_BF16) return fail(nullptr, DMTD_ERR_SHAPE, "attention: kv_dtype");
+  if (D != 64 && D != 128) return fail(nullptr, DMTD_ERR_SHAPE, "attention: head_dim must be 64 or 128");
+  if (nq < 1 || nkv < 1 || nq % nkv || nq / nkv > ATTN_QR)
+    return fail(nullptr, DMTD_ERR_SHAPE, "attention: n_q_heads must be a multiple of n_kv_heads, at most 16 per kv head");
+  if (pos0 + R > max_seq) return fail(nullptr, DMTD_ERR_CAPACITY, "attention: pos0 + R = %d exceeds max_seq = %d", pos0 + R, max_seq);
+  return DMTD_OK;
+}
+
+template <int D, typename KVT>
+dmtd_status attention_launch_t(const float *q, const void *k, const void *v, int B, int R, int nq, int nkv, int max_seq,
+                               int pos0, unsigned char *scratch, const AttnPlan &p, float *out, cudaStream_t stream) {
+  int *pos_dev = reinterpret_cast<int *>(scratch);
+  float *part_ml = reinterpret_cast<float *>(scratch + p.ml_off);
+  float *part_o = reinterpret_cast<float *>(scratch + p.o_off);
+  const int G = nq / nkv, RB = std::max(1, ATTN_QR / G), n_rb = (R + RB - 1) / RB, ld = nq * D;
+  set_int_kernel<<<1, 1, 0, stream>>>(pos_dev, pos0);
+  size_t smem = (size_t)ATTN_WARPS * ATTN_QR * D * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel<D, KVT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+  if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention: %s", cudaGetErrorString(e));
+  attn_partial_kernel<D, KVT><<<dim3(p.nsplit, nkv * n_rb, B), ATTN_WARPS * 32, smem, stream>>>(
+      q, ld, static_cast<const KVT *>(k), static_cast<const KVT *>(v), max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o,
+      part_ml, p.nsplit);
+  int n_rh = B * R * nq;
+  attn_merge_kernel<D><<<(n_rh + 3) / 4, 128, 0, stream>>>(part_o, part_ml, p.nsplit, n_rh, nq, out, ld);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention: launch failed: %s", cudaGetErrorString(e));
+  return DMTD_OK;
+}
+
+dmtd_status attention_launch(const float *q, const void *k, const void *v, int kv_dtype, int B, int R, int nq, int nkv,
+                             int D, int max_seq, int pos0, unsigned char *scratch, const AttnPlan &p, float *out,
+                             cudaStream_t stream) {
+  bool bf = kv_dtype == DMTD_BF16;
+  if (D == 128)
+    return bf ? attention_launch_t<128, __nv_bfloat16>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream)
+              : attention_launch_t<128, float>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream);
+  return bf ? attention_launch_t<64, __nv_bfloat16>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream)
+            : attention_launch_t<64, float>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t dmtd_attention_scratch_bytes(int32_t B, int32_t R, int32_t nq, int32_t D, int32_t n_keys) {
+  if (B < 1 || R < 1 || nq < 1 || D < 1 || n_keys < 1) return 0;
+  return attn_plan(B, R, nq, D, n_keys).bytes;
+}
+
+dmtd_status dmtd_attention_decode(const float *q, const void *k, const void *v, int32_t kv_dtype, int32_t B, int32_t R,
+                                  int32_t nq, int32_t nkv, int32_t D, int32_t max_seq, int32_t pos0, void *scratch,
+                                  size_t scratch_bytes, float *out, void *cuda_stream) {
+  dmtd_status st = attention_check(q, k, v, kv_dtype, B, R, nq, nkv, D, max_seq, pos0, out);
+  if (st != DMTD_OK) return st;
+  AttnPlan p = attn_plan(B, R, nq, D, pos0 + R);
+  if (!scratch) return fail(nullptr, DMTD_ERR_INVALID_ARG, "attention: null scratch");
+  if (scratch_bytes < p.bytes)
+    return fail(nullptr, DMTD_ERR_CAPACITY, "attention: scratch of %zu bytes is smaller than the %zu needed", scratch_bytes, p.bytes);
+  return attention_launch(q, k, v, kv_dtype, B, R, nq, nkv, D, max_seq, pos0, static_cast<unsigned char *>(scratch), p, out,
+                          static_cast<cudaStream_t>(cuda_stream));
+}
+
+}  // extern "C"

@@ -225,3 +225,25 @@ def test_errors(dmtd):
     rc, n, _ = eng.decode_cycle(3, allow_capacity=True)     # position 8 does not fit max_seq = 8
     assert rc == S["CAPACITY"] and n == 0
     assert eng.device_state() == eng.state()
+
+
+@pytest.mark.parametrize("kvdt,B,R,nq,nkv,D,pos0,max_seq", [
+    ("bf16", 1, 1, 32, 8, 128, 700, 1024),       # one decode row, several key slices, ragged last slice
+    ("bf16", 2, 3, 8, 2, 128, 37, 64),           # a refill chunk: causal among the 3 new rows
+    ("f32", 3, 4, 4, 2, 64, 0, 8),               # no history at all
+    ("bf16", 1, 5, 16, 1, 128, 2300, 2400),      # 16 query heads per KV head, rows split in blocks, long slices
+])
+def test_attention_decode_matches_oracle(dmtd, oracle_lib, kvdt, B, R, nq, nkv, D, pos0, max_seq):
+    """dmtd_attention_decode against the oracle's attention on the same (rounded) K and V."""
+    g = torch.Generator().manual_seed(11)
+    dt = torch.float32 if kvdt == "f32" else torch.bfloat16
+    q = torch.randn(B, R, nq, D, generator=g)
+    k = torch.randn(B, nkv, max_seq, D, generator=g).to(dt)
+    v = torch.randn(B, nkv, max_seq, D, generator=g).to(dt)
+    got = dmtd.attention_decode(q.cuda(), k.cuda(), v.cuda(), pos0)
+    torch.cuda.synchronize()
+    n = pos0 + R
+    for b in range(B):
+        ref = oracle_lib.attention(q[b].double().numpy(), k[b, :, :n].double().permute(1, 0, 2).numpy(),
+                                   v[b, :, :n].double().permute(1, 0, 2).numpy(), pos0)
+        assert np.abs(got[b].double().cpu().numpy() - ref).max() <= 2e-5 * max(1.0, np.abs(ref).max())
