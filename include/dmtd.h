@@ -154,6 +154,28 @@ dmtd_status dmtd_attention_decode(const float *q, const void *k, const void *v, 
                                   int32_t head_dim, int32_t max_seq, int32_t pos0, void *scratch,
                                   size_t scratch_bytes, float *out, void *cuda_stream);
 
+/* dmtd_attention_decode for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, not a step of the method.)  It is
+ * meant for a serving process that has handed every free byte of the GPU to its own memory pool,
+ * so a cudaMalloc for the scratch would fail or fragment that pool, and for a latency-critical
+ * decode loop where cudaMalloc / cudaFree would stall the whole device.  Arguments and results
+ * are those of dmtd_attention_decode, minus the scratch: the per-slice partial results live in a
+ * fixed array of DMTD_ATTENTION_STATIC_SCRATCH_BYTES bytes inside the library's device image
+ * (every GPU that loads the library holds that much until the process exits).  The call makes no
+ * cudaMalloc, cudaFree or other allocating call.
+ *   - A problem whose dmtd_attention_scratch_bytes(...) exceeds that size is rejected with
+ *     CAPACITY and nothing runs.
+ *   - The first call on a device looks up the array's device address (once per device, with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls in the process share the one array.  It keeps the previous call's partials; the
+ *     kernels overwrite every entry they later read, so nothing has to be cleared, but two calls
+ *     whose kernels overlap on the GPU (different streams, different threads) race on it. */
+#define DMTD_ATTENTION_STATIC_SCRATCH_BYTES (4u << 20)
+dmtd_status dmtd_attention_decode_static(const float *q, const void *k, const void *v,
+                                         int32_t kv_dtype, int32_t B, int32_t R, int32_t n_q_heads,
+                                         int32_t n_kv_heads, int32_t head_dim, int32_t max_seq,
+                                         int32_t pos0, float *out, void *cuda_stream);
+
 /* Host-buffer forms of prefill and decode_cycle (same semantics; the copies to and from the
  * device are part of the call, which returns after the stream has drained).
  *   prompt_host [B][P], out_token_host [B], out_tokens_host [B][tau] */

@@ -5,4 +5,4 @@ Python binding (argument marshalling only).  Importing the package does not load
 library; creating a `Dmtd` does, and fails loudly if the library has not been built or no
 CUDA device is present.  There is no CPU fallback.
 """
-from .binding import Dmtd, DmtdError, load_library, library_path, declared_symbols, attention_decode  # noqa: F401
+from .binding import Dmtd, DmtdError, load_library, library_path, declared_symbols, attention_decode, attention_decode_static  # noqa: F401

@@ -90,6 +90,7 @@ def load_library():
         "dmtd_get_kv": [vp, i32, C.POINTER(vp), C.POINTER(vp)],
         "dmtd_get_launch_count": [vp, C.POINTER(i64)],
         "dmtd_attention_decode": [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp, C.c_size_t, vp, vp],
+        "dmtd_attention_decode_static": [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(d, name)
@@ -270,6 +271,30 @@ def attention_decode(q, k, v, pos0, scratch=None):
     rc = dll.dmtd_attention_decode(_ptr(q), _ptr(k), _ptr(v), _kv_code(k), B, R, nq, nkv, D, max_seq, pos0,
                                    _ptr(scratch), scratch.numel(), _ptr(out),
                                    C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    if rc:
+        raise DmtdError(rc, dll.dmtd_last_error(None).decode())
+    return out
+
+
+ATTENTION_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def attention_decode_static(q, k, v, pos0, out):
+    """dmtd_attention_decode_static: the same attention for callers that cannot allocate.
+
+    Nothing is allocated here or in the library: the caller passes `out` (cuda float32, shape of
+    q) and the partial results use the library's built-in array of ATTENTION_STATIC_SCRATCH_BYTES
+    bytes, shared by every call in the process.  Raises DmtdError (CAPACITY) if the problem
+    needs more scratch than that.
+    """
+    dll = load_library()
+    assert q.is_cuda and q.dtype == torch.float32 and q.is_contiguous()
+    assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous() and out.shape == q.shape
+    assert k.is_cuda and v.is_cuda and k.is_contiguous() and v.is_contiguous() and k.dtype == v.dtype
+    B, R, nq, D = q.shape
+    _, nkv, max_seq, _ = k.shape
+    rc = dll.dmtd_attention_decode_static(_ptr(q), _ptr(k), _ptr(v), _kv_code(k), B, R, nq, nkv, D, max_seq, pos0,
+                                          _ptr(out), C.c_void_p(torch.cuda.current_stream().cuda_stream))
     if rc:
         raise DmtdError(rc, dll.dmtd_last_error(None).decode())
     return out

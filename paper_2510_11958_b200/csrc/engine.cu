@@ -8,6 +8,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <numeric>
 #include <string>
 #include <vector>
@@ -805,3 +806,55 @@ dmtd_status dmtd_attention_decode(const float *q, const void *k, const void *v, 
 }
 
 }  // extern "C"
+
+// ---- the same call with its scratch inside the library ------------------------------------
+//
+// For callers that must not allocate: the partial results go to a fixed array in the device
+// image.  In host code the array's name is only a handle; the device address is looked up
+// once per device (with that device current) and passed to the kernels like any pointer.
+
+static __device__ __align__(256) unsigned char g_attention_static_scratch[DMTD_ATTENTION_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+unsigned char *g_static_scratch_addr[kMaxDevices] = {};
+std::mutex g_static_scratch_mu;
+
+// Device address of the fixed scratch on the current device.
+dmtd_status static_scratch_address(unsigned char **out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention_static: cudaGetDevice: %s", cudaGetErrorString(e));
+  if (dev < 0 || dev >= kMaxDevices) return fail(nullptr, DMTD_ERR_UNSUPPORTED, "attention_static: device index %d", dev);
+  std::lock_guard<std::mutex> lock(g_static_scratch_mu);
+  if (!g_static_scratch_addr[dev]) {
+    void *p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_attention_static_scratch);
+    if (e != cudaSuccess || !p)
+      return fail(nullptr, DMTD_ERR_CUDA, "attention_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+    g_static_scratch_addr[dev] = static_cast<unsigned char *>(p);
+  }
+  *out = g_static_scratch_addr[dev];
+  return DMTD_OK;
+}
+
+}  // namespace
+
+extern "C" dmtd_status dmtd_attention_decode_static(const float *q, const void *k, const void *v, int32_t kv_dtype,
+                                                    int32_t B, int32_t R, int32_t nq, int32_t nkv, int32_t D,
+                                                    int32_t max_seq, int32_t pos0, float *out, void *cuda_stream) {
+  dmtd_status st = attention_check(q, k, v, kv_dtype, B, R, nq, nkv, D, max_seq, pos0, out);
+  if (st != DMTD_OK) return st;
+  AttnPlan p = attn_plan(B, R, nq, D, pos0 + R);
+  if (p.bytes > (size_t)DMTD_ATTENTION_STATIC_SCRATCH_BYTES)
+    return fail(nullptr, DMTD_ERR_CAPACITY,
+                "attention_static: this problem needs %zu bytes of scratch, the built-in array holds %zu; "
+                "use dmtd_attention_decode with caller-owned scratch", p.bytes, (size_t)DMTD_ATTENTION_STATIC_SCRATCH_BYTES);
+  unsigned char *scratch = nullptr;
+  st = static_scratch_address(&scratch);
+  if (st != DMTD_OK) return st;
+  // nothing to clear: every (row, head, slice) entry the merge reads is written by this call
+  return attention_launch(q, k, v, kv_dtype, B, R, nq, nkv, D, max_seq, pos0, scratch, p, out,
+                          static_cast<cudaStream_t>(cuda_stream));
+}
