@@ -197,6 +197,9 @@ dmtd_status dmtd_set_tau(dmtd_ctx *ctx, int32_t tau);
  *   "cuda_graph"   0/1  replay captured CUDA graphs for whole passes (default 1)
  *   "literal_sum"  0/1  upper-layer input of a full pass = embedding + lower-stack output, the
  *                       literal sum of Eq. 4, instead of the lower-stack output alone (default 0)
+ *   "fused_pass"   0/1  run each decode pass as one persistent kernel where the model and batch
+ *                       allow it (bf16 weights and KV, head_dim 128, at most 4 rows per pass);
+ *                       0 = always the per-step kernels (default 1)
  * Errors: INVALID_ARG for an unknown name or value. */
 dmtd_status dmtd_set_option(dmtd_ctx *ctx, const char *name, int64_t value);
 

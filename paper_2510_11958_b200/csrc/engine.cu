@@ -15,6 +15,7 @@
 
 #include "../../include/dmtd.h"
 #include "kernels.cuh"
+#include "pass_kernel.cuh"
 
 using namespace dmtd;
 
@@ -60,7 +61,14 @@ struct dmtd_ctx {
   float2 *rope_tab = nullptr;
 
   // options
-  bool use_graph = true, literal_sum = false;
+  bool use_graph = true, literal_sum = false, use_fused = true;
+
+  // fused pass kernel: one persistent launch per pass
+  bool fused_ok = false;
+  PassLayer *pass_layers = nullptr;         // device [n_layers]
+  float *f_part_o = nullptr, *f_part_ml = nullptr, *amax_val = nullptr;
+  int *amax_idx = nullptr;
+  unsigned int *grid_bar = nullptr;
 
   // graphs: [kind 1 = full, 2 = upper-only]
   cudaGraphExec_t graph_exec[3] = {nullptr, nullptr, nullptr};
@@ -304,12 +312,104 @@ dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, floa
   return DMTD_OK;
 }
 
+// ---------------------------------------------------------------------------- fused pass
+
+// Can the block-per-SM pass kernel stream this matrix?  Its k-slab must fit the staging area
+// and one block's share must not reach over more than two slabs.
+bool fused_matrix_ok(const PackedMat &m, int grid) {
+  if (!m.w) return false;
+  long long slab_atoms = (long long)m.n_tiles * m.aps, per_block = (packed_atoms(m) + grid - 1) / grid;
+  return m.aps * 32 <= PK_MAX_KS && per_block <= slab_atoms;
+}
+
+// Set up what the fused pass kernel needs; leaves fused_ok false when the model or the device
+// does not fit it (the per-step kernels then run every pass).
+dmtd_status setup_fused(dmtd_ctx *c) {
+  const dmtd_model_shape &s = c->s;
+  c->fused_ok = false;
+  if (!is_bf16(c) || s.kv_dtype != DMTD_BF16 || s.head_dim != PK_D || s.n_layers > PK_MAX_LAYERS) return DMTD_OK;
+  if (s.n_q_heads / s.n_kv_heads > PK_QR || s.hidden % 8) return DMTD_OK;
+  int coop = 0;
+  CUDA_TRY(c, cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
+  if (!coop) return DMTD_OK;
+  if (cudaFuncSetAttribute(dmtd_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PK_SMEM_BYTES) != cudaSuccess) {
+    cudaGetLastError();
+    return DMTD_OK;
+  }
+  int per_sm = 0;
+  CUDA_TRY(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dmtd_pass_kernel, PK_THREADS, PK_SMEM_BYTES));
+  if (per_sm < 1) return DMTD_OK;
+  if (!fused_matrix_ok(c->embed, c->n_sms)) return DMTD_OK;
+  for (const LayerDev &ld : c->layers) {
+    if (!fused_matrix_ok(ld.qkv, c->n_sms) || !fused_matrix_ok(ld.o, c->n_sms) || !fused_matrix_ok(ld.gu, c->n_sms) ||
+        !fused_matrix_ok(ld.down, c->n_sms))
+      return DMTD_OK;
+    int KS_o = ld.o.aps * 32;
+    if (KS_o % PK_D || 2 * KS_o / PK_D > PK_MERGE_HEADS) return DMTD_OK;
+  }
+  std::vector<PassLayer> h(s.n_layers);
+  for (int l = 0; l < s.n_layers; ++l) {
+    const LayerDev &ld = c->layers[l];
+    h[l].qkv = ld.qkv; h[l].o = ld.o; h[l].gu = ld.gu; h[l].down = ld.down;
+    h[l].w_in = ld.w_in; h[l].w_post = ld.w_post; h[l].w_qn = ld.w_qn; h[l].w_kn = ld.w_kn;
+    h[l].kc = static_cast<__nv_bfloat16 *>(c->kc) + (size_t)l * c->kv_layer_elems;
+    h[l].vc = static_cast<__nv_bfloat16 *>(c->vc) + (size_t)l * c->kv_layer_elems;
+  }
+  TRY(dev_alloc(c, &c->pass_layers, h.size()));
+  CUDA_TRY(c, cudaMemcpyAsync(c->pass_layers, h.data(), h.size() * sizeof(PassLayer), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  size_t slots = (size_t)PK_MAX_ROWS * s.n_q_heads * PK_NSPLIT_CAP;
+  TRY(dev_alloc(c, &c->f_part_o, slots * PK_D));
+  TRY(dev_alloc(c, &c->f_part_ml, slots * 2));
+  TRY(dev_alloc(c, &c->amax_val, (size_t)PK_MAX_ROWS * c->n_sms));
+  TRY(dev_alloc(c, &c->amax_idx, (size_t)PK_MAX_ROWS * c->n_sms));
+  TRY(dev_alloc(c, &c->grid_bar, 1));
+  c->fused_ok = true;
+  return DMTD_OK;
+}
+
+bool fused_pass_ok(const dmtd_ctx *c, int kind, int R_lower) {
+  if (!c->fused_ok || !c->use_fused) return false;
+  const int lo = c->s.n_layers - c->L_d;
+  const int R = (kind == 1 && lo > 0) ? R_lower : 1;
+  return c->B * R <= PK_MAX_ROWS && R * (c->s.n_q_heads / c->s.n_kv_heads) <= PK_QR;
+}
+
+// One pass (Section 2.2) as a single cooperative launch of the persistent pass kernel.
+dmtd_status enqueue_pass_fused(dmtd_ctx *c, int kind, int R_lower, bool write_token, int *out_argmax, float *out_logits) {
+  const dmtd_model_shape &s = c->s;
+  const int L = s.n_layers, lo = L - c->L_d;
+  PassParams P{};
+  P.layers = c->pass_layers; P.embed = c->embed; P.w_final = c->w_final; P.inv_freq = c->inv_freq;
+  P.l_begin = (kind == 1 && lo > 0) ? 0 : lo; P.l_split = lo; P.l_end = L;
+  P.R_lo = (kind == 1 && lo > 0) ? R_lower : 1; P.B = c->B;
+  P.H = s.hidden; P.I = s.intermediate; P.nq = s.n_q_heads; P.nkv = s.n_kv_heads; P.vocab = s.vocab;
+  P.max_seq = c->max_seq; P.ldl = c->ldl; P.eps = s.rms_eps;
+  P.kind = kind; P.write_token = write_token ? 1 : 0; P.literal_sum = c->literal_sum ? 1 : 0;
+  P.tokens = c->tokens; P.st = c->dstate;
+  P.x_lo = c->x_lo; P.x_up = c->x_up; P.qkv = c->qkv; P.gu = c->gu; P.logits = c->logits;
+  P.part_o = c->f_part_o; P.part_ml = c->f_part_ml; P.amax_val = c->amax_val; P.amax_idx = c->amax_idx;
+  P.out_argmax = out_argmax; P.barrier = c->grid_bar; P.error = &c->dstate->error;
+  P.wait_limit = 2000000000ll;              // about a second of SM clock
+  CUDA_TRY(c, cudaMemsetAsync(c->grid_bar, 0, sizeof(unsigned int), c->stream));
+  void *args[] = {&P};
+  CUDA_TRY(c, cudaLaunchCooperativeKernel((const void *)dmtd_pass_kernel, dim3(c->n_sms), dim3(PK_THREADS), args,
+                                          (size_t)PK_SMEM_BYTES, c->stream));
+  c->launches += 1;
+  if (out_logits)
+    CUDA_TRY(c, cudaMemcpy2DAsync(out_logits, (size_t)s.vocab * 4, c->logits, (size_t)c->ldl * 4, (size_t)s.vocab * 4, c->B,
+                                  cudaMemcpyDeviceToDevice, c->stream));
+  return DMTD_OK;
+}
+
 // One pass of the decode stage (Section 2.2).  kind 1: full pass - the R = n_known - lo_len
 // pending rows through the lower layers (refill), the newest row through the decoding
 // layers.  kind 2: the newest token's embedding through the decoding layers only.
 dmtd_status enqueue_pass(dmtd_ctx *c, int kind, int R_lower, bool write_token, int *out_argmax, float *out_logits) {
   const int B = c->B, L = c->s.n_layers, lo = L - c->L_d, H = c->s.hidden;
   const int newest = c->h.n_known - 1;
+  if (!c->capturing && fused_pass_ok(c, kind, R_lower))
+    return enqueue_pass_fused(c, kind, R_lower, write_token, out_argmax, out_logits);
   if (kind == 1 && lo > 0) {
     TRY(launch_embed(c, &c->dstate->lo_len, B, R_lower, c->x_lo, false));
     TRY(launch_rope_table(c, &c->dstate->lo_len, R_lower));
@@ -373,7 +473,9 @@ dmtd_status run_greedy_pass(dmtd_ctx *c) {
   int kind = c->h.slot == 0 ? 1 : 2;
   int R_lower = c->h.n_known - c->h.lo_len;
   bool steady = (kind == 2) || (R_lower == c->tau);
-  if (c->use_graph && steady) {
+  if (fused_pass_ok(c, kind, R_lower)) {
+    TRY(enqueue_pass_fused(c, kind, R_lower, true, nullptr, nullptr));
+  } else if (c->use_graph && steady) {
     if (c->graph_B != c->B || c->graph_tau != c->tau) { drop_graphs(c); c->graph_B = c->B; c->graph_tau = c->tau; }
     if (!c->graph_exec[kind]) TRY(capture_pass(c, kind));
     CUDA_TRY(c, cudaGraphLaunch(c->graph_exec[kind], c->stream));
@@ -495,6 +597,7 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   CTRY(dev_alloc(c, &c->part_o, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * D));
   CTRY(dev_alloc(c, &c->part_ml, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * 2));
   CTRY(dev_alloc(c, &c->rope_tab, (size_t)c->ws_rows * (D / 2)));
+  CTRY(setup_fused(c));
   CTRY(dmtd_reset(c));
   CCUDA(cudaStreamSynchronize(c->stream));   // repacking done: the caller may free its weights
 #undef CTRY
@@ -663,7 +766,8 @@ dmtd_status dmtd_get_device_state(dmtd_ctx *c, dmtd_state *out) {
   DevState d{};
   CUDA_TRY(c, cudaMemcpyAsync(&d, c->dstate, sizeof d, cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
-  if (d.error) return fail(c, DMTD_ERR_INVALID_ARG, "a token id outside [0, vocab) reached the embedding gather");
+  if (d.error == PK_ERR_TOKEN) return fail(c, DMTD_ERR_INVALID_ARG, "a token id outside [0, vocab) reached the embedding gather");
+  if (d.error) return fail(c, DMTD_ERR_TIMEOUT, "a device-side wait of the pass kernel gave up (%s)", d.error == PK_ERR_COPY_WAIT ? "weight copy" : "grid barrier");
   out->n_known = d.n_known; out->lo_len = d.lo_len; out->up_len = d.up_len; out->cycle = d.cycle;
   out->slot = d.slot; out->n_emitted = d.n_emitted; out->tau = d.tau; out->L_d = c->L_d;
   return DMTD_OK;
@@ -685,6 +789,7 @@ dmtd_status dmtd_set_option(dmtd_ctx *c, const char *name, int64_t value) {
   if (value != 0 && value != 1) return fail(c, DMTD_ERR_INVALID_ARG, "option %s takes 0 or 1", name);
   if (!strcmp(name, "cuda_graph")) { c->use_graph = value != 0; return DMTD_OK; }
   if (!strcmp(name, "literal_sum")) { c->literal_sum = value != 0; drop_graphs(c); return DMTD_OK; }
+  if (!strcmp(name, "fused_pass")) { c->use_fused = value != 0; return DMTD_OK; }
   return fail(c, DMTD_ERR_INVALID_ARG, "unknown option %s", name);
 }
 
