@@ -10,7 +10,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libdmtd_b200.so")
 SOURCES = ["engine.cu"]
-HEADERS = ["common.cuh", "kernels.cuh", "pass_kernel.cuh"]
+HEADERS = ["common.cuh", "kernels.cuh", "pass_common.cuh", "pass_stream.cuh", "pass_prologues.cuh",
+           "pass_attention.cuh", "pass_kernel.cuh"]
 
 
 def _stale() -> bool:

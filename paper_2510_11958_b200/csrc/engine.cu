@@ -69,6 +69,8 @@ struct dmtd_ctx {
   float *f_part_o = nullptr, *f_part_ml = nullptr, *amax_val = nullptr;
   int *amax_idx = nullptr;
   unsigned int *grid_bar = nullptr;
+  int *attn_count = nullptr;
+  long long *pass_timing = nullptr;         // profiling builds only
 
   // graphs: [kind 1 = full, 2 = upper-only]
   cudaGraphExec_t graph_exec[3] = {nullptr, nullptr, nullptr};
@@ -319,7 +321,8 @@ dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, floa
 bool fused_matrix_ok(const PackedMat &m, int grid) {
   if (!m.w) return false;
   long long slab_atoms = (long long)m.n_tiles * m.aps, per_block = (packed_atoms(m) + grid - 1) / grid;
-  return m.aps * 32 <= PK_MAX_KS && per_block <= slab_atoms;
+  // 32-bit stream arithmetic in the kernel: atoms * blocks must fit
+  return m.aps * 32 <= PK_MAX_KS && per_block <= slab_atoms && packed_atoms(m) * (grid + 1) < (1ll << 31);
 }
 
 // Set up what the fused pass kernel needs; leaves fused_ok false when the model or the device
@@ -328,7 +331,8 @@ dmtd_status setup_fused(dmtd_ctx *c) {
   const dmtd_model_shape &s = c->s;
   c->fused_ok = false;
   if (!is_bf16(c) || s.kv_dtype != DMTD_BF16 || s.head_dim != PK_D || s.n_layers > PK_MAX_LAYERS) return DMTD_OK;
-  if (s.n_q_heads / s.n_kv_heads > PK_QR || s.hidden % 8) return DMTD_OK;
+  if (s.n_q_heads / s.n_kv_heads > PK_QR || s.hidden % 8 || s.hidden > PK_XS_FLOATS) return DMTD_OK;
+  if (c->max_batch * s.n_kv_heads > PK_THREADS) return DMTD_OK;
   int coop = 0;
   CUDA_TRY(c, cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
   if (!coop) return DMTD_OK;
@@ -344,8 +348,6 @@ dmtd_status setup_fused(dmtd_ctx *c) {
     if (!fused_matrix_ok(ld.qkv, c->n_sms) || !fused_matrix_ok(ld.o, c->n_sms) || !fused_matrix_ok(ld.gu, c->n_sms) ||
         !fused_matrix_ok(ld.down, c->n_sms))
       return DMTD_OK;
-    int KS_o = ld.o.aps * 32;
-    if (KS_o % PK_D || 2 * KS_o / PK_D > PK_MERGE_HEADS) return DMTD_OK;
   }
   std::vector<PassLayer> h(s.n_layers);
   for (int l = 0; l < s.n_layers; ++l) {
@@ -364,15 +366,20 @@ dmtd_status setup_fused(dmtd_ctx *c) {
   TRY(dev_alloc(c, &c->amax_val, (size_t)PK_MAX_ROWS * c->n_sms));
   TRY(dev_alloc(c, &c->amax_idx, (size_t)PK_MAX_ROWS * c->n_sms));
   TRY(dev_alloc(c, &c->grid_bar, 1));
+  TRY(dev_alloc(c, &c->attn_count, (size_t)c->max_batch * s.n_kv_heads));
+#ifdef DMTD_PASS_TIMING
+  TRY(dev_alloc(c, &c->pass_timing, (size_t)2 * PK_TIMING_SLOTS));
+#endif
   c->fused_ok = true;
   return DMTD_OK;
 }
 
 bool fused_pass_ok(const dmtd_ctx *c, int kind, int R_lower) {
-  if (!c->fused_ok || !c->use_fused) return false;
+  if (!c->fused_ok || !c->use_fused || c->literal_sum) return false;
   const int lo = c->s.n_layers - c->L_d;
   const int R = (kind == 1 && lo > 0) ? R_lower : 1;
-  return c->B * R <= PK_MAX_ROWS && R * (c->s.n_q_heads / c->s.n_kv_heads) <= PK_QR;
+  return c->B * R <= PK_MAX_ROWS && R * (c->s.n_q_heads / c->s.n_kv_heads) <= PK_QR &&
+         c->B * R * c->s.hidden <= PK_XS_FLOATS;
 }
 
 // One pass (Section 2.2) as a single cooperative launch of the persistent pass kernel.
@@ -385,9 +392,10 @@ dmtd_status enqueue_pass_fused(dmtd_ctx *c, int kind, int R_lower, bool write_to
   P.R_lo = (kind == 1 && lo > 0) ? R_lower : 1; P.B = c->B;
   P.H = s.hidden; P.I = s.intermediate; P.nq = s.n_q_heads; P.nkv = s.n_kv_heads; P.vocab = s.vocab;
   P.max_seq = c->max_seq; P.ldl = c->ldl; P.eps = s.rms_eps;
-  P.kind = kind; P.write_token = write_token ? 1 : 0; P.literal_sum = c->literal_sum ? 1 : 0;
+  P.kind = kind; P.write_token = write_token ? 1 : 0;
   P.tokens = c->tokens; P.st = c->dstate;
   P.x_lo = c->x_lo; P.x_up = c->x_up; P.qkv = c->qkv; P.gu = c->gu; P.logits = c->logits;
+  P.attn_out = c->act; P.lda = c->lda; P.attn_count = c->attn_count; P.timing = c->pass_timing;
   P.part_o = c->f_part_o; P.part_ml = c->f_part_ml; P.amax_val = c->amax_val; P.amax_idx = c->amax_idx;
   P.out_argmax = out_argmax; P.barrier = c->grid_bar; P.error = &c->dstate->error;
   P.wait_limit = 2000000000ll;              // about a second of SM clock
@@ -963,3 +971,12 @@ extern "C" dmtd_status dmtd_attention_decode_static(const float *q, const void *
   return attention_launch(q, k, v, kv_dtype, B, R, nq, nkv, D, max_seq, pos0, scratch, p, out,
                           static_cast<cudaStream_t>(cuda_stream));
 }
+
+#ifdef DMTD_PASS_TIMING
+// Profiling builds: copy out the stage time stamps of the last pass (2 x PK_TIMING_SLOTS ticks).
+extern "C" int dmtd_debug_pass_timing(dmtd_ctx *c, long long *host_out) {
+  if (!c || !c->pass_timing) return -1;
+  cudaStreamSynchronize(c->stream);
+  return (int)cudaMemcpy(host_out, c->pass_timing, sizeof(long long) * 2 * PK_TIMING_SLOTS, cudaMemcpyDeviceToHost);
+}
+#endif

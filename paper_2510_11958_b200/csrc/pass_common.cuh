@@ -1,0 +1,157 @@
+// Shared definitions of the persistent pass kernel: sizes, parameters, PTX wrappers, the
+// shared-memory map, the per-warp weight stream and the grid barrier.
+//
+// Lessons the layout encodes (measured on B200):
+//  * every stage runs once per layer and the stages of a layer are different code, so the code
+//    of one layer must stay resident in the instruction cache: stage functions are separate,
+//    small, and loop instead of unrolling;
+//  * any load that crosses the chip costs a microsecond or more while the weight stream is
+//    running, so a stage issues all of its loads before it uses any, and nothing in the weight
+//    loop touches local or global memory;
+//  * more bulk copies in flight than bandwidth x latency only lengthen every other round trip.
+#pragma once
+
+#include "common.cuh"
+
+namespace dmtd {
+
+constexpr int PK_WARPS = 8;
+constexpr int PK_THREADS = PK_WARPS * 32;
+constexpr int PK_CHUNK_ATOMS = 4;                          // atoms (1 KiB each) per bulk copy
+constexpr int PK_CHUNK_BYTES = PK_CHUNK_ATOMS * 1024;
+constexpr int PK_SLOTS = 4;                                // ring slots per warp
+constexpr int PK_MAX_ROWS = 4;                             // activation rows (B*R) per stage
+constexpr int PK_MAX_KS = 1280;                            // largest k-slab of a packed matrix
+constexpr int PK_MAX_LAYERS = 40;
+constexpr int PK_NSPLIT_CAP = 32;                          // key slices per (sequence, kv head)
+constexpr int PK_D = 128;                                  // head_dim
+constexpr int PK_QR = 16;                                  // query rows per attention item
+constexpr int PK_XS_FLOATS = 10240;                        // row staging: B*R*hidden floats at most
+
+// shared memory map (bytes)
+constexpr int PK_RING_BYTES = PK_WARPS * PK_SLOTS * PK_CHUNK_BYTES;           // 131072
+constexpr int PK_BROW_MAX = PK_MAX_KS * 2 + 64;                               // 2624
+constexpr int PK_BSTAGE_BYTES = 2 * 8 * PK_BROW_MAX;                          // 41984: two slabs of 8 columns
+constexpr int PK_XS_BYTES = PK_XS_FLOATS * 4;                                 // 40960
+constexpr int PK_OFF_RING = 0;
+constexpr int PK_OFF_BSTAGE = PK_OFF_RING + PK_RING_BYTES;
+constexpr int PK_OFF_XS = PK_OFF_BSTAGE + PK_BSTAGE_BYTES;                    // directly behind bstage
+constexpr int PK_OFF_BARS = PK_OFF_XS + PK_XS_BYTES;
+constexpr int PK_OFF_SMALL = PK_OFF_BARS + PK_WARPS * PK_SLOTS * 8;
+constexpr int PK_SMALL_BYTES = 1024;
+constexpr int PK_OFF_LAYERS = PK_OFF_SMALL + PK_SMALL_BYTES;
+
+enum { PK_ERR_NONE = 0, PK_ERR_TOKEN = 1, PK_ERR_COPY_WAIT = 2, PK_ERR_BARRIER_WAIT = 3 };
+
+struct PassLayer {
+  PackedMat qkv, o, gu, down;
+  const float *w_in, *w_post, *w_qn, *w_kn;
+  __nv_bfloat16 *kc, *vc;                 // this layer's cache [sequence][kv head][max_seq][128]
+};
+
+struct PassParams {
+  const PassLayer *layers;                // device array, all layers of the model
+  PackedMat embed;
+  const float *w_final;
+  const double *inv_freq;
+  int l_begin, l_split, l_end;            // layers [l_begin, l_split): R_lo rows at lo_len..; [l_split, l_end): newest row
+  int R_lo, B;
+  int H, I, nq, nkv, vocab, max_seq, ldl;
+  float eps;
+  int kind;                               // 1 full pass, 2 decoding layers only (counter update)
+  int write_token;
+  int *tokens;
+  DevState *st;
+  float *x_lo, *x_up, *qkv, *gu, *logits, *part_o, *part_ml;
+  float *attn_out;                        // merged attention output [row][lda]
+  int lda;
+  int *attn_count;                        // finished key slices per (sequence, kv head)
+  float *amax_val;
+  int *amax_idx;
+  int *out_argmax;
+  unsigned int *barrier;                  // zero at launch
+  int *error;                             // sticky, 0 = fine
+  long long wait_limit;                   // clock ticks a device-side wait may take
+  long long *timing;                      // stage time stamps (profiling builds), or NULL
+};
+
+constexpr int PK_SMEM_BYTES = PK_OFF_LAYERS + PK_MAX_LAYERS * (int)sizeof(PassLayer);
+static_assert(PK_SMEM_BYTES <= 227 * 1024, "shared memory map too large");
+
+// ---------------------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// global -> this block's shared memory, completion counted in bytes on an mbarrier
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_add(unsigned *p, unsigned v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void pk_sync() { __syncthreads(); }
+
+// ---------------------------------------------------------------------------- block state
+
+struct WarpPipe;
+
+struct PassShared {
+  unsigned char *ring;      // [warp][slot][PK_CHUNK_BYTES]
+  unsigned char *bstage;    // activation columns of up to two k-slabs; attention scratch (with xs)
+  float *xs;                // staged activation rows
+  uint64_t *bars;           // [warp][slot]
+  volatile int *abort_flag;
+  float *red;               // [PK_WARPS][PK_MAX_ROWS]
+  WarpPipe *pipes;          // [PK_WARPS] ring state of every warp between stages
+  PassLayer *layers;        // layers [l_begin, l_end) of this pass
+};
+
+extern __shared__ __align__(1024) unsigned char pk_smem[];
+
+// The block's shared memory map: constant offsets, so building it costs nothing.
+__device__ __forceinline__ PassShared pass_shared() {
+  PassShared S;
+  S.ring = pk_smem + PK_OFF_RING;
+  S.bstage = pk_smem + PK_OFF_BSTAGE;
+  S.xs = reinterpret_cast<float *>(pk_smem + PK_OFF_XS);
+  S.bars = reinterpret_cast<uint64_t *>(pk_smem + PK_OFF_BARS);
+  S.abort_flag = reinterpret_cast<volatile int *>(pk_smem + PK_OFF_SMALL);
+  S.red = reinterpret_cast<float *>(pk_smem + PK_OFF_SMALL + 64);
+  S.pipes = reinterpret_cast<WarpPipe *>(pk_smem + PK_OFF_SMALL + 256);
+  S.layers = reinterpret_cast<PassLayer *>(pk_smem + PK_OFF_LAYERS);
+  return S;
+}
+
+}  // namespace dmtd

@@ -1,0 +1,187 @@
+// The per-warp weight stream of the pass kernel, the grid barrier, and small load/store helpers.
+#pragma once
+
+#include "pass_common.cuh"
+
+namespace dmtd {
+
+// Position in one warp's weight stream: its share of every matrix of the pass, in pass order.
+// Atom counts are 32-bit: the host checks atoms * blocks < 2^31 for every matrix.
+struct StreamCursor {
+  int mat, n_mats, warp;
+  int pos, end;
+  const uint4 *base;
+};
+
+// A warp's ring: lane 0 runs the producer cursor; all lanes agree on `consumed`.  Lives in
+// shared memory between stages and in registers inside a projection.
+struct WarpPipe {
+  uint32_t ring, bars;      // shared addresses of this warp's slots and barriers
+  unsigned issued, consumed;
+  StreamCursor cur;
+};
+static_assert(sizeof(WarpPipe) * PK_WARPS <= PK_SMALL_BYTES - 256, "pipe state does not fit");
+
+__device__ __forceinline__ const PackedMat &pass_matrix(const PassParams &P, const PassShared &S, int q) {
+  int n_layer_mats = 4 * (P.l_end - P.l_begin);
+  if (q >= n_layer_mats) return P.embed;
+  const PassLayer &L = S.layers[q >> 2];
+  switch (q & 3) {
+    case 0: return L.qkv;
+    case 1: return L.o;
+    case 2: return L.gu;
+    default: return L.down;
+  }
+}
+
+// Atoms [c0, c1) of the block and [w0, w1) of the warp: equal contiguous cuts of the stream.
+__device__ __forceinline__ void stream_ranges(const PackedMat &W, int warp, int &c0, int &c1, int &w0, int &w1) {
+  const unsigned A = (unsigned)(W.n_slabs * W.n_tiles * W.aps);
+  c0 = (int)(A * blockIdx.x / gridDim.x);
+  c1 = (int)(A * (blockIdx.x + 1) / gridDim.x);
+  w0 = c0 + (c1 - c0) * warp / PK_WARPS;
+  w1 = c0 + (c1 - c0) * (warp + 1) / PK_WARPS;
+}
+
+__device__ __forceinline__ void cursor_init(StreamCursor &c, const PassParams &P, int warp) {
+  c.mat = -1; c.n_mats = 4 * (P.l_end - P.l_begin) + 1; c.warp = warp;
+  c.pos = c.end = 0; c.base = nullptr;
+}
+
+// Move the cursor to the warp's share of the next matrix that has one (once per matrix).
+__device__ __noinline__ bool cursor_next_matrix(StreamCursor &c, const PassParams &P) {
+  const PassShared S = pass_shared();
+  while (c.pos >= c.end) {
+    if (++c.mat >= c.n_mats) { c.mat = c.n_mats; return false; }
+    const PackedMat &W = pass_matrix(P, S, c.mat);
+    int c0, c1, w0, w1;
+    stream_ranges(W, c.warp, c0, c1, w0, w1);
+    c.pos = w0; c.end = w1; c.base = W.w;
+  }
+  return true;
+}
+
+// Lane 0: issue the next chunk of the warp's stream, if any is left in the pass.
+__device__ __forceinline__ void pipe_issue(const PassParams &P, WarpPipe &pp) {
+  if (pp.cur.pos >= pp.cur.end && !cursor_next_matrix(pp.cur, P)) return;
+  const int n = min(PK_CHUNK_ATOMS, pp.cur.end - pp.cur.pos);
+  const unsigned slot = pp.issued % PK_SLOTS;
+  const uint32_t bar = pp.bars + slot * 8;
+  mbar_expect_tx(bar, (uint32_t)n * 1024u);
+  bulk_g2s(pp.ring + slot * PK_CHUNK_BYTES, pp.cur.base + (size_t)pp.cur.pos * 64, (uint32_t)n * 1024u, bar);
+  pp.cur.pos += n;
+  pp.issued += 1;
+}
+
+__device__ __noinline__ bool pipe_wait_slow(const PassParams &P, uint32_t bar, uint32_t parity) {
+  const PassShared S = pass_shared();
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > P.wait_limit || *S.abort_flag) {
+      *S.abort_flag = 1;
+      atomicMax(P.error, PK_ERR_COPY_WAIT);
+      return false;
+    }
+  }
+  return true;
+}
+
+// All lanes: wait until chunk `consumed` has landed.  Bounded; false = gave up.
+__device__ __forceinline__ bool pipe_wait(const PassParams &P, const WarpPipe &pp) {
+  const unsigned slot = pp.consumed % PK_SLOTS;
+  const uint32_t parity = (pp.consumed / PK_SLOTS) & 1u;
+  const uint32_t bar = pp.bars + slot * 8;
+  if (mbar_try_wait(bar, parity)) return true;
+  return pipe_wait_slow(P, bar, parity);
+}
+
+// Grid-wide barrier: every block arrives once per stage; `target` counts arrivals so far.
+__device__ __noinline__ bool grid_barrier(const PassParams &P, unsigned &target) {
+  const PassShared S = pass_shared();
+  pk_sync();
+  if (threadIdx.x == 0) {
+    target += gridDim.x;
+    if (*S.abort_flag) {
+      atomicMax(P.error, PK_ERR_BARRIER_WAIT);
+    } else {
+      red_release_add(P.barrier, 1u);
+      const long long t0 = clock64();
+      unsigned spins = 0;
+      while (ld_acquire_u32(P.barrier) < target) {
+        if ((++spins & 63u) == 0u &&
+            (clock64() - t0 > P.wait_limit || *reinterpret_cast<volatile int *>(P.error) > PK_ERR_TOKEN)) {
+          atomicMax(P.error, PK_ERR_BARRIER_WAIT);
+          *S.abort_flag = 1;
+          break;
+        }
+      }
+    }
+  }
+  pk_sync();
+  return *S.abort_flag == 0;
+}
+
+// ---------------------------------------------------------------------------- small helpers
+
+__device__ __forceinline__ void unpack8(uint4 v, float (&f)[8]) {
+  uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    f[2 * j] = bf16_bits_to_float(w[j] & 0xffffu);
+    f[2 * j + 1] = bf16_bits_to_float(w[j] >> 16);
+  }
+}
+
+// Values k = 8u .. 8u+7 of row `tok` of the packed embedding matrix.
+__device__ __forceinline__ void embed8(const PackedMat &E, int tok, int u, float (&f)[8]) {
+  const int k = u * 8, atom = k >> 5, t = (k >> 3) & 3;
+  const int s = atom / E.aps, a = atom % E.aps;
+  const int T = tok >> 4, half = (tok >> 3) & 1, g = tok & 7;
+  unpack8(__ldg(E.w + (((long long)s * E.n_tiles + T) * E.aps + a) * 64 + half * 32 + g * 4 + t), f);
+}
+
+__device__ __forceinline__ int b_row_bytes(int KS) { return ((KS * 2) % 128 == 64) ? KS * 2 : KS * 2 + 64; }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Write 4 activation values (k_local .. k_local+3 of a slab) of row m as the hi and lo bf16
+// columns: x = hi + lo with |error| <= 2^-17 |x|.
+__device__ __forceinline__ void store_act4(unsigned char *slab_base, int row_bytes, int m, int k_local, float4 v) {
+  const uint32_t h0 = pack_bf16x2(v.x, v.y), h1 = pack_bf16x2(v.z, v.w);
+  const float r0 = v.x - __uint_as_float(h0 << 16), r1 = v.y - __uint_as_float(h0 & 0xffff0000u);
+  const float r2 = v.z - __uint_as_float(h1 << 16), r3 = v.w - __uint_as_float(h1 & 0xffff0000u);
+  *reinterpret_cast<uint2 *>(slab_base + (size_t)(2 * m) * row_bytes + k_local * 2) = make_uint2(h0, h1);
+  *reinterpret_cast<uint2 *>(slab_base + (size_t)(2 * m + 1) * row_bytes + k_local * 2) =
+      make_uint2(pack_bf16x2(r0, r1), pack_bf16x2(r2, r3));
+}
+
+// Which k-slabs this block's share of W touches.
+struct SlabSpan { int first, count, KS, row_bytes; };
+__device__ __forceinline__ SlabSpan slab_span(const PackedMat &W) {
+  int c0, c1, w0, w1;
+  stream_ranges(W, 0, c0, c1, w0, w1);
+  SlabSpan sp;
+  sp.KS = W.aps * 32;
+  sp.row_bytes = b_row_bytes(sp.KS);
+  const int slab_atoms = W.n_tiles * W.aps;
+  if (c0 >= c1) { sp.first = 0; sp.count = 0; return sp; }
+  sp.first = c0 / slab_atoms;
+  sp.count = (c1 - 1) / slab_atoms - sp.first + 1;
+  return sp;
+}
+
+// Clear `n` floats, the work spread over the grid.
+__device__ __forceinline__ void grid_zero(float *p, int n) {
+  for (int i = (blockIdx.x * PK_THREADS + threadIdx.x) * 4; i < n; i += gridDim.x * PK_THREADS * 4) {
+    if (i + 4 <= n) {
+      *reinterpret_cast<float4 *>(p + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+    } else {
+      for (int j = i; j < n; ++j) p[j] = 0.f;
+    }
+  }
+}
+
+}  // namespace dmtd
