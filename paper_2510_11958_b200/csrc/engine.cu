@@ -69,7 +69,6 @@ struct dmtd_ctx {
   float *f_part_o = nullptr, *f_part_ml = nullptr, *amax_val = nullptr;
   int *amax_idx = nullptr;
   unsigned int *grid_bar = nullptr;
-  int *attn_count = nullptr;
   long long *pass_timing = nullptr;         // profiling builds only
 
   // graphs: [kind 1 = full, 2 = upper-only]
@@ -130,22 +129,23 @@ dmtd_status check_launch(dmtd_ctx *c, const char *what) {
 bool is_bf16(const dmtd_ctx *c) { return c->s.weight_dtype == DMTD_BF16; }
 size_t wbytes(const dmtd_ctx *c) { return is_bf16(c) ? 2 : 4; }
 
-// Largest divisor of the atom count per row that keeps a k-slab at or below 40 atoms.
-int choose_aps(int K) {
+// Largest divisor of the atom count per row that keeps a k-slab at or below `cap` atoms.
+int choose_aps(int K, int cap) {
   int atoms = K / 32, best = 1;
-  for (int d = 1; d <= std::min(atoms, 40); ++d)
+  for (int d = 1; d <= std::min(atoms, cap); ++d)
     if (atoms % d == 0) best = d;
   return best;
 }
 
 // Build one packed matrix from up to three row blocks (e.g. q, k, v) of equal K.
-dmtd_status pack_matrix(dmtd_ctx *c, PackedMat *out, int K, const void *const *srcs, const int *Ns, int n_src) {
+dmtd_status pack_matrix(dmtd_ctx *c, PackedMat *out, int K, const void *const *srcs, const int *Ns, int n_src,
+                        int aps_cap = 40) {
   int N = 0;
   for (int i = 0; i < n_src; ++i) N += Ns[i];
   PackedMat m{};
   m.N = N; m.K = K; m.n_tiles = (N + 15) / 16;
   if (is_bf16(c)) {
-    m.aps = choose_aps(K);
+    m.aps = choose_aps(K, aps_cap);
     m.n_slabs = K / 32 / m.aps;
     uint4 *dst = nullptr;
     TRY(dev_alloc(c, &dst, (size_t)packed_atoms(m) * 64));
@@ -332,7 +332,6 @@ dmtd_status setup_fused(dmtd_ctx *c) {
   c->fused_ok = false;
   if (!is_bf16(c) || s.kv_dtype != DMTD_BF16 || s.head_dim != PK_D || s.n_layers > PK_MAX_LAYERS) return DMTD_OK;
   if (s.n_q_heads / s.n_kv_heads > PK_QR || s.hidden % 8 || s.hidden > PK_XS_FLOATS) return DMTD_OK;
-  if (c->max_batch * s.n_kv_heads > PK_THREADS) return DMTD_OK;
   int coop = 0;
   CUDA_TRY(c, cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
   if (!coop) return DMTD_OK;
@@ -348,6 +347,7 @@ dmtd_status setup_fused(dmtd_ctx *c) {
     if (!fused_matrix_ok(ld.qkv, c->n_sms) || !fused_matrix_ok(ld.o, c->n_sms) || !fused_matrix_ok(ld.gu, c->n_sms) ||
         !fused_matrix_ok(ld.down, c->n_sms))
       return DMTD_OK;
+    if ((ld.o.aps * 32) % PK_D) return DMTD_OK;
   }
   std::vector<PassLayer> h(s.n_layers);
   for (int l = 0; l < s.n_layers; ++l) {
@@ -366,7 +366,6 @@ dmtd_status setup_fused(dmtd_ctx *c) {
   TRY(dev_alloc(c, &c->amax_val, (size_t)PK_MAX_ROWS * c->n_sms));
   TRY(dev_alloc(c, &c->amax_idx, (size_t)PK_MAX_ROWS * c->n_sms));
   TRY(dev_alloc(c, &c->grid_bar, 1));
-  TRY(dev_alloc(c, &c->attn_count, (size_t)c->max_batch * s.n_kv_heads));
 #ifdef DMTD_PASS_TIMING
   TRY(dev_alloc(c, &c->pass_timing, (size_t)2 * PK_TIMING_SLOTS));
 #endif
@@ -395,7 +394,7 @@ dmtd_status enqueue_pass_fused(dmtd_ctx *c, int kind, int R_lower, bool write_to
   P.kind = kind; P.write_token = write_token ? 1 : 0;
   P.tokens = c->tokens; P.st = c->dstate;
   P.x_lo = c->x_lo; P.x_up = c->x_up; P.qkv = c->qkv; P.gu = c->gu; P.logits = c->logits;
-  P.attn_out = c->act; P.lda = c->lda; P.attn_count = c->attn_count; P.timing = c->pass_timing;
+  P.timing = c->pass_timing;
   P.part_o = c->f_part_o; P.part_ml = c->f_part_ml; P.amax_val = c->amax_val; P.amax_idx = c->amax_idx;
   P.out_argmax = out_argmax; P.barrier = c->grid_bar; P.error = &c->dstate->error;
   P.wait_limit = 2000000000ll;              // about a second of SM clock
@@ -556,7 +555,8 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
     int qkv_n[3] = {QD, KVD, KVD};
     CTRY(pack_matrix(c, &ld.qkv, H, qkv_src, qkv_n, 3));
     const void *o_src[1] = {lw.o_proj}; int o_n[1] = {H};
-    CTRY(pack_matrix(c, &ld.o, QD, o_src, o_n, 1));
+    // k-slabs of two heads: a block of the pass kernel then merges the attention slices of few heads
+    CTRY(pack_matrix(c, &ld.o, QD, o_src, o_n, 1, D == 128 ? 8 : 40));
     const void *gu_src[2] = {lw.gate_proj, lw.up_proj}; int gu_n[2] = {I, I};
     CTRY(pack_matrix(c, &ld.gu, H, gu_src, gu_n, 2));
     const void *d_src[1] = {lw.down_proj}; int d_n[1] = {H};

@@ -17,8 +17,7 @@ constexpr int PK_AT_Q = PK_AT_V + PK_TK * PK_VROW;            // [PK_QR][PK_QROW
 constexpr int PK_AT_NEW = PK_AT_Q + PK_QR * PK_QROW;          // K rows of the pass [4][256 B], then V rows [4][256 B]
 constexpr int PK_AT_OS = 0;                                   // after the tiles are consumed: [warps][16][128] floats
 constexpr int PK_AT_RED = PK_WARPS * PK_QR * PK_D * 4;        // running max [warps][16], running sum [warps][16]
-constexpr int PK_AT_FLAG = PK_AT_RED + 2 * PK_WARPS * PK_QR * 4;
-constexpr int PK_AT_END = PK_AT_FLAG + 16;
+constexpr int PK_AT_END = PK_AT_RED + 2 * PK_WARPS * PK_QR * 4;
 static_assert(PK_AT_NEW + 2 * PK_MAX_ROWS * 256 <= PK_AT_RED, "tiles overlap the reduction arrays");
 static_assert(PK_AT_END <= PK_BSTAGE_BYTES + PK_XS_BYTES, "attention scratch does not fit");
 
@@ -92,43 +91,11 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
   }
 }
 
-// The block that completes a (sequence, kv head) merges its key slices (online-softmax merge)
-// into the attention output rows; one warp per query row, one lane per 4 output values.
-__device__ __forceinline__ void attn_merge(const PassParams &P, int b, int kvh, int R, int nsplit) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int G = P.nq / P.nkv, nQ = R * G;
-  for (int qi = warp; qi < nQ; qi += PK_WARPS) {
-    const int m_row = b * R + qi / G, h = kvh * G + qi % G;
-    const size_t slot0 = ((size_t)m_row * P.nq + h) * PK_NSPLIT_CAP;
-    float2 ml = make_float2(-INFINITY, 0.f);
-    if (lane < nsplit) ml = __ldcg(reinterpret_cast<const float2 *>(P.part_ml) + slot0 + lane);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float wgt = 0.f, ltot = 1.f;
-    for (int s0 = 0; s0 < nsplit; s0 += PK_NSPLIT_CAP / 2) {
-      float4 po[PK_NSPLIT_CAP / 2];
-#pragma unroll
-      for (int s = 0; s < PK_NSPLIT_CAP / 2; ++s)
-        if (s0 + s < nsplit) po[s] = __ldcg(reinterpret_cast<const float4 *>(P.part_o + (slot0 + s0 + s) * PK_D) + lane);
-      if (s0 == 0) {
-        const float mxx = warp_max(ml.y > 0.f ? ml.x : -INFINITY);
-        wgt = ml.y > 0.f ? __expf(ml.x - mxx) : 0.f;
-        ltot = warp_sum(wgt * ml.y);
-      }
-#pragma unroll
-      for (int s = 0; s < PK_NSPLIT_CAP / 2; ++s) {
-        const float w = __shfl_sync(0xffffffffu, wgt, (s0 + s) & 31);
-        if (s0 + s < nsplit) { acc.x += w * po[s].x; acc.y += w * po[s].y; acc.z += w * po[s].z; acc.w += w * po[s].w; }
-      }
-    }
-    const float inv = 1.f / ltot;
-    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-    *reinterpret_cast<float4 *>(P.attn_out + (size_t)m_row * P.lda + (size_t)h * PK_D + lane * 4) = acc;
-  }
-}
-
 // Steps a3 + a4 for the items (sequence, kv head, key slice) of this block.  The R*G query rows
 // of an item form one m16 tile; S = Q K^T and O = P V run as mma.m16n8k16 with K and V staged in
 // shared memory, each warp taking 16 keys of a 64-key tile with its own running max and sum.
+// The slice's unnormalised partial output goes to global memory with its max and sum; the
+// prologue of the O projection merges the slices.
 __device__ __noinline__ void attention_stage(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
   const PassShared S = pass_shared();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -143,22 +110,31 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
   float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
   float *const red_m = reinterpret_cast<float *>(sc + PK_AT_RED);
   float *const red_l = red_m + PK_WARPS * PK_QR;
-  volatile int *const last_flag = reinterpret_cast<volatile int *>(sc + PK_AT_FLAG);
 
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
     const int split = item % nsplit, kvh = (item / nsplit) % P.nkv, b = item / (nsplit * P.nkv);
-    pk_sync();
-    // query rows beyond nQ are zero (the previous item's partial outputs lay over the Q tile)
-    for (int i = threadIdx.x; i < PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(q_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
-    pk_sync();
-    attn_new_rows(P, Ly, sc, b, kvh, R, pos0, split == 0);
-
     // keys [j0, j1) of the cache, then (last slice) the R keys of the pass
     const int j0 = split * CH, j1 = min(j0 + CH, pos0);
     const int n_cached = max(0, j1 - j0);
     const int n_keys = n_cached + (split == nsplit - 1 ? R : 0);
     const __nv_bfloat16 *kbase = Ly.kc + ((size_t)b * P.nkv + kvh) * P.max_seq * PK_D;
     const __nv_bfloat16 *vbase = Ly.vc + ((size_t)b * P.nkv + kvh) * P.max_seq * PK_D;
+    // cached rows of a tile: asynchronous copies, 16 bytes each (a row is 16 K parts and 16 V parts)
+    auto fetch_cached = [&](int tile0) {
+      const int n_c = min(PK_TK, n_cached - tile0);
+      for (int c = threadIdx.x; c < n_c * 32; c += PK_THREADS) {
+        const int row = c >> 5, part = c & 31;
+        const uint32_t dst = part < 16 ? k_tile + row * PK_KROW + part * 16 : v_tile + row * PK_VROW + (part - 16) * 16;
+        cp_async16(dst, (part < 16 ? kbase : vbase) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
+      }
+    };
+    pk_sync();                                            // the previous item is done with the scratch
+    // query rows beyond nQ are zero (the previous item's partial outputs lay over the Q tile)
+    for (int i = threadIdx.x; i < PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(q_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
+    fetch_cached(0);                                      // in flight while the pass's own rows are prepared
+    pk_sync();
+    attn_new_rows(P, Ly, sc, b, kvh, R, pos0, split == 0);
+
     float m_run[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};
     float o[16][4];
 #pragma unroll
@@ -167,15 +143,12 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
       const int n_t = min(PK_TK, n_keys - tile0);
       pk_sync();                                          // new rows written / previous tile consumed
-      for (int c = threadIdx.x; c < n_t * 32; c += PK_THREADS) {
+      if (tile0 > 0) fetch_cached(tile0);
+      for (int c = threadIdx.x + max(0, n_cached - tile0) * 32; c < n_t * 32; c += PK_THREADS) {
         const int row = c >> 5, part = c & 31, idx = tile0 + row;
         const uint32_t dst = part < 16 ? k_tile + row * PK_KROW + part * 16 : v_tile + row * PK_VROW + (part - 16) * 16;
-        if (idx < n_cached) {
-          cp_async16(dst, (part < 16 ? kbase : vbase) + (size_t)(j0 + idx) * PK_D + (part & 15) * 8);
-        } else {
-          const unsigned char *src = sc + PK_AT_NEW + ((part < 16 ? 0 : PK_MAX_ROWS) + (idx - n_cached)) * 256 + (part & 15) * 16;
-          sts128(dst, *reinterpret_cast<const uint4 *>(src));
-        }
+        const unsigned char *src = sc + PK_AT_NEW + ((part < 16 ? 0 : PK_MAX_ROWS) + (idx - n_cached)) * 256 + (part & 15) * 16;
+        sts128(dst, *reinterpret_cast<const uint4 *>(src));
       }
       const int n16 = min(PK_TK, (n_t + 15) & ~15);
       for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS)      // P = 0 times stale bits must stay 0
@@ -283,15 +256,6 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
       if (dd == 0) { P.part_ml[slot * 2] = m; P.part_ml[slot * 2 + 1] = l; }
     }
 
-    __threadfence();
-    pk_sync();
-    if (threadIdx.x == 0) *last_flag = atomicAdd(P.attn_count + b * P.nkv + kvh, 1) == nsplit - 1;
-    pk_sync();
-    if (*last_flag) {
-      __threadfence();
-      attn_merge(P, b, kvh, R, nsplit);
-      if (threadIdx.x == 0) P.attn_count[b * P.nkv + kvh] = 0;
-    }
   }
   pk_sync();
 }

@@ -1,14 +1,16 @@
 // Shared definitions of the persistent pass kernel: sizes, parameters, PTX wrappers, the
 // shared-memory map, the per-warp weight stream and the grid barrier.
 //
-// Lessons the layout encodes (measured on B200):
+// Lessons the layout encodes (measured on B200, Qwen3-4B shape, batch 1):
 //  * every stage runs once per layer and the stages of a layer are different code, so the code
 //    of one layer must stay resident in the instruction cache: stage functions are separate,
 //    small, and loop instead of unrolling;
 //  * any load that crosses the chip costs a microsecond or more while the weight stream is
 //    running, so a stage issues all of its loads before it uses any, and nothing in the weight
 //    loop touches local or global memory;
-//  * more bulk copies in flight than bandwidth x latency only lengthen every other round trip.
+//  * more bulk copies in flight than bandwidth x latency only lengthen every other round trip:
+//    with 16 KiB per warp in flight a barrier poll or an activation load waited 3-4 us behind
+//    the block's own weight traffic, with 8 KiB about half of that, at the same stream rate.
 #pragma once
 
 #include "common.cuh"
@@ -19,20 +21,23 @@ constexpr int PK_WARPS = 8;
 constexpr int PK_THREADS = PK_WARPS * 32;
 constexpr int PK_CHUNK_ATOMS = 4;                          // atoms (1 KiB each) per bulk copy
 constexpr int PK_CHUNK_BYTES = PK_CHUNK_ATOMS * 1024;
-constexpr int PK_SLOTS = 4;                                // ring slots per warp
+#ifndef DMTD_PASS_SLOTS
+#define DMTD_PASS_SLOTS 2
+#endif
+constexpr int PK_SLOTS = DMTD_PASS_SLOTS;                  // ring slots per warp
 constexpr int PK_MAX_ROWS = 4;                             // activation rows (B*R) per stage
 constexpr int PK_MAX_KS = 1280;                            // largest k-slab of a packed matrix
 constexpr int PK_MAX_LAYERS = 40;
-constexpr int PK_NSPLIT_CAP = 32;                          // key slices per (sequence, kv head)
+constexpr int PK_NSPLIT_CAP = 16;                          // key slices per (sequence, kv head)
 constexpr int PK_D = 128;                                  // head_dim
 constexpr int PK_QR = 16;                                  // query rows per attention item
-constexpr int PK_XS_FLOATS = 10240;                        // row staging: B*R*hidden floats at most
+constexpr int PK_XS_FLOATS = 20480;                        // activation staging area, floats
 
 // shared memory map (bytes)
-constexpr int PK_RING_BYTES = PK_WARPS * PK_SLOTS * PK_CHUNK_BYTES;           // 131072
+constexpr int PK_RING_BYTES = PK_WARPS * PK_SLOTS * PK_CHUNK_BYTES;           // 65536
 constexpr int PK_BROW_MAX = PK_MAX_KS * 2 + 64;                               // 2624
 constexpr int PK_BSTAGE_BYTES = 2 * 8 * PK_BROW_MAX;                          // 41984: two slabs of 8 columns
-constexpr int PK_XS_BYTES = PK_XS_FLOATS * 4;                                 // 40960
+constexpr int PK_XS_BYTES = PK_XS_FLOATS * 4;                                 // 81920
 constexpr int PK_OFF_RING = 0;
 constexpr int PK_OFF_BSTAGE = PK_OFF_RING + PK_RING_BYTES;
 constexpr int PK_OFF_XS = PK_OFF_BSTAGE + PK_BSTAGE_BYTES;                    // directly behind bstage
@@ -63,9 +68,6 @@ struct PassParams {
   int *tokens;
   DevState *st;
   float *x_lo, *x_up, *qkv, *gu, *logits, *part_o, *part_ml;
-  float *attn_out;                        // merged attention output [row][lda]
-  int lda;
-  int *attn_count;                        // finished key slices per (sequence, kv head)
   float *amax_val;
   int *amax_idx;
   int *out_argmax;
@@ -104,6 +106,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
                : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
   unsigned v;
@@ -133,6 +136,8 @@ struct PassShared {
   float *xs;                // staged activation rows
   uint64_t *bars;           // [warp][slot]
   volatile int *abort_flag;
+  volatile unsigned *stage_uses;        // completed uses of stage_bar (its parity)
+  uint64_t *stage_bar;      // completion of the bulk copies that stage a prologue's inputs
   float *red;               // [PK_WARPS][PK_MAX_ROWS]
   WarpPipe *pipes;          // [PK_WARPS] ring state of every warp between stages
   PassLayer *layers;        // layers [l_begin, l_end) of this pass
@@ -148,6 +153,8 @@ __device__ __forceinline__ PassShared pass_shared() {
   S.xs = reinterpret_cast<float *>(pk_smem + PK_OFF_XS);
   S.bars = reinterpret_cast<uint64_t *>(pk_smem + PK_OFF_BARS);
   S.abort_flag = reinterpret_cast<volatile int *>(pk_smem + PK_OFF_SMALL);
+  S.stage_uses = reinterpret_cast<volatile unsigned *>(pk_smem + PK_OFF_SMALL + 4);
+  S.stage_bar = reinterpret_cast<uint64_t *>(pk_smem + PK_OFF_SMALL + 8);
   S.red = reinterpret_cast<float *>(pk_smem + PK_OFF_SMALL + 64);
   S.pipes = reinterpret_cast<WarpPipe *>(pk_smem + PK_OFF_SMALL + 256);
   S.layers = reinterpret_cast<PassLayer *>(pk_smem + PK_OFF_LAYERS);

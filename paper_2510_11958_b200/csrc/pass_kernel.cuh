@@ -170,7 +170,11 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
     int *dst = reinterpret_cast<int *>(S.layers);
     for (int i = threadIdx.x; i < nL * (int)(sizeof(PassLayer) / 4); i += PK_THREADS) dst[i] = src[i];
   }
-  if (threadIdx.x == 0) *S.abort_flag = 0;
+  if (threadIdx.x == 0) {
+    *S.abort_flag = 0;
+    *S.stage_uses = 0u;
+    mbar_init(smem_u32(S.stage_bar), 1);
+  }
   if (lane == 0) {
     for (int s = 0; s < PK_SLOTS; ++s) mbar_init(smem_u32(S.bars + warp * PK_SLOTS + s), 1);
     fence_mbar_init();
@@ -204,7 +208,6 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
   grid_zero(P.qkv, M_max * ldqkv);
   grid_zero(P.gu, M_max * ldgu);
   grid_zero(P.logits, P.B * P.ldl);
-  if (blockIdx.x == 0 && (int)threadIdx.x < P.B * P.nkv) P.attn_count[threadIdx.x] = 0;
   if (has_lower) embed_rows(P, P.x_lo, M_max, P.R_lo, lo_len);
   else embed_rows(P, P.x_up, P.B, 1, newest);
   bool ok = grid_barrier(P, bar_target);
@@ -239,12 +242,14 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
       }
       W = &Ly.qkv; out = P.qkv; ldo = ldqkv;
     } else if (ph == 1) {
-      // a3 + a4: QK-norm, RoPE, KV append, attention over the key slices and their merge
+      // a3 + a4: QK-norm, RoPE, KV append, attention over the key slices
       attention_stage(P, Ly, R, pos0);
     } else if (ph == 2) {
-      // a5: O projection into the residual rows
+      // a4 merge of the key slices + a5: O projection into the residual rows
       grid_zero(P.gu, M_max * ldgu);
-      plain_prologue(P.attn_out, P.lda, M, Ly.o);
+      int nsplit, CH;
+      attn_plan_device(P, pos0, nsplit, CH);
+      merge_prologue(P, M, nsplit, Ly.o);
       W = &Ly.o; out = x; ldo = P.H;
     } else if (ph == 3) {
       // a6: RMSNorm, gate and up projections

@@ -8,26 +8,25 @@
 
 namespace dmtd {
 
-constexpr int PK_BATCH = 4;          // float4 loads a thread keeps in flight in an elementwise prologue
-constexpr int PK_STAGE_BATCH = 8;    // float4 loads a thread keeps in flight while staging rows
 constexpr int PK_SPAN_UNITS = 3;     // float4 units of a block's k-slab span per thread: span <= 3072 values
 
-// Copy M rows of H floats (row r at src + r * row_stride) into shared memory.
-__device__ __forceinline__ void stage_rows(float *xs, const float *src, size_t row_stride, int M, int H) {
-  const int h4 = H / 4, n4 = M * h4;
-  for (int base = 0; base < n4; base += PK_STAGE_BATCH * PK_THREADS) {
-    float4 tmp[PK_STAGE_BATCH];
-#pragma unroll
-    for (int j = 0; j < PK_STAGE_BATCH; ++j) {
-      const int i = base + j * PK_THREADS + threadIdx.x;
-      if (i < n4) tmp[j] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)(i / h4) * row_stride) + i % h4);
-    }
-#pragma unroll
-    for (int j = 0; j < PK_STAGE_BATCH; ++j) {
-      const int i = base + j * PK_THREADS + threadIdx.x;
-      if (i < n4) reinterpret_cast<float4 *>(xs)[i] = tmp[j];
-    }
-  }
+// Inputs of a prologue come into shared memory as bulk copies issued by one thread: no load
+// instruction waits in a register, and the whole input costs one trip to L2.  stage_begin
+// (thread 0) arms the barrier, stage_copy adds a copy, stage_wait (all threads) waits for them.
+__device__ __forceinline__ void stage_begin(const PassShared &S, uint32_t bytes) {
+  fence_proxy_async_all();              // the copies must see what other blocks wrote before the grid barrier
+  mbar_expect_tx(smem_u32(S.stage_bar), bytes);
+}
+__device__ __forceinline__ void stage_copy(const PassShared &S, void *dst, const void *src, uint32_t bytes) {
+  bulk_g2s(smem_u32(dst), src, bytes, smem_u32(S.stage_bar));
+}
+__device__ __forceinline__ bool stage_wait(const PassParams &P, const PassShared &S) {
+  const unsigned uses = *S.stage_uses;
+  const uint32_t bar = smem_u32(S.stage_bar);
+  bool ok = mbar_try_wait(bar, uses & 1u) || pipe_wait_slow(P, bar, uses & 1u);
+  pk_sync();
+  if (threadIdx.x == 0) *S.stage_uses = uses + 1;
+  return ok;
 }
 
 // RMSNorm of M rows (row r at x + r * row_stride), written as bf16 hi/lo columns for the
@@ -36,6 +35,10 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
                                            const float *w_norm, const PackedMat &W) {
   const PassShared S = pass_shared();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, H = P.H;
+  if (threadIdx.x == 0) {
+    stage_begin(S, (uint32_t)(M * H * 4));
+    for (int m = 0; m < M; ++m) stage_copy(S, S.xs + m * H, x + (size_t)m * row_stride, (uint32_t)(H * 4));
+  }
   const SlabSpan sp = slab_span(W);
   const int ks4 = sp.KS / 4, nu = sp.count * ks4;
   float4 wv[PK_SPAN_UNITS];
@@ -45,8 +48,7 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
     wv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (u < nu) wv[j] = __ldg(reinterpret_cast<const float4 *>(w_norm + sp.first * sp.KS) + u);
   }
-  stage_rows(S.xs, x, row_stride, M, H);
-  pk_sync();
+  stage_wait(P, S);
   for (int m = 0; m < M; ++m) {
     float ss = 0.f;
     for (int k4 = threadIdx.x; k4 < H / 4; k4 += PK_THREADS) {
@@ -81,59 +83,57 @@ __device__ __noinline__ void swiglu_prologue(const PassParams &P, int M, const P
   const PassShared S = pass_shared();
   const SlabSpan sp = slab_span(W);
   const int ks4 = sp.KS / 4, ldgu = 2 * P.I, total = sp.count * M * ks4;
-  for (int base = 0; base < total; base += PK_BATCH * PK_THREADS) {
-    float4 g[PK_BATCH], u[PK_BATCH];
-#pragma unroll
-    for (int j = 0; j < PK_BATCH; ++j) {
-      const int idx = base + j * PK_THREADS + threadIdx.x;
-      if (idx < total) {
-        const int u4 = idx % ks4, m = (idx / ks4) % M, sl = idx / (ks4 * M);
-        const float *src = P.gu + (size_t)m * ldgu + (sp.first + sl) * sp.KS + u4 * 4;
-        g[j] = __ldcg(reinterpret_cast<const float4 *>(src));
-        u[j] = __ldcg(reinterpret_cast<const float4 *>(src + P.I));
-      }
+  if (threadIdx.x == 0) {
+    stage_begin(S, (uint32_t)(sp.count * M * 2 * sp.KS * 4));
+    for (int i = 0; i < sp.count * M; ++i) {             // i = sl * M + m: gate values, then up values
+      const float *src = P.gu + (size_t)(i % M) * ldgu + (sp.first + i / M) * sp.KS;
+      stage_copy(S, S.xs + (size_t)i * 2 * sp.KS, src, (uint32_t)(sp.KS * 4));
+      stage_copy(S, S.xs + (size_t)i * 2 * sp.KS + sp.KS, src + P.I, (uint32_t)(sp.KS * 4));
     }
-#pragma unroll
-    for (int j = 0; j < PK_BATCH; ++j) {
-      const int idx = base + j * PK_THREADS + threadIdx.x;
-      if (idx < total) {
-        const int u4 = idx % ks4, m = (idx / ks4) % M, sl = idx / (ks4 * M);
-        float4 a;
-        a.x = g[j].x / (1.f + __expf(-g[j].x)) * u[j].x;
-        a.y = g[j].y / (1.f + __expf(-g[j].y)) * u[j].y;
-        a.z = g[j].z / (1.f + __expf(-g[j].z)) * u[j].z;
-        a.w = g[j].w / (1.f + __expf(-g[j].w)) * u[j].w;
-        store_act4(S.bstage + (size_t)sl * 8 * sp.row_bytes, sp.row_bytes, m, u4 * 4, a);
-      }
-    }
+  }
+  stage_wait(P, S);
+  for (int idx = threadIdx.x; idx < total; idx += PK_THREADS) {
+    const int i = idx / ks4, u4 = idx - i * ks4;
+    const float4 g = reinterpret_cast<const float4 *>(S.xs + (size_t)i * 2 * sp.KS)[u4];
+    const float4 u = reinterpret_cast<const float4 *>(S.xs + (size_t)i * 2 * sp.KS + sp.KS)[u4];
+    float4 a;
+    a.x = g.x / (1.f + __expf(-g.x)) * u.x;
+    a.y = g.y / (1.f + __expf(-g.y)) * u.y;
+    a.z = g.z / (1.f + __expf(-g.z)) * u.z;
+    a.w = g.w / (1.f + __expf(-g.w)) * u.w;
+    store_act4(S.bstage + (size_t)(i / M) * 8 * sp.row_bytes, sp.row_bytes, i % M, u4 * 4, a);
   }
   pk_sync();
 }
 
-// Rows of `src` [M][ld] as bf16 hi/lo columns for the k-slabs this block needs of W (the merged
-// attention output entering the O projection).
-__device__ __noinline__ void plain_prologue(const float *src, int ld, int M, const PackedMat &W) {
+// Online-softmax merge of the key slices (step a4, second half) for the heads this block's share
+// of the O projection multiplies, written as bf16 hi/lo columns: one warp per (row, head), one
+// lane per 4 output values, every slice's partial output loaded before any is used.
+__device__ __noinline__ void merge_prologue(const PassParams &P, int M, int nsplit, const PackedMat &W) {
   const PassShared S = pass_shared();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const SlabSpan sp = slab_span(W);
-  const int ks4 = sp.KS / 4, total = sp.count * M * ks4;
-  for (int base = 0; base < total; base += PK_BATCH * PK_THREADS) {
-    float4 v[PK_BATCH];
+  const int heads_per_slab = sp.KS / PK_D, n_heads = sp.count * heads_per_slab;
+  for (int pair = warp; pair < M * n_heads; pair += PK_WARPS) {
+    const int m = pair / n_heads, hh = pair - m * n_heads;
+    const int sl = hh / heads_per_slab, h = sp.first * heads_per_slab + hh;
+    const size_t slot0 = ((size_t)m * P.nq + h) * PK_NSPLIT_CAP;
+    float4 po[PK_NSPLIT_CAP];
 #pragma unroll
-    for (int j = 0; j < PK_BATCH; ++j) {
-      const int idx = base + j * PK_THREADS + threadIdx.x;
-      if (idx < total) {
-        const int u4 = idx % ks4, m = (idx / ks4) % M, sl = idx / (ks4 * M);
-        v[j] = __ldcg(reinterpret_cast<const float4 *>(src + (size_t)m * ld + (sp.first + sl) * sp.KS + u4 * 4));
-      }
-    }
+    for (int s = 0; s < PK_NSPLIT_CAP; ++s)
+      if (s < nsplit) po[s] = __ldcg(reinterpret_cast<const float4 *>(P.part_o + (slot0 + s) * PK_D) + lane);
+    float2 ml = make_float2(-INFINITY, 0.f);
+    if (lane < nsplit) ml = __ldcg(reinterpret_cast<const float2 *>(P.part_ml) + slot0 + lane);
+    const float mxx = warp_max(ml.y > 0.f ? ml.x : -INFINITY);
+    float wgt = ml.y > 0.f ? __expf(ml.x - mxx) : 0.f;
+    wgt /= warp_sum(wgt * ml.y);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int j = 0; j < PK_BATCH; ++j) {
-      const int idx = base + j * PK_THREADS + threadIdx.x;
-      if (idx < total) {
-        const int u4 = idx % ks4, m = (idx / ks4) % M, sl = idx / (ks4 * M);
-        store_act4(S.bstage + (size_t)sl * 8 * sp.row_bytes, sp.row_bytes, m, u4 * 4, v[j]);
-      }
+    for (int s = 0; s < PK_NSPLIT_CAP; ++s) {
+      const float w = __shfl_sync(0xffffffffu, wgt, s);
+      if (s < nsplit) { acc.x += w * po[s].x; acc.y += w * po[s].y; acc.z += w * po[s].z; acc.w += w * po[s].w; }
     }
+    store_act4(S.bstage + (size_t)sl * 8 * sp.row_bytes, sp.row_bytes, m, (hh - sl * heads_per_slab) * PK_D + lane * 4, acc);
   }
   pk_sync();
 }
