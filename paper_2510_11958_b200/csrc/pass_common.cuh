@@ -10,7 +10,9 @@
 //    loop touches local or global memory;
 //  * more bulk copies in flight than bandwidth x latency only lengthen every other round trip:
 //    with 16 KiB per warp in flight a barrier poll or an activation load waited 3-4 us behind
-//    the block's own weight traffic, with 8 KiB about half of that, at the same stream rate.
+//    the block's own weight traffic, with 8 KiB about half of that, at the same stream rate;
+//    asking for the next projection's weights to be prefetched into L2 at a stage boundary made
+//    the following projection slower, not faster, so nothing is requested beyond the ring.
 #pragma once
 
 #include "common.cuh"
