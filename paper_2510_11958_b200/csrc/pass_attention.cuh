@@ -2,7 +2,7 @@
 // (split-KV attention on the tensor cores, online-softmax merge of the key slices).
 #pragma once
 
-#include "pass_stream.cuh"
+#include "pass_prologues.cuh"
 
 namespace dmtd {
 
@@ -15,9 +15,12 @@ constexpr int PK_AT_K = 0;                                    // [PK_TK][PK_KROW
 constexpr int PK_AT_V = PK_AT_K + PK_TK * PK_KROW;            // [PK_TK][PK_VROW]
 constexpr int PK_AT_Q = PK_AT_V + PK_TK * PK_VROW;            // [PK_QR][PK_QROW]
 constexpr int PK_AT_NEW = PK_AT_Q + PK_QR * PK_QROW;          // K rows of the pass [4][256 B], then V rows [4][256 B]
-constexpr int PK_AT_OS = 0;                                   // after the tiles are consumed: [warps][16][128] floats
-constexpr int PK_AT_RED = PK_WARPS * PK_QR * PK_D * 4;        // running max [warps][16], running sum [warps][16]
-constexpr int PK_AT_END = PK_AT_RED + 2 * PK_WARPS * PK_QR * 4;
+constexpr int PK_AT_OS = 0;                                   // after the tiles are consumed: [warps][16][PK_OROW] floats
+constexpr int PK_OROW = PK_D + 8;                             // padded: the 8 rows a warp stores at once hit different banks
+constexpr int PK_AT_RED = PK_WARPS * PK_QR * PK_OROW * 4;     // running max [warps][16], then each warp's merge factor [warps][16]
+constexpr int PK_AT_ROWS = PK_AT_RED + 2 * PK_WARPS * PK_QR * 4;   // the pass's q | k | v vectors of one kv head, fp32, per row
+constexpr int PK_AT_ROW_FLOATS = (PK_QR + 2) * PK_D;
+constexpr int PK_AT_END = PK_AT_ROWS + PK_MAX_ROWS * PK_AT_ROW_FLOATS * 4;
 static_assert(PK_AT_NEW + 2 * PK_MAX_ROWS * 256 <= PK_AT_RED, "tiles overlap the reduction arrays");
 static_assert(PK_AT_END <= PK_BSTAGE_BYTES + PK_XS_BYTES, "attention scratch does not fit");
 
@@ -42,24 +45,26 @@ __device__ __forceinline__ void attn_plan_device(const PassParams &P, int pos0, 
   nsplit = max(1, (pos0 + CH - 1) / CH);
 }
 
-// Step a3 for one (sequence, kv head): one warp per head vector of the pass's rows.  Query rows
+// Step a3 for one (sequence, kv head): one warp per head vector of the pass's rows (staged in
+// shared memory as q heads | k | v per row).  Query rows
 // go to the Q tile (bf16, scaled by 1/sqrt(d)); K and V rows go to the new-row area and, from
 // the block that owns slice 0, into the cache.
 __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLayer &Ly, unsigned char *sc, int b, int kvh,
                                               int R, int pos0, bool write_cache) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int G = P.nq / P.nkv, nQ = R * G, ldq = (P.nq + 2 * P.nkv) * PK_D;
+  const int G = P.nq / P.nkv, nQ = R * G;
+  const float *rows = reinterpret_cast<const float *>(sc + PK_AT_ROWS);
   const float scale = rsqrtf((float)PK_D);
   for (int task = warp; task < nQ + 2 * R; task += PK_WARPS) {
     int r, col, kind;                                   // kind 0 q, 1 k, 2 v
-    if (task < nQ) { r = task / G; col = (kvh * G + task % G) * PK_D; kind = 0; }
-    else if (task < nQ + R) { r = task - nQ; col = (P.nq + kvh) * PK_D; kind = 1; }
-    else { r = task - nQ - R; col = (P.nq + P.nkv + kvh) * PK_D; kind = 2; }
-    const float *src = P.qkv + (size_t)(b * R + r) * ldq + col;
+    if (task < nQ) { r = task / G; col = (task % G) * PK_D; kind = 0; }
+    else if (task < nQ + R) { r = task - nQ; col = G * PK_D; kind = 1; }
+    else { r = task - nQ - R; col = (G + 1) * PK_D; kind = 2; }
+    const float *src = rows + r * PK_AT_ROW_FLOATS + col;
     const int pos = pos0 + r;
     float v[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) v[j] = __ldcg(src + lane + 32 * j);
+    for (int j = 0; j < 4; ++j) v[j] = src[lane + 32 * j];
     if (kind != 2) {
       float ss = v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
       ss = warp_sum(ss);
@@ -91,6 +96,20 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
   }
 }
 
+// Profiling builds: cycles thread 0 of block 0 spends in each part of the attention stage.
+#ifdef DMTD_PASS_TIMING
+#define AT_STAMP(i)                                                              \
+  do {                                                                           \
+    if (threadIdx.x == 0 && blockIdx.x == 0 && P.timing) {                       \
+      const long long now_ = clock64();                                          \
+      P.timing[2 * 4096 - 16 + (i)] += now_ - at_t;                              \
+      at_t = now_;                                                               \
+    }                                                                            \
+  } while (0)
+#else
+#define AT_STAMP(i) do {} while (0)
+#endif
+
 // Steps a3 + a4 for the items (sequence, kv head, key slice) of this block.  The R*G query rows
 // of an item form one m16 tile; S = Q K^T and O = P V run as mma.m16n8k16 with K and V staged in
 // shared memory, each warp taking 16 keys of a 64-key tile with its own running max and sum.
@@ -111,6 +130,9 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
   float *const red_m = reinterpret_cast<float *>(sc + PK_AT_RED);
   float *const red_l = red_m + PK_WARPS * PK_QR;
 
+#ifdef DMTD_PASS_TIMING
+  long long at_t = clock64();
+#endif
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
     const int split = item % nsplit, kvh = (item / nsplit) % P.nkv, b = item / (nsplit * P.nkv);
     // keys [j0, j1) of the cache, then (last slice) the R keys of the pass
@@ -129,11 +151,26 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
       }
     };
     pk_sync();                                            // the previous item is done with the scratch
+    if (threadIdx.x == 0) {
+      // the pass's own q | k | v vectors of this kv head: three bulk copies per row
+      const int ldq = (P.nq + 2 * P.nkv) * PK_D;
+      stage_begin(S, (uint32_t)(R * (G + 2) * PK_D * 4));
+      for (int r = 0; r < R; ++r) {
+        const float *src = P.qkv + (size_t)(b * R + r) * ldq;
+        float *dst = reinterpret_cast<float *>(sc + PK_AT_ROWS) + r * PK_AT_ROW_FLOATS;
+        stage_copy(S, dst, src + kvh * G * PK_D, (uint32_t)(G * PK_D * 4));
+        stage_copy(S, dst + G * PK_D, src + (P.nq + kvh) * PK_D, PK_D * 4);
+        stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
+      }
+    }
+    fetch_cached(0);                                      // in flight while the pass's own rows are prepared
     // query rows beyond nQ are zero (the previous item's partial outputs lay over the Q tile)
     for (int i = threadIdx.x; i < PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(q_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
-    fetch_cached(0);                                      // in flight while the pass's own rows are prepared
-    pk_sync();
+    AT_STAMP(0);
+    stage_wait(P, S);
+    AT_STAMP(1);
     attn_new_rows(P, Ly, sc, b, kvh, R, pos0, split == 0);
+    AT_STAMP(2);
 
     float m_run[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};
     float o[16][4];
@@ -155,6 +192,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
         sts128(v_tile + (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16, make_uint4(0u, 0u, 0u, 0u));
       cp_async_wait_all();
       pk_sync();
+      AT_STAMP(3);
       if (tile0 == 0) {
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
@@ -224,6 +262,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
       }
     }
 
+    AT_STAMP(4);
     // combine the warps into this slice's partial result
     pk_sync();                                            // tiles consumed: their space becomes o_s
 #pragma unroll
@@ -232,29 +271,50 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
       l_part[hr] += __shfl_xor_sync(0xffffffffu, l_part[hr], 2);
       if (t == 0) { red_m[warp * PK_QR + g + 8 * hr] = m_run[hr]; red_l[warp * PK_QR + g + 8 * hr] = l_part[hr]; }
     }
+    if (g < nQ) {
 #pragma unroll
-    for (int dt = 0; dt < 16; ++dt) {
-      *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g) * PK_D + dt * 8 + 2 * t) = make_float2(o[dt][0], o[dt][1]);
-      *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g + 8) * PK_D + dt * 8 + 2 * t) = make_float2(o[dt][2], o[dt][3]);
+      for (int dt = 0; dt < 16; ++dt)
+        *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][0], o[dt][1]);
+    }
+    if (g + 8 < nQ) {
+#pragma unroll
+      for (int dt = 0; dt < 16; ++dt)
+        *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g + 8) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][2], o[dt][3]);
     }
     pk_sync();
-    for (int idx = threadIdx.x; idx < nQ * PK_D; idx += PK_THREADS) {
-      const int qi = idx / PK_D, dd = idx % PK_D;
+    AT_STAMP(5);
+    // per query row: the slice's max and sum, and the factor each warp's share is scaled by
+    if ((int)threadIdx.x < nQ) {
+      const int qi = threadIdx.x;
       float m = -INFINITY;
 #pragma unroll
       for (int w = 0; w < PK_WARPS; ++w) m = fmaxf(m, red_m[w * PK_QR + qi]);
-      float l = 0.f, acc = 0.f;
+      float l = 0.f;
 #pragma unroll
       for (int w = 0; w < PK_WARPS; ++w) {
         const float mw = red_m[w * PK_QR + qi];
         const float f = mw > -INFINITY ? __expf(mw - m) : 0.f;
         l += red_l[w * PK_QR + qi] * f;
-        acc += o_s[(w * PK_QR + qi) * PK_D + dd] * f;
+        red_l[w * PK_QR + qi] = f;
       }
       const size_t slot = ((size_t)(b * R + qi / G) * P.nq + kvh * G + qi % G) * PK_NSPLIT_CAP + split;
-      P.part_o[slot * PK_D + dd] = acc;
-      if (dd == 0) { P.part_ml[slot * 2] = m; P.part_ml[slot * 2 + 1] = l; }
+      P.part_ml[slot * 2] = m;
+      P.part_ml[slot * 2 + 1] = l;
     }
+    pk_sync();
+    for (int idx = threadIdx.x; idx < nQ * (PK_D / 4); idx += PK_THREADS) {
+      const int qi = idx / (PK_D / 4), d4 = idx % (PK_D / 4);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int w = 0; w < PK_WARPS; ++w) {
+        const float f = red_l[w * PK_QR + qi];
+        const float4 v = *reinterpret_cast<const float4 *>(o_s + (w * PK_QR + qi) * PK_OROW + d4 * 4);
+        acc.x += v.x * f; acc.y += v.y * f; acc.z += v.z * f; acc.w += v.w * f;
+      }
+      const size_t slot = ((size_t)(b * R + qi / G) * P.nq + kvh * G + qi % G) * PK_NSPLIT_CAP + split;
+      *reinterpret_cast<float4 *>(P.part_o + slot * PK_D + d4 * 4) = acc;
+    }
+    AT_STAMP(6);
 
   }
   pk_sync();

@@ -12,7 +12,6 @@
 #pragma once
 
 #include "pass_attention.cuh"
-#include "pass_prologues.cuh"
 
 namespace dmtd {
 

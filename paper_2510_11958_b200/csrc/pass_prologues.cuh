@@ -14,7 +14,7 @@ constexpr int PK_SPAN_UNITS = 3;     // float4 units of a block's k-slab span pe
 // instruction waits in a register, and the whole input costs one trip to L2.  stage_begin
 // (thread 0) arms the barrier, stage_copy adds a copy, stage_wait (all threads) waits for them.
 __device__ __forceinline__ void stage_begin(const PassShared &S, uint32_t bytes) {
-  fence_proxy_async_all();              // the copies must see what other blocks wrote before the grid barrier
+  fence_proxy_async_global();           // the copies must see what other blocks wrote before the grid barrier
   mbar_expect_tx(smem_u32(S.stage_bar), bytes);
 }
 __device__ __forceinline__ void stage_copy(const PassShared &S, void *dst, const void *src, uint32_t bytes) {
