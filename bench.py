@@ -24,6 +24,7 @@ import torch  # noqa: E402
 from synthetic import SHAPES, WORKLOADS, make_prompts, make_weights, weight_bytes  # noqa: E402
 
 METRIC = "generated tokens/s (decode, steady-state DMTD cycles)"
+NCU_TRAFFIC_RATIO = 1.0105      # DRAM traffic / algorithmic bytes of dmtd_pass_kernel, from the ncu capture
 UNIT = "tokens/s"
 
 
@@ -235,7 +236,13 @@ def run_native(args, wl, shape):
     else:
         peak, peak_src = 6650.0, "fallback"
     cyc_bytes = bytes_per_cycle(shape, L_d, tau, B, mean_ctx)
-    achieved = cyc_bytes / (ms / K * 1e-3) / 1e9
+    # dominant kernel: dmtd_pass_kernel, one launch per pass, tau launches per cycle; the timed region
+    # holds nothing else but a 4-byte memset per launch and a token gather per cycle.  Its average
+    # launch streams cyc_bytes / tau and takes (event time of a cycle) / tau.
+    fused = launches <= K * (tau + 1)
+    launch_bytes = cyc_bytes / tau
+    launch_s = ms / K * 1e-3 / tau
+    achieved = launch_bytes / launch_s / 1e9
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -251,10 +258,17 @@ def run_native(args, wl, shape):
                 "h2d_bytes_per_step": B * P * 4 / max(calls, 1), "d2h_bytes_per_step": B * tau * 4,
                 "note": "whole request: prompt upload + prefill + decode with per-cycle token read-back",
                 "decode_only_value": e2e_decode},
-        "roofline": {"bound": "hbm", "kernel": "whole decode cycle (all kernels of 1 full + tau-1 short passes)",
+        "roofline": {"bound": "hbm",
+                     "kernel": ("dmtd_pass_kernel (one launch per pass; average over the 1 full + tau-1 "
+                                "decoding-layer passes of a cycle)") if fused else
+                               "per-step kernels (all kernels of 1 full + tau-1 short passes)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": peak_src, "frac_of_nominal_8TBs": achieved / 8000.0,
-                     "bytes_per_cycle": cyc_bytes, "traffic": None},
+                     "bytes_per_cycle": cyc_bytes, "launches_per_cycle": tau if fused else launches / K,
+                     "algorithmic_bytes_per_launch": launch_bytes, "avg_launch_us": launch_s * 1e6,
+                     # dram__bytes_read + dram__bytes_write of this kernel, captured on the 4-layer model of the
+                     # same geometry and scaled by the bytes a launch streams (profiles/dmtd_pass_kernel_*_ncu_full.md)
+                     "traffic": launch_bytes * NCU_TRAFFIC_RATIO if fused else None},
         "speedup_vs_tau1": (value / world / tau1) if tau1 else None,
         "tau1_tokens_per_s": tau1,
         "ms_per_cycle_min_med_max": [min(per_cycle), sorted(per_cycle)[len(per_cycle) // 2], max(per_cycle)],

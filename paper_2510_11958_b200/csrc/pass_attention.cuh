@@ -96,20 +96,6 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
   }
 }
 
-// Profiling builds: cycles thread 0 of block 0 spends in each part of the attention stage.
-#ifdef DMTD_PASS_TIMING
-#define AT_STAMP(i)                                                              \
-  do {                                                                           \
-    if (threadIdx.x == 0 && blockIdx.x == 0 && P.timing) {                       \
-      const long long now_ = clock64();                                          \
-      P.timing[2 * 4096 - 16 + (i)] += now_ - at_t;                              \
-      at_t = now_;                                                               \
-    }                                                                            \
-  } while (0)
-#else
-#define AT_STAMP(i) do {} while (0)
-#endif
-
 // Steps a3 + a4 for the items (sequence, kv head, key slice) of this block.  The R*G query rows
 // of an item form one m16 tile; S = Q K^T and O = P V run as mma.m16n8k16 with K and V staged in
 // shared memory, each warp taking 16 keys of a 64-key tile with its own running max and sum.
@@ -130,9 +116,6 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
   float *const red_m = reinterpret_cast<float *>(sc + PK_AT_RED);
   float *const red_l = red_m + PK_WARPS * PK_QR;
 
-#ifdef DMTD_PASS_TIMING
-  long long at_t = clock64();
-#endif
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
     const int split = item % nsplit, kvh = (item / nsplit) % P.nkv, b = item / (nsplit * P.nkv);
     // keys [j0, j1) of the cache, then (last slice) the R keys of the pass
@@ -166,11 +149,8 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     fetch_cached(0);                                      // in flight while the pass's own rows are prepared
     // query rows beyond nQ are zero (the previous item's partial outputs lay over the Q tile)
     for (int i = threadIdx.x; i < PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(q_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
-    AT_STAMP(0);
     stage_wait(P, S);
-    AT_STAMP(1);
     attn_new_rows(P, Ly, sc, b, kvh, R, pos0, split == 0);
-    AT_STAMP(2);
 
     float m_run[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};
     float o[16][4];
@@ -192,7 +172,6 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
         sts128(v_tile + (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16, make_uint4(0u, 0u, 0u, 0u));
       cp_async_wait_all();
       pk_sync();
-      AT_STAMP(3);
       if (tile0 == 0) {
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
@@ -262,7 +241,6 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
       }
     }
 
-    AT_STAMP(4);
     // combine the warps into this slice's partial result
     pk_sync();                                            // tiles consumed: their space becomes o_s
 #pragma unroll
@@ -282,7 +260,6 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
         *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g + 8) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][2], o[dt][3]);
     }
     pk_sync();
-    AT_STAMP(5);
     // per query row: the slice's max and sum, and the factor each warp's share is scaled by
     if ((int)threadIdx.x < nQ) {
       const int qi = threadIdx.x;
@@ -314,7 +291,6 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
       const size_t slot = ((size_t)(b * R + qi / G) * P.nq + kvh * G + qi % G) * PK_NSPLIT_CAP + split;
       *reinterpret_cast<float4 *>(P.part_o + slot * PK_D + d4 * 4) = acc;
     }
-    AT_STAMP(6);
 
   }
   pk_sync();

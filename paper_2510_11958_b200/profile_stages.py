@@ -1,0 +1,84 @@
+"""Per-stage time stamps of the persistent pass kernel.
+
+    python -m paper_2510_11958_b200.profile_stages [--workload qwen3_4b_b1] [--kind full|upper]
+
+Builds a profiling variant of the library (-DDMTD_PASS_TIMING, written beside the normal one as
+libdmtd_b200_timing.so), runs a few decode cycles of the workload and prints, for the first and
+the last block of the grid, how long thread 0 spent in every prologue, projection and grid
+barrier of one pass, averaged over the layers.  Times are clock64() ticks converted with
+--ghz (the SM clock under load; 1.965 GHz on B200 when the kernel is memory-bound).
+"""
+import argparse
+import ctypes as C
+import os
+import subprocess
+import sys
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+ROOT = os.path.dirname(HERE)
+LIB = os.path.join(HERE, "libdmtd_b200_timing.so")
+SLOTS = 4096
+NAMES = ["qkv_pro", "qkv_mma", "qkv_bar", "attn", "-", "attn_bar", "o_pro", "o_mma", "o_bar",
+         "gu_pro", "gu_mma", "gu_bar", "dn_pro", "dn_mma", "dn_bar"]
+
+
+def build_timing_library():
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
+           "-DDMTD_PASS_TIMING", "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"),
+           os.path.join(HERE, "csrc", "engine.cu"), "-o", LIB]
+    subprocess.run(cmd, check=True)
+    return LIB
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="qwen3_4b_b1")
+    ap.add_argument("--kind", default="full", choices=["full", "upper"])
+    ap.add_argument("--ghz", type=float, default=1.965)
+    ap.add_argument("--build-only", action="store_true")
+    args = ap.parse_args()
+    build_timing_library()
+    if args.build_only:
+        return
+    sys.path.insert(0, ROOT)
+    import torch
+    from paper_2510_11958_b200 import binding as bd
+    from synthetic import SHAPES, WORKLOADS, make_prompts, make_weights
+    bd.library_path = lambda: LIB
+    wl = WORKLOADS[args.workload]
+    shape = SHAPES[wl.shape]
+    w = make_weights(shape, seed=wl.weight_seed, device="cuda")
+    eng = bd.Dmtd(shape, w, L_d=wl.L_d, tau=wl.tau, max_batch=wl.batch, max_seq=wl.prompt_len + 64)
+    del w
+    eng.prefill(make_prompts(shape.vocab, wl.batch, wl.prompt_len, seed=wl.prompt_seed).cuda())
+    for _ in range(4):
+        eng.decode_cycle(wl.tau)                     # ends at a cycle boundary: the next pass is a full one
+    if args.kind == "upper":
+        eng.decode_cycle(1)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    ev[0].record()
+    eng.decode_cycle(1)
+    ev[1].record()
+    torch.cuda.synchronize()
+    print(f"{args.workload}, {args.kind} pass: {ev[0].elapsed_time(ev[1]) * 1e3:.1f} us by CUDA events")
+    buf = np.zeros(2 * SLOTS, np.int64)
+    eng.dll.dmtd_debug_pass_timing.argtypes = [C.c_void_p, C.c_void_p]
+    assert eng.dll.dmtd_debug_pass_timing(eng._ctx, buf.ctypes.data_as(C.c_void_p)) == 0
+    n_layers = shape.n_layers if args.kind == "full" else wl.L_d
+    for blk, label in ((0, "first block"), (1, "last block")):
+        s = buf[blk * SLOTS:(blk + 1) * SLOTS]
+        n = 1 + n_layers * 15 + 3
+        d = np.diff(s[:n]) / (args.ghz * 1e3)
+        per = d[: n_layers * 15].reshape(n_layers, 15)
+        print(f"{label}: {(s[n - 1] - s[0]) / (args.ghz * 1e3):.1f} us from first to last stamp")
+        print("  us per layer (mean over layers 1..): " +
+              " ".join(f"{nm}={per[1:, i].mean():.1f}" for i, nm in enumerate(NAMES) if nm != "-") +
+              f" | sum {per[1:].mean(0).sum():.1f}")
+        print("  head: prologue %.1f, projection %.1f, barrier %.1f" % tuple(d[n_layers * 15: n_layers * 15 + 3]))
+
+
+if __name__ == "__main__":
+    main()

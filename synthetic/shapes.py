@@ -46,6 +46,10 @@ SHAPES = {
     # The paper's default base model (Section 3.1): 36 layers, last 8 are decoding layers.
     "qwen3_4b": ModelShape(n_layers=36, hidden=2560, n_q_heads=32, n_kv_heads=8, head_dim=128,
                            intermediate=9728, vocab=151936, dtype="bf16"),
+    # The same layer and head geometry with 4 layers: small enough (1.6 GB) to capture with a
+    # profiler, large enough that every launch streams far more than the L2 holds.
+    "qwen3_4b_l4": ModelShape(n_layers=4, hidden=2560, n_q_heads=32, n_kv_heads=8, head_dim=128,
+                              intermediate=9728, vocab=151936, dtype="bf16"),
 }
 
 
@@ -69,6 +73,8 @@ WORKLOADS = {
     "tiny_b1": Workload("tiny_b1", "tiny", L_d=2, tau=3, batch=1, prompt_len=32, gen_len=24),
     "qwen3_4b_b1": Workload("qwen3_4b_b1", "qwen3_4b", L_d=8, tau=3, batch=1, prompt_len=512,
                             gen_len=256),
+    "qwen3_4b_l4_b1": Workload("qwen3_4b_l4_b1", "qwen3_4b_l4", L_d=2, tau=3, batch=1, prompt_len=512,
+                               gen_len=64),
     "qwen3_4b_b32": Workload("qwen3_4b_b32", "qwen3_4b", L_d=8, tau=3, batch=32, prompt_len=1024,
                              gen_len=512),
     "qwen3_4b_long": Workload("qwen3_4b_long", "qwen3_4b", L_d=8, tau=3, batch=8,
