@@ -28,12 +28,12 @@ NCU_TRAFFIC_RATIO = 1.0105      # DRAM traffic / algorithmic bytes of dmtd_pass_
 UNIT = "tokens/s"
 
 
-def bytes_per_cycle(shape, L_d, tau, batch, mean_ctx):
+def bytes_per_cycle(shape, L_d, tau, batch, mean_ctx, kv_bytes=2):
     """Bytes the cycle must move: every layer-pass reads that layer's weights once and the KV
     of every sequence once; every pass reads the tied head once."""
     w_layer, w_head = weight_bytes(shape)
     layer_passes = shape.n_layers + (tau - 1) * L_d
-    kv_per_pos = 2 * shape.n_kv_heads * shape.head_dim * 2          # K and V, bf16
+    kv_per_pos = 2 * shape.n_kv_heads * shape.head_dim * kv_bytes   # K and V
     return layer_passes * w_layer + tau * w_head + layer_passes * batch * mean_ctx * kv_per_pos
 
 
@@ -158,7 +158,7 @@ def run_native(args, wl, shape):
     with torch.cuda.stream(stream):
         weights = make_weights(shape, seed=wl.weight_seed, device="cuda")
         wh = host_copy(weights) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
-        eng = Dmtd(shape, weights, L_d=L_d, tau=tau, max_batch=B, max_seq=max_seq)
+        eng = Dmtd(shape, weights, L_d=L_d, tau=tau, max_batch=B, max_seq=max_seq, kv_dtype=wl.kv_dtype)
         del weights
         torch.cuda.empty_cache()
         prompts_host = make_prompts(shape.vocab, B, P, seed=wl.prompt_seed).pin_memory()
@@ -235,7 +235,7 @@ def run_native(args, wl, shape):
         peak, peak_src = json.load(open(peaks_path))["hbm_gbs"], "measured"
     else:
         peak, peak_src = 6650.0, "fallback"
-    cyc_bytes = bytes_per_cycle(shape, L_d, tau, B, mean_ctx)
+    cyc_bytes = bytes_per_cycle(shape, L_d, tau, B, mean_ctx, kv_bytes=4 if wl.kv_dtype == "f32" else 2)
     # dominant kernel: dmtd_pass_kernel, one launch per pass, tau launches per cycle; the timed region
     # holds nothing else but a 4-byte memset per launch and a token gather per cycle.  Its average
     # launch streams cyc_bytes / tau and takes (event time of a cycle) / tau.
@@ -246,7 +246,7 @@ def run_native(args, wl, shape):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 weights and KV, fp32 accumulate" if shape.dtype == "bf16" else "f32",
+        "dtype": f"bf16 weights, {wl.kv_dtype} KV cache, fp32 accumulate" if shape.dtype == "bf16" else "f32",
         "data": "synthetic",
         "config": {"workload": wl.name, "shape": wl.shape, "tau": tau, "L_d": L_d, "batch": B,
                    "prompt_len": P, "context_during_timing": [ctx_begin, ctx_begin + K * tau],

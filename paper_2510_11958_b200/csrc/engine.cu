@@ -330,8 +330,8 @@ bool fused_matrix_ok(const PackedMat &m, int grid) {
 dmtd_status setup_fused(dmtd_ctx *c) {
   const dmtd_model_shape &s = c->s;
   c->fused_ok = false;
-  if (!is_bf16(c) || s.kv_dtype != DMTD_BF16 || s.head_dim != PK_D || s.n_layers > PK_MAX_LAYERS) return DMTD_OK;
-  if (s.n_q_heads / s.n_kv_heads > PK_QR || s.hidden % 8 || s.hidden > PK_XS_FLOATS) return DMTD_OK;
+  if (!is_bf16(c) || s.head_dim != PK_D || s.n_layers > PK_MAX_LAYERS) return DMTD_OK;
+  if (s.n_q_heads / s.n_kv_heads > PK_MAX_GROUP || s.hidden % 8 || s.hidden > PK_XS_FLOATS) return DMTD_OK;
   int coop = 0;
   CUDA_TRY(c, cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
   if (!coop) return DMTD_OK;
@@ -354,8 +354,9 @@ dmtd_status setup_fused(dmtd_ctx *c) {
     const LayerDev &ld = c->layers[l];
     h[l].qkv = ld.qkv; h[l].o = ld.o; h[l].gu = ld.gu; h[l].down = ld.down;
     h[l].w_in = ld.w_in; h[l].w_post = ld.w_post; h[l].w_qn = ld.w_qn; h[l].w_kn = ld.w_kn;
-    h[l].kc = static_cast<__nv_bfloat16 *>(c->kc) + (size_t)l * c->kv_layer_elems;
-    h[l].vc = static_cast<__nv_bfloat16 *>(c->vc) + (size_t)l * c->kv_layer_elems;
+    const size_t kvb = s.kv_dtype == DMTD_BF16 ? 2 : 4;
+    h[l].kc = static_cast<unsigned char *>(c->kc) + (size_t)l * c->kv_layer_elems * kvb;
+    h[l].vc = static_cast<unsigned char *>(c->vc) + (size_t)l * c->kv_layer_elems * kvb;
   }
   TRY(dev_alloc(c, &c->pass_layers, h.size()));
   CUDA_TRY(c, cudaMemcpyAsync(c->pass_layers, h.data(), h.size() * sizeof(PassLayer), cudaMemcpyHostToDevice, c->stream));
@@ -391,7 +392,7 @@ dmtd_status enqueue_pass_fused(dmtd_ctx *c, int kind, int R_lower, bool write_to
   P.R_lo = (kind == 1 && lo > 0) ? R_lower : 1; P.B = c->B;
   P.H = s.hidden; P.I = s.intermediate; P.nq = s.n_q_heads; P.nkv = s.n_kv_heads; P.vocab = s.vocab;
   P.max_seq = c->max_seq; P.ldl = c->ldl; P.eps = s.rms_eps;
-  P.kind = kind; P.write_token = write_token ? 1 : 0;
+  P.kind = kind; P.write_token = write_token ? 1 : 0; P.kv_f32 = s.kv_dtype == DMTD_F32 ? 1 : 0;
   P.tokens = c->tokens; P.st = c->dstate;
   P.x_lo = c->x_lo; P.x_up = c->x_up; P.qkv = c->qkv; P.gu = c->gu; P.logits = c->logits;
   P.timing = c->pass_timing;

@@ -1,27 +1,38 @@
 // Attention stage of the pass kernel: steps a3 (QK-norm, rotary embedding, KV append) and a4
-// (split-KV attention on the tensor cores, online-softmax merge of the key slices).
+// (split-KV attention on the tensor cores; the key slices are merged by the O projection's
+// prologue).
+//
+// Two precisions, chosen by the KV cache's storage type.  With a bf16 cache, Q, K, P and V enter
+// the MMAs as single bf16 values.  With an fp32 cache every operand is a bf16 hi + lo pair and
+// each product is three MMAs (hi*hi + hi*lo + lo*hi), which keeps the attention at fp32 accuracy:
+// on the 36-layer model the bf16 cache alone moves the logits by up to 0.05, an fp32 cache by 1e-4.
 #pragma once
 
 #include "pass_prologues.cuh"
 
 namespace dmtd {
 
+constexpr int PK_FETCH = 10;                                  // float4 units of an fp32 tile a thread loads at once
 constexpr int PK_TK = 64;                                     // keys per shared-memory tile
 constexpr int PK_KROW = 320;                                  // bytes per K row: 256 + 64, conflict-free 16-byte operand loads
 constexpr int PK_VROW = 272;                                  // bytes per V row: 256 + 16, conflict-free ldmatrix
 constexpr int PK_QROW = 272;
+constexpr int PK_OROW = PK_D + 8;                             // floats per partial-output row, padded against bank conflicts
 // layout of the attention scratch (the activation staging area and the row staging area behind it)
-constexpr int PK_AT_K = 0;                                    // [PK_TK][PK_KROW]
-constexpr int PK_AT_V = PK_AT_K + PK_TK * PK_KROW;            // [PK_TK][PK_VROW]
-constexpr int PK_AT_Q = PK_AT_V + PK_TK * PK_VROW;            // [PK_QR][PK_QROW]
-constexpr int PK_AT_NEW = PK_AT_Q + PK_QR * PK_QROW;          // K rows of the pass [4][256 B], then V rows [4][256 B]
+constexpr int PK_AT_KH = 0;                                   // K tile, hi parts [PK_TK][PK_KROW]
+constexpr int PK_AT_KL = PK_AT_KH + PK_TK * PK_KROW;          // K tile, lo parts (fp32 cache only)
+constexpr int PK_AT_VH = PK_AT_KL + PK_TK * PK_KROW;          // V tile, hi parts [PK_TK][PK_VROW]
+constexpr int PK_AT_VL = PK_AT_VH + PK_TK * PK_VROW;
+constexpr int PK_AT_QH = PK_AT_VL + PK_TK * PK_VROW;          // Q tile [PK_QR][PK_QROW], hi then lo
+constexpr int PK_AT_QL = PK_AT_QH + PK_QR * PK_QROW;
+constexpr int PK_AT_NEW = PK_AT_QL + PK_QR * PK_QROW;         // K rows of the pass [4][128] floats, then V rows [4][128]
+constexpr int PK_AT_TILES_END = PK_AT_NEW + 2 * PK_MAX_ROWS * PK_D * 4;
 constexpr int PK_AT_OS = 0;                                   // after the tiles are consumed: [warps][16][PK_OROW] floats
-constexpr int PK_OROW = PK_D + 8;                             // padded: the 8 rows a warp stores at once hit different banks
-constexpr int PK_AT_RED = PK_WARPS * PK_QR * PK_OROW * 4;     // running max [warps][16], then each warp's merge factor [warps][16]
+constexpr int PK_AT_RED = 90112;                              // running max [warps][16], then sum / merge factor [warps][16]
 constexpr int PK_AT_ROWS = PK_AT_RED + 2 * PK_WARPS * PK_QR * 4;   // the pass's q | k | v vectors of one kv head, fp32, per row
-constexpr int PK_AT_ROW_FLOATS = (PK_QR + 2) * PK_D;
+constexpr int PK_AT_ROW_FLOATS = (PK_MAX_GROUP + 2) * PK_D;
 constexpr int PK_AT_END = PK_AT_ROWS + PK_MAX_ROWS * PK_AT_ROW_FLOATS * 4;
-static_assert(PK_AT_NEW + 2 * PK_MAX_ROWS * 256 <= PK_AT_RED, "tiles overlap the reduction arrays");
+static_assert(PK_AT_TILES_END <= PK_AT_RED && PK_WARPS * PK_QR * PK_OROW * 4 <= PK_AT_RED, "attention scratch overlaps");
 static_assert(PK_AT_END <= PK_BSTAGE_BYTES + PK_XS_BYTES, "attention scratch does not fit");
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
@@ -45,10 +56,26 @@ __device__ __forceinline__ void attn_plan_device(const PassParams &P, int pos0, 
   nsplit = max(1, (pos0 + CH - 1) / CH);
 }
 
+// 8 values -> 16 bytes of bf16 hi parts and, if asked, 16 bytes of lo parts (x = hi + lo).
+template <bool PRECISE>
+__device__ __forceinline__ void split8(const float (&f)[8], uint4 &hi, uint4 &lo) {
+  uint32_t h[4], l[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    h[j] = pack_bf16x2(f[2 * j], f[2 * j + 1]);
+    l[j] = 0u;
+    if (PRECISE)
+      l[j] = pack_bf16x2(f[2 * j] - __uint_as_float(h[j] << 16), f[2 * j + 1] - __uint_as_float(h[j] & 0xffff0000u));
+  }
+  hi = make_uint4(h[0], h[1], h[2], h[3]);
+  lo = make_uint4(l[0], l[1], l[2], l[3]);
+}
+
 // Step a3 for one (sequence, kv head): one warp per head vector of the pass's rows (staged in
-// shared memory as q heads | k | v per row).  Query rows
-// go to the Q tile (bf16, scaled by 1/sqrt(d)); K and V rows go to the new-row area and, from
+// shared memory as q heads | k | v per row).  Query rows go to the Q tile (scaled by 1/sqrt(d));
+// K and V rows go to the new-row area as floats already rounded to the cache's type and, from
 // the block that owns slice 0, into the cache.
+template <bool PRECISE>
 __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLayer &Ly, unsigned char *sc, int b, int kvh,
                                               int R, int pos0, bool write_cache) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -84,14 +111,60 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
         v[j + 2] = x1 * cs + x0 * sn;
       }
     }
-    __nv_bfloat16 *row = reinterpret_cast<__nv_bfloat16 *>(
-        kind == 0 ? sc + PK_AT_Q + task * PK_QROW : sc + PK_AT_NEW + ((kind == 2 ? PK_MAX_ROWS : 0) + r) * 256);
-    __nv_bfloat16 *cache = (kind == 1 ? Ly.kc : Ly.vc) + (((size_t)b * P.nkv + kvh) * P.max_seq + pos) * PK_D;
+    if (kind == 0) {
+      __nv_bfloat16 *qh = reinterpret_cast<__nv_bfloat16 *>(sc + PK_AT_QH + task * PK_QROW);
+      __nv_bfloat16 *ql = reinterpret_cast<__nv_bfloat16 *>(sc + PK_AT_QL + task * PK_QROW);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const __nv_bfloat16 h = __float2bfloat16_rn(v[j]);
-      row[lane + 32 * j] = h;
-      if (kind != 0 && write_cache) cache[lane + 32 * j] = h;
+      for (int j = 0; j < 4; ++j) {
+        const __nv_bfloat16 h = __float2bfloat16_rn(v[j]);
+        qh[lane + 32 * j] = h;
+        if (PRECISE) ql[lane + 32 * j] = __float2bfloat16_rn(v[j] - __bfloat162float(h));
+      }
+    } else {
+      float *row = reinterpret_cast<float *>(sc + PK_AT_NEW) + ((kind == 2 ? PK_MAX_ROWS : 0) + r) * PK_D;
+      const size_t at = (((size_t)b * P.nkv + kvh) * P.max_seq + pos) * PK_D;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (PRECISE) {
+          row[lane + 32 * j] = v[j];
+          if (write_cache) reinterpret_cast<float *>(kind == 1 ? Ly.kc : Ly.vc)[at + lane + 32 * j] = v[j];
+        } else {
+          const __nv_bfloat16 h = __float2bfloat16_rn(v[j]);
+          row[lane + 32 * j] = __bfloat162float(h);
+          if (write_cache) reinterpret_cast<__nv_bfloat16 *>(kind == 1 ? Ly.kc : Ly.vc)[at + lane + 32 * j] = h;
+        }
+      }
+    }
+  }
+}
+
+// Cached rows of an fp32 tile: through registers, PK_FETCH float4 per thread in flight (one trip
+// for a slice of up to 40 keys), each split into bf16 hi and lo parts.  A function of its own so
+// that its registers are not counted against the attention loop's.
+__device__ __noinline__ void attn_fetch_f32(const float *k_rows, const float *v_rows, int n_rows, unsigned char *sc) {
+  const int total = n_rows * 64;                          // float4 units: 32 of K and 32 of V per row
+  for (int base = 0; base < total; base += PK_FETCH * PK_THREADS) {
+    float4 v[PK_FETCH];
+#pragma unroll
+    for (int j = 0; j < PK_FETCH; ++j) {
+      const int c = base + j * PK_THREADS + threadIdx.x;
+      if (c < total) {
+        const int row = c >> 6, u = c & 63;
+        v[j] = __ldcg(reinterpret_cast<const float4 *>((u < 32 ? k_rows : v_rows) + (size_t)row * PK_D) + (u & 31));
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < PK_FETCH; ++j) {
+      const int c = base + j * PK_THREADS + threadIdx.x;
+      if (c < total) {
+        const int row = c >> 6, u = c & 63;
+        const uint32_t h0 = pack_bf16x2(v[j].x, v[j].y), h1 = pack_bf16x2(v[j].z, v[j].w);
+        const uint32_t l0 = pack_bf16x2(v[j].x - __uint_as_float(h0 << 16), v[j].y - __uint_as_float(h0 & 0xffff0000u));
+        const uint32_t l1 = pack_bf16x2(v[j].z - __uint_as_float(h1 << 16), v[j].w - __uint_as_float(h1 & 0xffff0000u));
+        const int off = u < 32 ? row * PK_KROW + u * 8 : row * PK_VROW + (u - 32) * 8;
+        *reinterpret_cast<uint2 *>(sc + (u < 32 ? PK_AT_KH : PK_AT_VH) + off) = make_uint2(h0, h1);
+        *reinterpret_cast<uint2 *>(sc + (u < 32 ? PK_AT_KL : PK_AT_VL) + off) = make_uint2(l0, l1);
+      }
     }
   }
 }
@@ -101,6 +174,7 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
 // shared memory, each warp taking 16 keys of a 64-key tile with its own running max and sum.
 // The slice's unnormalised partial output goes to global memory with its max and sum; the
 // prologue of the O projection merges the slices.
+template <bool PRECISE>
 __device__ __noinline__ void attention_stage(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
   const PassShared S = pass_shared();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -111,10 +185,20 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
   if ((int)blockIdx.x >= items) return;
 
   unsigned char *const sc = S.bstage;
-  const uint32_t k_tile = smem_u32(sc + PK_AT_K), v_tile = smem_u32(sc + PK_AT_V), q_tile = smem_u32(sc + PK_AT_Q);
+  const uint32_t kh_tile = smem_u32(sc + PK_AT_KH), kl_tile = smem_u32(sc + PK_AT_KL);
+  const uint32_t vh_tile = smem_u32(sc + PK_AT_VH), vl_tile = smem_u32(sc + PK_AT_VL);
+  const uint32_t qh_tile = smem_u32(sc + PK_AT_QH), ql_tile = smem_u32(sc + PK_AT_QL);
   float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
   float *const red_m = reinterpret_cast<float *>(sc + PK_AT_RED);
   float *const red_l = red_m + PK_WARPS * PK_QR;
+  // a 16-byte part (8 values) of a tile row: parts 0..15 are K, 16..31 are V
+  auto put_part = [&](int row, int part, const float (&f)[8]) {
+    uint4 hi, lo;
+    split8<PRECISE>(f, hi, lo);
+    const uint32_t off = part < 16 ? row * PK_KROW + part * 16 : row * PK_VROW + (part - 16) * 16;
+    sts128((part < 16 ? kh_tile : vh_tile) + off, hi);
+    if (PRECISE) sts128((part < 16 ? kl_tile : vl_tile) + off, lo);
+  };
 
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
     const int split = item % nsplit, kvh = (item / nsplit) % P.nkv, b = item / (nsplit * P.nkv);
@@ -122,15 +206,22 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     const int j0 = split * CH, j1 = min(j0 + CH, pos0);
     const int n_cached = max(0, j1 - j0);
     const int n_keys = n_cached + (split == nsplit - 1 ? R : 0);
-    const __nv_bfloat16 *kbase = Ly.kc + ((size_t)b * P.nkv + kvh) * P.max_seq * PK_D;
-    const __nv_bfloat16 *vbase = Ly.vc + ((size_t)b * P.nkv + kvh) * P.max_seq * PK_D;
-    // cached rows of a tile: asynchronous copies, 16 bytes each (a row is 16 K parts and 16 V parts)
+    const size_t head_off = ((size_t)b * P.nkv + kvh) * P.max_seq * PK_D;
+    // cached rows of a tile
     auto fetch_cached = [&](int tile0) {
       const int n_c = min(PK_TK, n_cached - tile0);
-      for (int c = threadIdx.x; c < n_c * 32; c += PK_THREADS) {
-        const int row = c >> 5, part = c & 31;
-        const uint32_t dst = part < 16 ? k_tile + row * PK_KROW + part * 16 : v_tile + row * PK_VROW + (part - 16) * 16;
-        cp_async16(dst, (part < 16 ? kbase : vbase) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
+      if (!PRECISE) {
+        // bf16 cache: asynchronous copies, 16 bytes each
+        const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(Ly.kc) + head_off;
+        const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(Ly.vc) + head_off;
+        for (int c = threadIdx.x; c < n_c * 32; c += PK_THREADS) {
+          const int row = c >> 5, part = c & 31;
+          const uint32_t dst = part < 16 ? kh_tile + row * PK_KROW + part * 16 : vh_tile + row * PK_VROW + (part - 16) * 16;
+          cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
+        }
+      } else {
+        attn_fetch_f32(reinterpret_cast<const float *>(Ly.kc) + head_off + (size_t)(j0 + tile0) * PK_D,
+                       reinterpret_cast<const float *>(Ly.vc) + head_off + (size_t)(j0 + tile0) * PK_D, n_c, sc);
       }
     };
     pk_sync();                                            // the previous item is done with the scratch
@@ -146,37 +237,40 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
         stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
       }
     }
-    fetch_cached(0);                                      // in flight while the pass's own rows are prepared
-    // query rows beyond nQ are zero (the previous item's partial outputs lay over the Q tile)
-    for (int i = threadIdx.x; i < PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(q_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
+    fetch_cached(0);                                      // in flight while the pass's own rows arrive
+    // query rows beyond nQ are zero (the previous item's partial outputs lay over the Q tiles)
+    for (int i = threadIdx.x; i < 2 * PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(qh_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
     stage_wait(P, S);
-    attn_new_rows(P, Ly, sc, b, kvh, R, pos0, split == 0);
+    attn_new_rows<PRECISE>(P, Ly, sc, b, kvh, R, pos0, split == 0);
 
     float m_run[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};
     float o[16][4];
 #pragma unroll
     for (int dt = 0; dt < 16; ++dt) o[dt][0] = o[dt][1] = o[dt][2] = o[dt][3] = 0.f;
-    uint4 qf[4][2];
+    uint4 qh[4][2];
     for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
       const int n_t = min(PK_TK, n_keys - tile0);
       pk_sync();                                          // new rows written / previous tile consumed
       if (tile0 > 0) fetch_cached(tile0);
       for (int c = threadIdx.x + max(0, n_cached - tile0) * 32; c < n_t * 32; c += PK_THREADS) {
-        const int row = c >> 5, part = c & 31, idx = tile0 + row;
-        const uint32_t dst = part < 16 ? k_tile + row * PK_KROW + part * 16 : v_tile + row * PK_VROW + (part - 16) * 16;
-        const unsigned char *src = sc + PK_AT_NEW + ((part < 16 ? 0 : PK_MAX_ROWS) + (idx - n_cached)) * 256 + (part & 15) * 16;
-        sts128(dst, *reinterpret_cast<const uint4 *>(src));
+        const int row = c >> 5, part = c & 31, r = tile0 + row - n_cached;
+        const float *src = reinterpret_cast<const float *>(sc + PK_AT_NEW) + ((part < 16 ? 0 : PK_MAX_ROWS) + r) * PK_D + (part & 15) * 8;
+        const float f[8] = {src[0], src[1], src[2], src[3], src[4], src[5], src[6], src[7]};
+        put_part(row, part, f);
       }
       const int n16 = min(PK_TK, (n_t + 15) & ~15);
-      for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS)      // P = 0 times stale bits must stay 0
-        sts128(v_tile + (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16, make_uint4(0u, 0u, 0u, 0u));
+      for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS) {    // P = 0 times stale bits must stay 0
+        const uint32_t off = (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16;
+        sts128(vh_tile + off, make_uint4(0u, 0u, 0u, 0u));
+        if (PRECISE) sts128(vl_tile + off, make_uint4(0u, 0u, 0u, 0u));
+      }
       cp_async_wait_all();
       pk_sync();
       if (tile0 == 0) {
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
-          qf[kb][0] = lds128(q_tile + g * PK_QROW + kb * 64 + t * 16);
-          qf[kb][1] = lds128(q_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
+          qh[kb][0] = lds128(qh_tile + g * PK_QROW + kb * 64 + t * 16);
+          qh[kb][1] = lds128(qh_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
         }
       }
       if (warp * 16 < n_t) {
@@ -186,9 +280,20 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
           c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
 #pragma unroll
           for (int kb = 0; kb < 4; ++kb) {
-            const uint4 Kv = lds128(k_tile + (warp * 16 + nt * 8 + g) * PK_KROW + kb * 64 + t * 16);
-            mma_bf16_16816(c[nt], qf[kb][0].x, qf[kb][1].x, qf[kb][0].y, qf[kb][1].y, Kv.x, Kv.y);
-            mma_bf16_16816(c[nt], qf[kb][0].z, qf[kb][1].z, qf[kb][0].w, qf[kb][1].w, Kv.z, Kv.w);
+            const uint32_t off = (warp * 16 + nt * 8 + g) * PK_KROW + kb * 64 + t * 16;
+            const uint4 Kh = lds128(kh_tile + off);
+            mma_bf16_16816(c[nt], qh[kb][0].x, qh[kb][1].x, qh[kb][0].y, qh[kb][1].y, Kh.x, Kh.y);
+            mma_bf16_16816(c[nt], qh[kb][0].z, qh[kb][1].z, qh[kb][0].w, qh[kb][1].w, Kh.z, Kh.w);
+            if (PRECISE) {
+              // the lo parts of Q stay in shared memory: registers are short here
+              const uint4 Kl = lds128(kl_tile + off);
+              const uint4 q0 = lds128(ql_tile + g * PK_QROW + kb * 64 + t * 16);
+              const uint4 q1 = lds128(ql_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
+              mma_bf16_16816(c[nt], qh[kb][0].x, qh[kb][1].x, qh[kb][0].y, qh[kb][1].y, Kl.x, Kl.y);
+              mma_bf16_16816(c[nt], qh[kb][0].z, qh[kb][1].z, qh[kb][0].w, qh[kb][1].w, Kl.z, Kl.w);
+              mma_bf16_16816(c[nt], q0.x, q1.x, q0.y, q1.y, Kh.x, Kh.y);
+              mma_bf16_16816(c[nt], q0.z, q1.z, q0.w, q1.w, Kh.z, Kh.w);
+            }
           }
         }
         // causal / range mask: lane holds rows g (e = 0, 1) and g + 8 (e = 2, 3), keys 2t, 2t + 1 of each n-tile
@@ -225,18 +330,31 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
         }
         l_part[0] = l_part[0] * corr[0] + psum[0];
         l_part[1] = l_part[1] * corr[1] + psum[1];
-        const uint32_t a0 = pack_bf16x2(c[0][0], c[0][1]), a1 = pack_bf16x2(c[0][2], c[0][3]);
-        const uint32_t a2 = pack_bf16x2(c[1][0], c[1][1]), a3 = pack_bf16x2(c[1][2], c[1][3]);
+        // P as the A operand: hi parts and (fp32 cache) lo parts
+        uint32_t ah[4], al[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float p0 = c[i >> 1][(i & 1) * 2], p1 = c[i >> 1][(i & 1) * 2 + 1];
+          ah[i] = pack_bf16x2(p0, p1);
+          if (PRECISE) al[i] = pack_bf16x2(p0 - __uint_as_float(ah[i] << 16), p1 - __uint_as_float(ah[i] & 0xffff0000u));
+        }
         const int mi = lane >> 3, rr = lane & 7;
-        const uint32_t v_addr = v_tile + (warp * 16 + (mi & 1) * 8 + rr) * PK_VROW + (mi >> 1) * 16;
+        const uint32_t v_off = (warp * 16 + (mi & 1) * 8 + rr) * PK_VROW + (mi >> 1) * 16;
 #pragma unroll
         for (int d2 = 0; d2 < 8; ++d2) {
           uint32_t b0, b1, b2, b3;
-          ldmatrix_x4_trans(v_addr + d2 * 32, b0, b1, b2, b3);
+          ldmatrix_x4_trans(vh_tile + v_off + d2 * 32, b0, b1, b2, b3);
           o[2 * d2][0] *= corr[0]; o[2 * d2][1] *= corr[0]; o[2 * d2][2] *= corr[1]; o[2 * d2][3] *= corr[1];
           o[2 * d2 + 1][0] *= corr[0]; o[2 * d2 + 1][1] *= corr[0]; o[2 * d2 + 1][2] *= corr[1]; o[2 * d2 + 1][3] *= corr[1];
-          mma_bf16_16816(o[2 * d2], a0, a1, a2, a3, b0, b1);
-          mma_bf16_16816(o[2 * d2 + 1], a0, a1, a2, a3, b2, b3);
+          mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
+          mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+          if (PRECISE) {
+            mma_bf16_16816(o[2 * d2], al[0], al[1], al[2], al[3], b0, b1);
+            mma_bf16_16816(o[2 * d2 + 1], al[0], al[1], al[2], al[3], b2, b3);
+            ldmatrix_x4_trans(vl_tile + v_off + d2 * 32, b0, b1, b2, b3);
+            mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
+            mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+          }
         }
       }
     }
@@ -291,7 +409,6 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
       const size_t slot = ((size_t)(b * R + qi / G) * P.nq + kvh * G + qi % G) * PK_NSPLIT_CAP + split;
       *reinterpret_cast<float4 *>(P.part_o + slot * PK_D + d4 * 4) = acc;
     }
-
   }
   pk_sync();
 }

@@ -33,6 +33,7 @@ constexpr int PK_MAX_LAYERS = 40;
 constexpr int PK_NSPLIT_CAP = 16;                          // key slices per (sequence, kv head)
 constexpr int PK_D = 128;                                  // head_dim
 constexpr int PK_QR = 16;                                  // query rows per attention item
+constexpr int PK_MAX_GROUP = 8;                            // query heads per kv head
 constexpr int PK_XS_FLOATS = 20480;                        // activation staging area, floats
 
 // shared memory map (bytes)
@@ -53,7 +54,7 @@ enum { PK_ERR_NONE = 0, PK_ERR_TOKEN = 1, PK_ERR_COPY_WAIT = 2, PK_ERR_BARRIER_W
 struct PassLayer {
   PackedMat qkv, o, gu, down;
   const float *w_in, *w_post, *w_qn, *w_kn;
-  __nv_bfloat16 *kc, *vc;                 // this layer's cache [sequence][kv head][max_seq][128]
+  void *kc, *vc;                          // this layer's cache [sequence][kv head][max_seq][128], bf16 or fp32
 };
 
 struct PassParams {
@@ -66,6 +67,7 @@ struct PassParams {
   int H, I, nq, nkv, vocab, max_seq, ldl;
   float eps;
   int kind;                               // 1 full pass, 2 decoding layers only (counter update)
+  int kv_f32;                             // the KV cache holds fp32 (else bf16)
   int write_token;
   int *tokens;
   DevState *st;
@@ -80,7 +82,10 @@ struct PassParams {
 };
 
 constexpr int PK_SMEM_BYTES = PK_OFF_LAYERS + PK_MAX_LAYERS * (int)sizeof(PassLayer);
-static_assert(PK_SMEM_BYTES <= 227 * 1024, "shared memory map too large");
+// 196 KiB is a shared-memory configuration of the SM; one byte more selects the 228 KiB one and
+// leaves 28 KiB of L1, which the register spills of the prologues then thrash (measured: the merge
+// prologue went from 2.6 to 9.8 us)
+static_assert(PK_SMEM_BYTES <= 196 * 1024, "shared memory map too large");
 
 // ---------------------------------------------------------------------------- PTX wrappers
 

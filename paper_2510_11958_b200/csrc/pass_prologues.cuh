@@ -8,6 +8,7 @@
 
 namespace dmtd {
 
+constexpr int PK_MERGE_BATCH = 8;    // partial outputs (float4 per lane) in flight per warp in the merge
 constexpr int PK_SPAN_UNITS = 3;     // float4 units of a block's k-slab span per thread: span <= 3072 values
 
 // Inputs of a prologue come into shared memory as bulk copies issued by one thread: no load
@@ -118,20 +119,25 @@ __device__ __noinline__ void merge_prologue(const PassParams &P, int M, int nspl
     const int m = pair / n_heads, hh = pair - m * n_heads;
     const int sl = hh / heads_per_slab, h = sp.first * heads_per_slab + hh;
     const size_t slot0 = ((size_t)m * P.nq + h) * PK_NSPLIT_CAP;
-    float4 po[PK_NSPLIT_CAP];
-#pragma unroll
-    for (int s = 0; s < PK_NSPLIT_CAP; ++s)
-      if (s < nsplit) po[s] = __ldcg(reinterpret_cast<const float4 *>(P.part_o + (slot0 + s) * PK_D) + lane);
     float2 ml = make_float2(-INFINITY, 0.f);
     if (lane < nsplit) ml = __ldcg(reinterpret_cast<const float2 *>(P.part_ml) + slot0 + lane);
-    const float mxx = warp_max(ml.y > 0.f ? ml.x : -INFINITY);
-    float wgt = ml.y > 0.f ? __expf(ml.x - mxx) : 0.f;
-    wgt /= warp_sum(wgt * ml.y);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float wgt = 0.f;
+    for (int s0 = 0; s0 < nsplit; s0 += PK_MERGE_BATCH) {
+      float4 po[PK_MERGE_BATCH];
 #pragma unroll
-    for (int s = 0; s < PK_NSPLIT_CAP; ++s) {
-      const float w = __shfl_sync(0xffffffffu, wgt, s);
-      if (s < nsplit) { acc.x += w * po[s].x; acc.y += w * po[s].y; acc.z += w * po[s].z; acc.w += w * po[s].w; }
+      for (int s = 0; s < PK_MERGE_BATCH; ++s)
+        if (s0 + s < nsplit) po[s] = __ldcg(reinterpret_cast<const float4 *>(P.part_o + (slot0 + s0 + s) * PK_D) + lane);
+      if (s0 == 0) {
+        const float mxx = warp_max(ml.y > 0.f ? ml.x : -INFINITY);
+        wgt = ml.y > 0.f ? __expf(ml.x - mxx) : 0.f;
+        wgt /= warp_sum(wgt * ml.y);
+      }
+#pragma unroll
+      for (int s = 0; s < PK_MERGE_BATCH; ++s) {
+        const float w = __shfl_sync(0xffffffffu, wgt, (s0 + s) & 31);
+        if (s0 + s < nsplit) { acc.x += w * po[s].x; acc.y += w * po[s].y; acc.z += w * po[s].z; acc.w += w * po[s].w; }
+      }
     }
     store_act4(S.bstage + (size_t)sl * 8 * sp.row_bytes, sp.row_bytes, m, (hh - sl * heads_per_slab) * PK_D + lane * 4, acc);
   }

@@ -38,6 +38,7 @@ def main():
     ap.add_argument("--workload", default="qwen3_4b_b1")
     ap.add_argument("--kind", default="full", choices=["full", "upper"])
     ap.add_argument("--ghz", type=float, default=1.965)
+    ap.add_argument("--kv", default=None, choices=["bf16", "f32"], help="KV cache type (default: the workload's)")
     ap.add_argument("--build-only", action="store_true")
     args = ap.parse_args()
     build_timing_library()
@@ -51,7 +52,8 @@ def main():
     wl = WORKLOADS[args.workload]
     shape = SHAPES[wl.shape]
     w = make_weights(shape, seed=wl.weight_seed, device="cuda")
-    eng = bd.Dmtd(shape, w, L_d=wl.L_d, tau=wl.tau, max_batch=wl.batch, max_seq=wl.prompt_len + 64)
+    eng = bd.Dmtd(shape, w, L_d=wl.L_d, tau=wl.tau, max_batch=wl.batch, max_seq=wl.prompt_len + 64,
+                  kv_dtype=args.kv or wl.kv_dtype)
     del w
     eng.prefill(make_prompts(shape.vocab, wl.batch, wl.prompt_len, seed=wl.prompt_seed).cuda())
     for _ in range(4):
@@ -63,7 +65,7 @@ def main():
     eng.decode_cycle(1)
     ev[1].record()
     torch.cuda.synchronize()
-    print(f"{args.workload}, {args.kind} pass: {ev[0].elapsed_time(ev[1]) * 1e3:.1f} us by CUDA events")
+    print(f"{args.workload}, KV {args.kv or wl.kv_dtype}, {args.kind} pass: {ev[0].elapsed_time(ev[1]) * 1e3:.1f} us by CUDA events")
     buf = np.zeros(2 * SLOTS, np.int64)
     eng.dll.dmtd_debug_pass_timing.argtypes = [C.c_void_p, C.c_void_p]
     assert eng.dll.dmtd_debug_pass_timing(eng._ctx, buf.ctypes.data_as(C.c_void_p)) == 0

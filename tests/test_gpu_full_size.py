@@ -1,0 +1,45 @@
+"""Parity at the full matrix sizes of the benchmark workload (Qwen3-4B shape, batch 1, tau = 3,
+last 8 layers decoding), through the launch configuration `bench.py` times: the persistent pass
+kernel.  The oracle needs about a quarter of a second per token row of the 36-layer model, so the
+full-depth case keeps the prompt short, and the case at the benchmark's context length (512-token
+prompt, several key slices per head) keeps two layers of the same geometry.  The KV cache is fp32
+as in the benchmark workload: a bf16 cache alone moves these logits by up to 0.05."""
+import numpy as np
+import pytest
+import torch
+
+from synthetic import SHAPES, make_prompts, make_weights
+
+from helpers import check_logits, gpu_forced, oracle_forced, to_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(shape, L_d, tau, P, n_new, seed):
+    import paper_2510_11958_b200 as pkg
+    w = make_weights(shape, seed=seed)
+    prompts = make_prompts(shape.vocab, 1, P, seed=1).numpy()
+    forced = make_prompts(shape.vocab, 1, n_new, seed=2).numpy()
+    ref_logits, ref_am, o = oracle_forced(shape, w, L_d, tau, prompts, forced)
+    wc = to_cuda(w)
+    del w
+    eng = pkg.Dmtd(shape, wc, L_d=L_d, tau=tau, max_batch=1, max_seq=P + n_new + 1, kv_dtype="f32")
+    del wc
+    l0 = eng.launch_count()
+    got_logits, got_am = gpu_forced(eng, prompts, forced)
+    err, clear = check_logits(got_logits, ref_logits, got_am, ref_am)
+    assert eng.device_state() == o.state()
+    return err, clear, eng
+
+
+def test_full_depth_qwen3_4b_short_prompt():
+    """All 36 layers, full vocabulary: two whole cycles after the prefill's."""
+    err, clear, eng = _run(SHAPES["qwen3_4b"], 8, 3, 40, 9, seed=0)
+    print(f"full depth: max|dlogit|={err:.2e}, clear-margin steps {clear:.0%}")
+
+
+def test_two_layers_qwen3_4b_geometry_benchmark_context():
+    """Layer and head matrices of the 4B shape at the benchmark's context length."""
+    shape = SHAPES["qwen3_4b"].with_(n_layers=2)
+    err, clear, eng = _run(shape, 1, 3, 512, 10, seed=3)
+    print(f"two layers, P=512: max|dlogit|={err:.2e}, clear-margin steps {clear:.0%}")

@@ -311,17 +311,20 @@ def test_fused_pass_kernel_free_running(dmtd):
 
 
 FUSED_CASES = [
-    # name, L_d, tau, B, P, n_new
-    ("b1_tau3", 2, 3, 1, 37, 13),
-    ("b1_tau4_long_prompt", 2, 4, 1, 300, 9),     # several key slices per kv head, two key tiles
-    ("b2_tau2", 4, 2, 2, 9, 8),
-    ("b4_tau1", 2, 1, 4, 12, 5),
-    ("b1_tau3_all_layers_decode", 6, 3, 1, 11, 7),
+    # name, L_d, tau, B, P, n_new, kv cache type
+    ("b1_tau3", 2, 3, 1, 37, 13, "bf16"),
+    ("b1_tau4_long_prompt", 2, 4, 1, 300, 9, "bf16"),     # several key slices per kv head
+    ("b2_tau2", 4, 2, 2, 9, 8, "bf16"),
+    ("b4_tau1", 2, 1, 4, 12, 5, "bf16"),
+    ("b1_tau3_all_layers_decode", 6, 3, 1, 11, 7, "bf16"),
+    ("b1_tau3_f32kv", 2, 3, 1, 37, 13, "f32"),
+    ("b1_tau4_long_prompt_f32kv", 2, 4, 1, 1300, 9, "f32"),    # two key tiles per slice
+    ("b2_tau2_f32kv", 4, 2, 2, 9, 8, "f32"),
 ]
 
 
-@pytest.mark.parametrize("name,L_d,tau,B,P,n_new", FUSED_CASES, ids=[c[0] for c in FUSED_CASES])
-def test_fused_pass_kernel_teacher_forced(dmtd, name, L_d, tau, B, P, n_new):
+@pytest.mark.parametrize("name,L_d,tau,B,P,n_new,kv", FUSED_CASES, ids=[c[0] for c in FUSED_CASES])
+def test_fused_pass_kernel_teacher_forced(dmtd, name, L_d, tau, B, P, n_new, kv):
     """The one-kernel-per-pass path (at most 4 rows per pass) against the oracle, and against the
     per-step kernels on the same inputs."""
     shape = SHAPES["mid"]
@@ -332,12 +335,14 @@ def test_fused_pass_kernel_teacher_forced(dmtd, name, L_d, tau, B, P, n_new):
     wc = to_cuda(w)
     res = {}
     for fused in (1, 0):
-        eng = _engine(dmtd, shape, wc, L_d, tau, B, P + n_new + 1)
+        eng = _engine(dmtd, shape, wc, L_d, tau, B, P + n_new + 1, kv_dtype=kv)
         eng.set_option("fused_pass", fused)
         l0 = eng.launch_count()
         got_logits, got_am = gpu_forced(eng, prompts, toks)
         res[fused] = (got_logits, eng.launch_count() - l0)
-        check_logits(got_logits, ref_logits, got_am, ref_am)
+        err, _ = check_logits(got_logits, ref_logits, got_am, ref_am)
+        if kv == "f32":
+            assert err < 1e-3                  # nothing is rounded to bf16 but the weights
         assert eng.state() == o.state()
         assert eng.device_state() == o.state()
     # the fused path really ran: one launch per decode pass instead of dozens
