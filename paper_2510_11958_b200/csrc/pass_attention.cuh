@@ -138,142 +138,26 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
   }
 }
 
-// Cached rows of an fp32 tile: through registers, PK_FETCH float4 per thread in flight (one trip
-// for a slice of up to 40 keys), each split into bf16 hi and lo parts.  A function of its own so
-// that its registers are not counted against the attention loop's.
-__device__ __noinline__ void attn_fetch_f32(const float *k_rows, const float *v_rows, int n_rows, unsigned char *sc) {
-  const int total = n_rows * 64;                          // float4 units: 32 of K and 32 of V per row
-  for (int base = 0; base < total; base += PK_FETCH * PK_THREADS) {
-    float4 v[PK_FETCH];
-#pragma unroll
-    for (int j = 0; j < PK_FETCH; ++j) {
-      const int c = base + j * PK_THREADS + threadIdx.x;
-      if (c < total) {
-        const int row = c >> 6, u = c & 63;
-        v[j] = __ldcg(reinterpret_cast<const float4 *>((u < 32 ? k_rows : v_rows) + (size_t)row * PK_D) + (u & 31));
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < PK_FETCH; ++j) {
-      const int c = base + j * PK_THREADS + threadIdx.x;
-      if (c < total) {
-        const int row = c >> 6, u = c & 63;
-        const uint32_t h0 = pack_bf16x2(v[j].x, v[j].y), h1 = pack_bf16x2(v[j].z, v[j].w);
-        const uint32_t l0 = pack_bf16x2(v[j].x - __uint_as_float(h0 << 16), v[j].y - __uint_as_float(h0 & 0xffff0000u));
-        const uint32_t l1 = pack_bf16x2(v[j].z - __uint_as_float(h1 << 16), v[j].w - __uint_as_float(h1 & 0xffff0000u));
-        const int off = u < 32 ? row * PK_KROW + u * 8 : row * PK_VROW + (u - 32) * 8;
-        *reinterpret_cast<uint2 *>(sc + (u < 32 ? PK_AT_KH : PK_AT_VH) + off) = make_uint2(h0, h1);
-        *reinterpret_cast<uint2 *>(sc + (u < 32 ? PK_AT_KL : PK_AT_VL) + off) = make_uint2(l0, l1);
-      }
-    }
-  }
-}
+// One 64-key tile against the 16 query rows: this warp's 16 keys.  acc holds the warp's running
+// max, running sum (per lane, summed over the four lanes of a row at the end) and output.
+struct AttnAcc {
+  float m_run[2], l_part[2];
+  float o[16][4];
+};
 
-// Steps a3 + a4 for the items (sequence, kv head, key slice) of this block.  The R*G query rows
-// of an item form one m16 tile; S = Q K^T and O = P V run as mma.m16n8k16 with K and V staged in
-// shared memory, each warp taking 16 keys of a 64-key tile with its own running max and sum.
-// The slice's unnormalised partial output goes to global memory with its max and sum; the
-// prologue of the O projection merges the slices.
+// Keys of the tile are key_idx0 + row; key index i sits at position (i < n_cached ? j0 + i :
+// pos_new + i - n_cached); query row q may see positions up to row_pos0 + q / G.
 template <bool PRECISE>
-__device__ __noinline__ void attention_stage(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
-  const PassShared S = pass_shared();
+__device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc, const uint4 (&qh)[4][2], int n_t, int tile0,
+                                                  int n_cached, int j0, int pos_new, int row_pos0, int G) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-  const int G = P.nq / P.nkv, nQ = R * G;
-  int nsplit, CH;
-  attn_plan_device(P, pos0, nsplit, CH);
-  const int items = P.B * P.nkv * nsplit;
-  if ((int)blockIdx.x >= items) return;
-
-  unsigned char *const sc = S.bstage;
   const uint32_t kh_tile = smem_u32(sc + PK_AT_KH), kl_tile = smem_u32(sc + PK_AT_KL);
   const uint32_t vh_tile = smem_u32(sc + PK_AT_VH), vl_tile = smem_u32(sc + PK_AT_VL);
-  const uint32_t qh_tile = smem_u32(sc + PK_AT_QH), ql_tile = smem_u32(sc + PK_AT_QL);
-  float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
-  float *const red_m = reinterpret_cast<float *>(sc + PK_AT_RED);
-  float *const red_l = red_m + PK_WARPS * PK_QR;
-  // a 16-byte part (8 values) of a tile row: parts 0..15 are K, 16..31 are V
-  auto put_part = [&](int row, int part, const float (&f)[8]) {
-    uint4 hi, lo;
-    split8<PRECISE>(f, hi, lo);
-    const uint32_t off = part < 16 ? row * PK_KROW + part * 16 : row * PK_VROW + (part - 16) * 16;
-    sts128((part < 16 ? kh_tile : vh_tile) + off, hi);
-    if (PRECISE) sts128((part < 16 ? kl_tile : vl_tile) + off, lo);
-  };
-
-  for (int item = blockIdx.x; item < items; item += gridDim.x) {
-    const int split = item % nsplit, kvh = (item / nsplit) % P.nkv, b = item / (nsplit * P.nkv);
-    // keys [j0, j1) of the cache, then (last slice) the R keys of the pass
-    const int j0 = split * CH, j1 = min(j0 + CH, pos0);
-    const int n_cached = max(0, j1 - j0);
-    const int n_keys = n_cached + (split == nsplit - 1 ? R : 0);
-    const size_t head_off = ((size_t)b * P.nkv + kvh) * P.max_seq * PK_D;
-    // cached rows of a tile
-    auto fetch_cached = [&](int tile0) {
-      const int n_c = min(PK_TK, n_cached - tile0);
-      if (!PRECISE) {
-        // bf16 cache: asynchronous copies, 16 bytes each
-        const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(Ly.kc) + head_off;
-        const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(Ly.vc) + head_off;
-        for (int c = threadIdx.x; c < n_c * 32; c += PK_THREADS) {
-          const int row = c >> 5, part = c & 31;
-          const uint32_t dst = part < 16 ? kh_tile + row * PK_KROW + part * 16 : vh_tile + row * PK_VROW + (part - 16) * 16;
-          cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
-        }
-      } else {
-        attn_fetch_f32(reinterpret_cast<const float *>(Ly.kc) + head_off + (size_t)(j0 + tile0) * PK_D,
-                       reinterpret_cast<const float *>(Ly.vc) + head_off + (size_t)(j0 + tile0) * PK_D, n_c, sc);
-      }
-    };
-    pk_sync();                                            // the previous item is done with the scratch
-    if (threadIdx.x == 0) {
-      // the pass's own q | k | v vectors of this kv head: three bulk copies per row
-      const int ldq = (P.nq + 2 * P.nkv) * PK_D;
-      stage_begin(S, (uint32_t)(R * (G + 2) * PK_D * 4));
-      for (int r = 0; r < R; ++r) {
-        const float *src = P.qkv + (size_t)(b * R + r) * ldq;
-        float *dst = reinterpret_cast<float *>(sc + PK_AT_ROWS) + r * PK_AT_ROW_FLOATS;
-        stage_copy(S, dst, src + kvh * G * PK_D, (uint32_t)(G * PK_D * 4));
-        stage_copy(S, dst + G * PK_D, src + (P.nq + kvh) * PK_D, PK_D * 4);
-        stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
-      }
-    }
-    fetch_cached(0);                                      // in flight while the pass's own rows arrive
-    // query rows beyond nQ are zero (the previous item's partial outputs lay over the Q tiles)
-    for (int i = threadIdx.x; i < 2 * PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(qh_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
-    stage_wait(P, S);
-    attn_new_rows<PRECISE>(P, Ly, sc, b, kvh, R, pos0, split == 0);
-
-    float m_run[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};
-    float o[16][4];
-#pragma unroll
-    for (int dt = 0; dt < 16; ++dt) o[dt][0] = o[dt][1] = o[dt][2] = o[dt][3] = 0.f;
-    uint4 qh[4][2];
-    for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
-      const int n_t = min(PK_TK, n_keys - tile0);
-      pk_sync();                                          // new rows written / previous tile consumed
-      if (tile0 > 0) fetch_cached(tile0);
-      for (int c = threadIdx.x + max(0, n_cached - tile0) * 32; c < n_t * 32; c += PK_THREADS) {
-        const int row = c >> 5, part = c & 31, r = tile0 + row - n_cached;
-        const float *src = reinterpret_cast<const float *>(sc + PK_AT_NEW) + ((part < 16 ? 0 : PK_MAX_ROWS) + r) * PK_D + (part & 15) * 8;
-        const float f[8] = {src[0], src[1], src[2], src[3], src[4], src[5], src[6], src[7]};
-        put_part(row, part, f);
-      }
-      const int n16 = min(PK_TK, (n_t + 15) & ~15);
-      for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS) {    // P = 0 times stale bits must stay 0
-        const uint32_t off = (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16;
-        sts128(vh_tile + off, make_uint4(0u, 0u, 0u, 0u));
-        if (PRECISE) sts128(vl_tile + off, make_uint4(0u, 0u, 0u, 0u));
-      }
-      cp_async_wait_all();
-      pk_sync();
-      if (tile0 == 0) {
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          qh[kb][0] = lds128(qh_tile + g * PK_QROW + kb * 64 + t * 16);
-          qh[kb][1] = lds128(qh_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
-        }
-      }
-      if (warp * 16 < n_t) {
+  const uint32_t ql_tile = smem_u32(sc + PK_AT_QL);
+  float (&m_run)[2] = A.m_run;
+  float (&l_part)[2] = A.l_part;
+  float (&o)[16][4] = A.o;
+  if (warp * 16 < n_t) {
         float c[2][4];
 #pragma unroll
         for (int nt = 0; nt < 2; ++nt) {
@@ -303,8 +187,8 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int kl = warp * 16 + nt * 8 + 2 * t + (e & 1), idx = tile0 + kl, row = g + (e >> 1) * 8;
-            const int key_pos = idx < n_cached ? j0 + idx : pos0 + (idx - n_cached);
-            const bool ok = kl < n_t && key_pos <= pos0 + row / G;
+            const int key_pos = idx < n_cached ? j0 + idx : pos_new + (idx - n_cached);
+            const bool ok = kl < n_t && key_pos <= row_pos0 + row / G;
             c[nt][e] = ok ? c[nt][e] : -INFINITY;
             mx[e >> 1] = fmaxf(mx[e >> 1], c[nt][e]);
           }
@@ -357,58 +241,210 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
           }
         }
       }
+}
+
+// Combine the warps of the block into the slice's partial result: unnormalised output with its
+// max and sum, written to part_o / part_ml at slot (row0 + q / G, head0 + q % G, split), where a
+// (row, head) owns `slot_stride` consecutive slots.
+__device__ __forceinline__ void attn_combine_store(AttnAcc &A, unsigned char *sc, int nQ, int G, int row0, int head0, int nq,
+                                                   int slot_stride, int split, float *part_o, float *part_ml) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
+  float *const red_m = reinterpret_cast<float *>(sc + PK_AT_RED);
+  float *const red_l = red_m + PK_WARPS * PK_QR;
+  float (&m_run)[2] = A.m_run;
+  float (&l_part)[2] = A.l_part;
+  float (&o)[16][4] = A.o;
+  // combine the warps into this slice's partial result
+  pk_sync();                                            // tiles consumed: their space becomes o_s
+#pragma unroll
+  for (int hr = 0; hr < 2; ++hr) {
+    l_part[hr] += __shfl_xor_sync(0xffffffffu, l_part[hr], 1);
+    l_part[hr] += __shfl_xor_sync(0xffffffffu, l_part[hr], 2);
+    if (t == 0) { red_m[warp * PK_QR + g + 8 * hr] = m_run[hr]; red_l[warp * PK_QR + g + 8 * hr] = l_part[hr]; }
+  }
+  if (g < nQ) {
+#pragma unroll
+    for (int dt = 0; dt < 16; ++dt)
+      *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][0], o[dt][1]);
+  }
+  if (g + 8 < nQ) {
+#pragma unroll
+    for (int dt = 0; dt < 16; ++dt)
+      *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g + 8) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][2], o[dt][3]);
+  }
+  pk_sync();
+  // per query row: the slice's max and sum, and the factor each warp's share is scaled by
+  if ((int)threadIdx.x < nQ) {
+    const int qi = threadIdx.x;
+    float m = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < PK_WARPS; ++w) m = fmaxf(m, red_m[w * PK_QR + qi]);
+    float l = 0.f;
+#pragma unroll
+    for (int w = 0; w < PK_WARPS; ++w) {
+      const float mw = red_m[w * PK_QR + qi];
+      const float f = mw > -INFINITY ? __expf(mw - m) : 0.f;
+      l += red_l[w * PK_QR + qi] * f;
+      red_l[w * PK_QR + qi] = f;
+    }
+    const size_t slot = ((size_t)(row0 + qi / G) * nq + head0 + qi % G) * slot_stride + split;
+    part_ml[slot * 2] = m;
+    part_ml[slot * 2 + 1] = l;
+  }
+  pk_sync();
+  for (int idx = threadIdx.x; idx < nQ * (PK_D / 4); idx += PK_THREADS) {
+    const int qi = idx / (PK_D / 4), d4 = idx % (PK_D / 4);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int w = 0; w < PK_WARPS; ++w) {
+      const float f = red_l[w * PK_QR + qi];
+      const float4 v = *reinterpret_cast<const float4 *>(o_s + (w * PK_QR + qi) * PK_OROW + d4 * 4);
+      acc.x += v.x * f; acc.y += v.y * f; acc.z += v.z * f; acc.w += v.w * f;
+    }
+    const size_t slot = ((size_t)(row0 + qi / G) * nq + head0 + qi % G) * slot_stride + split;
+    *reinterpret_cast<float4 *>(part_o + slot * PK_D + d4 * 4) = acc;
+  }
+}
+
+// Cached rows of an fp32 tile: through registers, PK_FETCH float4 per thread in flight (one trip
+// for a slice of up to 40 keys), each split into bf16 hi and lo parts.  A function of its own so
+// that its registers are not counted against the attention loop's.
+__device__ __noinline__ void attn_fetch_f32(const float *k_rows, const float *v_rows, int n_rows, unsigned char *sc) {
+  const int total = n_rows * 64;                          // float4 units: 32 of K and 32 of V per row
+  for (int base = 0; base < total; base += PK_FETCH * PK_THREADS) {
+    float4 v[PK_FETCH];
+#pragma unroll
+    for (int j = 0; j < PK_FETCH; ++j) {
+      const int c = base + j * PK_THREADS + threadIdx.x;
+      if (c < total) {
+        const int row = c >> 6, u = c & 63;
+        v[j] = __ldcg(reinterpret_cast<const float4 *>((u < 32 ? k_rows : v_rows) + (size_t)row * PK_D) + (u & 31));
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < PK_FETCH; ++j) {
+      const int c = base + j * PK_THREADS + threadIdx.x;
+      if (c < total) {
+        const int row = c >> 6, u = c & 63;
+        const uint32_t h0 = pack_bf16x2(v[j].x, v[j].y), h1 = pack_bf16x2(v[j].z, v[j].w);
+        const uint32_t l0 = pack_bf16x2(v[j].x - __uint_as_float(h0 << 16), v[j].y - __uint_as_float(h0 & 0xffff0000u));
+        const uint32_t l1 = pack_bf16x2(v[j].z - __uint_as_float(h1 << 16), v[j].w - __uint_as_float(h1 & 0xffff0000u));
+        const int off = u < 32 ? row * PK_KROW + u * 8 : row * PK_VROW + (u - 32) * 8;
+        *reinterpret_cast<uint2 *>(sc + (u < 32 ? PK_AT_KH : PK_AT_VH) + off) = make_uint2(h0, h1);
+        *reinterpret_cast<uint2 *>(sc + (u < 32 ? PK_AT_KL : PK_AT_VL) + off) = make_uint2(l0, l1);
+      }
+    }
+  }
+}
+
+// Steps a3 + a4 for the items (sequence, kv head, key slice) of this block.  The R*G query rows
+// of an item form one m16 tile; S = Q K^T and O = P V run as mma.m16n8k16 with K and V staged in
+// shared memory, each warp taking 16 keys of a 64-key tile with its own running max and sum.
+// The slice's unnormalised partial output goes to global memory with its max and sum; the
+// prologue of the O projection merges the slices.
+template <bool PRECISE>
+__device__ __noinline__ void attention_stage(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
+  const PassShared S = pass_shared();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int G = P.nq / P.nkv, nQ = R * G;
+  int nsplit, CH;
+  attn_plan_device(P, pos0, nsplit, CH);
+  const int items = P.B * P.nkv * nsplit;
+  if ((int)blockIdx.x >= items) return;
+
+  unsigned char *const sc = S.bstage;
+  const uint32_t kh_tile = smem_u32(sc + PK_AT_KH), kl_tile = smem_u32(sc + PK_AT_KL);
+  const uint32_t vh_tile = smem_u32(sc + PK_AT_VH), vl_tile = smem_u32(sc + PK_AT_VL);
+  const uint32_t qh_tile = smem_u32(sc + PK_AT_QH), ql_tile = smem_u32(sc + PK_AT_QL);
+  // a 16-byte part (8 values) of a tile row: parts 0..15 are K, 16..31 are V
+  auto put_part = [&](int row, int part, const float (&f)[8]) {
+    uint4 hi, lo;
+    split8<PRECISE>(f, hi, lo);
+    const uint32_t off = part < 16 ? row * PK_KROW + part * 16 : row * PK_VROW + (part - 16) * 16;
+    sts128((part < 16 ? kh_tile : vh_tile) + off, hi);
+    if (PRECISE) sts128((part < 16 ? kl_tile : vl_tile) + off, lo);
+  };
+
+  for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    const int split = item % nsplit, kvh = (item / nsplit) % P.nkv, b = item / (nsplit * P.nkv);
+    // keys [j0, j1) of the cache, then (last slice) the R keys of the pass
+    const int j0 = split * CH, j1 = min(j0 + CH, pos0);
+    const int n_cached = max(0, j1 - j0);
+    const int n_keys = n_cached + (split == nsplit - 1 ? R : 0);
+    const size_t head_off = ((size_t)b * P.nkv + kvh) * P.max_seq * PK_D;
+    // cached rows of a tile
+    auto fetch_cached = [&](int tile0) {
+      const int n_c = min(PK_TK, n_cached - tile0);
+      if (!PRECISE) {
+        // bf16 cache: asynchronous copies, 16 bytes each
+        const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(Ly.kc) + head_off;
+        const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(Ly.vc) + head_off;
+        for (int c = threadIdx.x; c < n_c * 32; c += PK_THREADS) {
+          const int row = c >> 5, part = c & 31;
+          const uint32_t dst = part < 16 ? kh_tile + row * PK_KROW + part * 16 : vh_tile + row * PK_VROW + (part - 16) * 16;
+          cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
+        }
+      } else {
+        attn_fetch_f32(reinterpret_cast<const float *>(Ly.kc) + head_off + (size_t)(j0 + tile0) * PK_D,
+                       reinterpret_cast<const float *>(Ly.vc) + head_off + (size_t)(j0 + tile0) * PK_D, n_c, sc);
+      }
+    };
+    pk_sync();                                            // the previous item is done with the scratch
+    if (threadIdx.x == 0) {
+      // the pass's own q | k | v vectors of this kv head: three bulk copies per row
+      const int ldq = (P.nq + 2 * P.nkv) * PK_D;
+      stage_begin(S, (uint32_t)(R * (G + 2) * PK_D * 4));
+      for (int r = 0; r < R; ++r) {
+        const float *src = P.qkv + (size_t)(b * R + r) * ldq;
+        float *dst = reinterpret_cast<float *>(sc + PK_AT_ROWS) + r * PK_AT_ROW_FLOATS;
+        stage_copy(S, dst, src + kvh * G * PK_D, (uint32_t)(G * PK_D * 4));
+        stage_copy(S, dst + G * PK_D, src + (P.nq + kvh) * PK_D, PK_D * 4);
+        stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
+      }
+    }
+    fetch_cached(0);                                      // in flight while the pass's own rows arrive
+    // query rows beyond nQ are zero (the previous item's partial outputs lay over the Q tiles)
+    for (int i = threadIdx.x; i < 2 * PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(qh_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
+    stage_wait(P, S);
+    attn_new_rows<PRECISE>(P, Ly, sc, b, kvh, R, pos0, split == 0);
+
+    AttnAcc A;
+    A.m_run[0] = A.m_run[1] = -INFINITY;
+    A.l_part[0] = A.l_part[1] = 0.f;
+#pragma unroll
+    for (int dt = 0; dt < 16; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
+    uint4 qh[4][2];
+    for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
+      const int n_t = min(PK_TK, n_keys - tile0);
+      pk_sync();                                          // new rows written / previous tile consumed
+      if (tile0 > 0) fetch_cached(tile0);
+      for (int c = threadIdx.x + max(0, n_cached - tile0) * 32; c < n_t * 32; c += PK_THREADS) {
+        const int row = c >> 5, part = c & 31, r = tile0 + row - n_cached;
+        const float *src = reinterpret_cast<const float *>(sc + PK_AT_NEW) + ((part < 16 ? 0 : PK_MAX_ROWS) + r) * PK_D + (part & 15) * 8;
+        const float f[8] = {src[0], src[1], src[2], src[3], src[4], src[5], src[6], src[7]};
+        put_part(row, part, f);
+      }
+      const int n16 = min(PK_TK, (n_t + 15) & ~15);
+      for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS) {    // P = 0 times stale bits must stay 0
+        const uint32_t off = (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16;
+        sts128(vh_tile + off, make_uint4(0u, 0u, 0u, 0u));
+        if (PRECISE) sts128(vl_tile + off, make_uint4(0u, 0u, 0u, 0u));
+      }
+      cp_async_wait_all();
+      pk_sync();
+      if (tile0 == 0) {
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          qh[kb][0] = lds128(qh_tile + g * PK_QROW + kb * 64 + t * 16);
+          qh[kb][1] = lds128(qh_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
+        }
+      }
+      attn_tile_compute<PRECISE>(A, sc, qh, n_t, tile0, n_cached, j0, pos0, pos0, G);
     }
 
-    // combine the warps into this slice's partial result
-    pk_sync();                                            // tiles consumed: their space becomes o_s
-#pragma unroll
-    for (int hr = 0; hr < 2; ++hr) {
-      l_part[hr] += __shfl_xor_sync(0xffffffffu, l_part[hr], 1);
-      l_part[hr] += __shfl_xor_sync(0xffffffffu, l_part[hr], 2);
-      if (t == 0) { red_m[warp * PK_QR + g + 8 * hr] = m_run[hr]; red_l[warp * PK_QR + g + 8 * hr] = l_part[hr]; }
-    }
-    if (g < nQ) {
-#pragma unroll
-      for (int dt = 0; dt < 16; ++dt)
-        *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][0], o[dt][1]);
-    }
-    if (g + 8 < nQ) {
-#pragma unroll
-      for (int dt = 0; dt < 16; ++dt)
-        *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g + 8) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][2], o[dt][3]);
-    }
-    pk_sync();
-    // per query row: the slice's max and sum, and the factor each warp's share is scaled by
-    if ((int)threadIdx.x < nQ) {
-      const int qi = threadIdx.x;
-      float m = -INFINITY;
-#pragma unroll
-      for (int w = 0; w < PK_WARPS; ++w) m = fmaxf(m, red_m[w * PK_QR + qi]);
-      float l = 0.f;
-#pragma unroll
-      for (int w = 0; w < PK_WARPS; ++w) {
-        const float mw = red_m[w * PK_QR + qi];
-        const float f = mw > -INFINITY ? __expf(mw - m) : 0.f;
-        l += red_l[w * PK_QR + qi] * f;
-        red_l[w * PK_QR + qi] = f;
-      }
-      const size_t slot = ((size_t)(b * R + qi / G) * P.nq + kvh * G + qi % G) * PK_NSPLIT_CAP + split;
-      P.part_ml[slot * 2] = m;
-      P.part_ml[slot * 2 + 1] = l;
-    }
-    pk_sync();
-    for (int idx = threadIdx.x; idx < nQ * (PK_D / 4); idx += PK_THREADS) {
-      const int qi = idx / (PK_D / 4), d4 = idx % (PK_D / 4);
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int w = 0; w < PK_WARPS; ++w) {
-        const float f = red_l[w * PK_QR + qi];
-        const float4 v = *reinterpret_cast<const float4 *>(o_s + (w * PK_QR + qi) * PK_OROW + d4 * 4);
-        acc.x += v.x * f; acc.y += v.y * f; acc.z += v.z * f; acc.w += v.w * f;
-      }
-      const size_t slot = ((size_t)(b * R + qi / G) * P.nq + kvh * G + qi % G) * PK_NSPLIT_CAP + split;
-      *reinterpret_cast<float4 *>(P.part_o + slot * PK_D + d4 * 4) = acc;
-    }
+
+    attn_combine_store(A, sc, nQ, G, b * R, kvh * G, P.nq, PK_NSPLIT_CAP, split, P.part_o, P.part_ml);
   }
   pk_sync();
 }
