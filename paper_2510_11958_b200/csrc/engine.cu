@@ -11,11 +11,13 @@
 #include <mutex>
 #include <numeric>
 #include <string>
+#include <type_traits>
 #include <vector>
 
 #include "../../include/dmtd.h"
 #include "kernels.cuh"
 #include "pass_kernel.cuh"
+#include "attention_kernel.cuh"
 
 using namespace dmtd;
 
@@ -61,7 +63,7 @@ struct dmtd_ctx {
   float2 *rope_tab = nullptr;
 
   // options
-  bool use_graph = true, literal_sum = false, use_fused = true;
+  bool use_graph = true, literal_sum = false, use_fused = true, use_tc_attention = true;
 
   // fused pass kernel: one persistent launch per pass
   bool fused_ok = false;
@@ -230,6 +232,17 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
       c->max_seq);
   LAUNCH_OK(c, "qk_norm_rope_append_kernel");
   int RB = std::max(1, ATTN_QR / G), n_rb = (R + RB - 1) / RB;
+  if (D == PK_D && c->use_tc_attention) {
+    // tensor-core kernel (head_dim 128): hi+lo operands with an fp32 cache, plain bf16 otherwise
+    constexpr bool kPrecise = std::is_same<KVT, float>::value;
+    static bool tc_configured = false;
+    if (!tc_configured) {
+      CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<kPrecise>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM));
+      tc_configured = true;
+    }
+    attn_tc_kernel<kPrecise><<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
+        c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
+  } else {
   size_t smem = (size_t)ATTN_WARPS * ATTN_QR * D * sizeof(float);
   static bool configured = false;
   if (!configured) {
@@ -239,6 +252,7 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
   attn_partial_kernel<D, KVT><<<dim3(nsplit, s.n_kv_heads * n_rb, B), ATTN_WARPS * 32, smem, c->stream>>>(
       c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml,
       nsplit);
+  }
   LAUNCH_OK(c, "attn_partial_kernel");
   int n_rh = M * s.n_q_heads;
   attn_merge_kernel<D><<<(n_rh + 3) / 4, 128, 0, c->stream>>>(c->part_o, c->part_ml, nsplit, n_rh, s.n_q_heads,
@@ -799,6 +813,7 @@ dmtd_status dmtd_set_option(dmtd_ctx *c, const char *name, int64_t value) {
   if (!strcmp(name, "cuda_graph")) { c->use_graph = value != 0; return DMTD_OK; }
   if (!strcmp(name, "literal_sum")) { c->literal_sum = value != 0; drop_graphs(c); return DMTD_OK; }
   if (!strcmp(name, "fused_pass")) { c->use_fused = value != 0; return DMTD_OK; }
+  if (!strcmp(name, "tc_attention")) { c->use_tc_attention = value != 0; drop_graphs(c); return DMTD_OK; }
   return fail(c, DMTD_ERR_INVALID_ARG, "unknown option %s", name);
 }
 
@@ -873,12 +888,21 @@ dmtd_status attention_launch_t(const float *q, const void *k, const void *v, int
   float *part_o = reinterpret_cast<float *>(scratch + p.o_off);
   const int G = nq / nkv, RB = std::max(1, ATTN_QR / G), n_rb = (R + RB - 1) / RB, ld = nq * D;
   set_int_kernel<<<1, 1, 0, stream>>>(pos_dev, pos0);
-  size_t smem = (size_t)ATTN_WARPS * ATTN_QR * D * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel<D, KVT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-  if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention: %s", cudaGetErrorString(e));
-  attn_partial_kernel<D, KVT><<<dim3(p.nsplit, nkv * n_rb, B), ATTN_WARPS * 32, smem, stream>>>(
-      q, ld, static_cast<const KVT *>(k), static_cast<const KVT *>(v), max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o,
-      part_ml, p.nsplit);
+  cudaError_t e;
+  if (D == PK_D) {
+    constexpr bool kPrecise = std::is_same<KVT, float>::value;
+    e = cudaFuncSetAttribute(attn_tc_kernel<kPrecise>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM);
+    if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention: %s", cudaGetErrorString(e));
+    attn_tc_kernel<kPrecise><<<dim3(p.nsplit, nkv * n_rb, B), PK_THREADS, ATTN_TC_SMEM, stream>>>(
+        q, ld, k, v, max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o, part_ml, p.nsplit);
+  } else {
+    size_t smem = (size_t)ATTN_WARPS * ATTN_QR * D * sizeof(float);
+    e = cudaFuncSetAttribute(attn_partial_kernel<D, KVT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention: %s", cudaGetErrorString(e));
+    attn_partial_kernel<D, KVT><<<dim3(p.nsplit, nkv * n_rb, B), ATTN_WARPS * 32, smem, stream>>>(
+        q, ld, static_cast<const KVT *>(k), static_cast<const KVT *>(v), max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o,
+        part_ml, p.nsplit);
+  }
   int n_rh = B * R * nq;
   attn_merge_kernel<D><<<(n_rh + 3) / 4, 128, 0, stream>>>(part_o, part_ml, p.nsplit, n_rh, nq, out, ld);
   e = cudaGetLastError();
