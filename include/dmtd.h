@@ -200,6 +200,10 @@ dmtd_status dmtd_set_tau(dmtd_ctx *ctx, int32_t tau);
  *   "fused_pass"   0/1  run each decode pass as one persistent kernel where the model and batch
  *                       allow it (bf16 weights and KV, head_dim 128, at most 4 rows per pass);
  *                       0 = always the per-step kernels (default 1)
+ *   "tc_attention" 0/1  attention of the per-step kernels on the tensor cores (head_dim 128; default 1)
+ *   "tcgen05_gemm" 0/1  projections of more than 8 rows on the tcgen05 tensor cores; only contexts
+ *                       created with max_batch * tau > 8 hold the second weight copy it reads
+ *                       (default 1)
  * Errors: INVALID_ARG for an unknown name or value. */
 dmtd_status dmtd_set_option(dmtd_ctx *ctx, const char *name, int64_t value);
 

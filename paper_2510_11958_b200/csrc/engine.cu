@@ -18,6 +18,7 @@
 #include "kernels.cuh"
 #include "pass_kernel.cuh"
 #include "attention_kernel.cuh"
+#include "gemm_tc05.cuh"
 
 using namespace dmtd;
 
@@ -27,6 +28,7 @@ thread_local std::string g_create_error;
 
 struct LayerDev {
   PackedMat qkv, o, gu, down;
+  UmmaMat qkv_u{}, o_u{}, gu_u{}, down_u{};     // second copy for the tcgen05 GEMM (contexts with many rows)
   float *w_in, *w_post, *w_qn, *w_kn;
 };
 
@@ -44,6 +46,9 @@ struct dmtd_ctx {
   // model
   std::vector<LayerDev> layers;
   PackedMat embed{};
+  UmmaMat embed_u{};
+  bool umma_ok = false, use_umma = true;    // tcgen05 GEMM for projections of more than 8 rows
+  uint4 *act_blocks = nullptr;
   float *w_final = nullptr;
   double *inv_freq = nullptr;
 
@@ -187,6 +192,29 @@ dmtd_status vec_to_float(dmtd_ctx *c, float **out, const void *src, int n) {
   return DMTD_OK;
 }
 
+// Second copy of a (fused) matrix in the block order of the tcgen05 GEMM.
+dmtd_status pack_umma(dmtd_ctx *c, UmmaMat *out, int K, const void *const *srcs, const int *Ns, int n_src) {
+  int N = 0;
+  for (int i = 0; i < n_src; ++i) N += Ns[i];
+  UmmaMat m{};
+  m.N = N; m.K = K; m.n_tiles = (N + TG_ROWS - 1) / TG_ROWS; m.n_kb = K / TG_KB;
+  uint4 *dst = nullptr;
+  size_t units = (size_t)m.n_tiles * m.n_kb * (TG_WBLOCK / 16);
+  TRY(dev_alloc(c, &dst, units));
+  CUDA_TRY(c, cudaMemsetAsync(dst, 0, units * 16, c->stream));
+  int row0 = 0;
+  for (int i = 0; i < n_src; ++i) {
+    long long total = (long long)Ns[i] * (K / 8);
+    int grid = (int)std::min<long long>((total + 255) / 256, 65535);
+    pack_umma_kernel<<<grid, 256, 0, c->stream>>>(static_cast<const __nv_bfloat16 *>(srcs[i]), Ns[i], K, row0, m.n_kb, dst);
+    LAUNCH_OK(c, "pack_umma_kernel");
+    row0 += Ns[i];
+  }
+  m.w = dst;
+  *out = m;
+  return DMTD_OK;
+}
+
 // ---------------------------------------------------------------------------- launches
 
 int gemv_smem_bytes(const PackedMat &W, int NT) {
@@ -208,8 +236,37 @@ dmtd_status launch_gemv_nt(dmtd_ctx *c, const PackedMat &W, const float *act, in
   return DMTD_OK;
 }
 
+// out[m][n] += sum_k W[n][k] act[m][k] on the tcgen05 tensor cores, 128 activation rows at a time.
+dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, int lda, int M, float *out, int ldo) {
+  for (int m0 = 0; m0 < M; m0 += TG_MAX_COLS / 2) {
+    GemmTcParams P{};
+    P.W = W; P.act_blocks = c->act_blocks;
+    P.rows = std::min(TG_MAX_COLS / 2, M - m0);
+    P.n_cols = (2 * P.rows + 15) / 16 * 16;
+    P.out = out + (size_t)m0 * ldo; P.ldo = ldo;
+    P.ksplit = std::max(1, std::min(W.n_kb, (c->n_sms + W.n_tiles - 1) / W.n_tiles));
+    P.error = &c->dstate->error; P.wait_limit = 2000000000ll;
+    long long units = (long long)W.n_kb * 8 * P.n_cols;
+    act_blocks_kernel<<<(int)std::min<long long>((units + 255) / 256, 4096), 256, 0, c->stream>>>(
+        act + (size_t)m0 * lda, lda, P.rows, W.K, P.n_cols, c->act_blocks);
+    LAUNCH_OK(c, "act_blocks_kernel");
+    int smem = TG_STAGES * (TG_WBLOCK + P.n_cols * 128) + 128;
+    static int configured = 0;
+    if (configured < smem) {
+      CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       TG_STAGES * (TG_WBLOCK + TG_MAX_COLS * 128) + 128));
+      configured = TG_STAGES * (TG_WBLOCK + TG_MAX_COLS * 128) + 128;
+    }
+    gemm_tc05_kernel<<<W.n_tiles * P.ksplit, TG_THREADS, smem, c->stream>>>(P);
+    LAUNCH_OK(c, "gemm_tc05_kernel");
+  }
+  return DMTD_OK;
+}
+
 // out[m][n] += sum_k W[n][k] act[m][k]
-dmtd_status launch_gemv(dmtd_ctx *c, const PackedMat &W, const float *act, int lda, int M, float *out, int ldo) {
+dmtd_status launch_gemv(dmtd_ctx *c, const PackedMat &W, const UmmaMat &U, const float *act, int lda, int M, float *out,
+                        int ldo) {
+  if (U.w && c->use_umma && M > 8) return launch_gemm_tc05(c, U, act, lda, M, out, ldo);
   if (W.wf) {
     gemv_f32_kernel<<<2 * c->n_sms, 256, 0, c->stream>>>(W, act, lda, M, out, ldo);
     LAUNCH_OK(c, "gemv_f32_kernel");
@@ -299,16 +356,16 @@ dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos
   int M = B * R, H = s.hidden, I = s.intermediate, QD = s.n_q_heads * s.head_dim;
   prep_norm_kernel<<<M, 256, 0, c->stream>>>(x, H, lw.w_in, H, s.rms_eps, c->act, c->lda, c->qkv, c->ldqkv, c->ldqkv);
   LAUNCH_OK(c, "prep_norm_kernel");
-  TRY(launch_gemv(c, lw.qkv, c->act, c->lda, M, c->qkv, c->ldqkv));
+  TRY(launch_gemv(c, lw.qkv, lw.qkv_u, c->act, c->lda, M, c->qkv, c->ldqkv));
   TRY(launch_attention(c, l, B, R, pos0, splits_for(c, pos_end)));
   (void)QD;
-  TRY(launch_gemv(c, lw.o, c->act, c->lda, M, x, H));
+  TRY(launch_gemv(c, lw.o, lw.o_u, c->act, c->lda, M, x, H));
   prep_norm_kernel<<<M, 256, 0, c->stream>>>(x, H, lw.w_post, H, s.rms_eps, c->act, c->lda, c->gu, c->ldgu, c->ldgu);
   LAUNCH_OK(c, "prep_norm_kernel");
-  TRY(launch_gemv(c, lw.gu, c->act, c->lda, M, c->gu, c->ldgu));
+  TRY(launch_gemv(c, lw.gu, lw.gu_u, c->act, c->lda, M, c->gu, c->ldgu));
   prep_swiglu_kernel<<<dim3((I + 255) / 256, M), 256, 0, c->stream>>>(c->gu, c->ldgu, I, c->act, c->lda);
   LAUNCH_OK(c, "prep_swiglu_kernel");
-  TRY(launch_gemv(c, lw.down, c->act, c->lda, M, x, H));
+  TRY(launch_gemv(c, lw.down, lw.down_u, c->act, c->lda, M, x, H));
   return DMTD_OK;
 }
 
@@ -318,7 +375,7 @@ dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, floa
   prep_norm_kernel<<<B, 256, 0, c->stream>>>(c->x_up, s.hidden, c->w_final, s.hidden, s.rms_eps, c->act, c->lda,
                                              c->logits, c->ldl, c->ldl);
   LAUNCH_OK(c, "prep_norm_kernel");
-  TRY(launch_gemv(c, c->embed, c->act, c->lda, B, c->logits, c->ldl));
+  TRY(launch_gemv(c, c->embed, c->embed_u, c->act, c->lda, B, c->logits, c->ldl));
   if (out_logits)
     CUDA_TRY(c, cudaMemcpy2DAsync(out_logits, (size_t)s.vocab * 4, c->logits, (size_t)c->ldl * 4, (size_t)s.vocab * 4, B,
                                   cudaMemcpyDeviceToDevice, c->stream));
@@ -557,7 +614,10 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   const dmtd_model_shape &s = c->s;
   const int H = s.hidden, D = s.head_dim, QD = s.n_q_heads * D, KVD = s.n_kv_heads * D, I = s.intermediate;
 
-  // weights
+  // weights; contexts whose passes can hold more than 8 rows (batch x cycle length) also get the
+  // copy the tcgen05 GEMM reads
+  c->umma_ok = s.weight_dtype == DMTD_BF16 && (long long)max_batch * std::max(tau, 1) > 8 && H % TG_KB == 0 &&
+               QD % TG_KB == 0 && I % TG_KB == 0;
   c->layers.resize(s.n_layers);
   for (int l = 0; l < s.n_layers; ++l) {
     const dmtd_layer_weights &lw = w->layers[l];
@@ -576,6 +636,12 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
     CTRY(pack_matrix(c, &ld.gu, H, gu_src, gu_n, 2));
     const void *d_src[1] = {lw.down_proj}; int d_n[1] = {H};
     CTRY(pack_matrix(c, &ld.down, I, d_src, d_n, 1));
+    if (c->umma_ok) {
+      CTRY(pack_umma(c, &ld.qkv_u, H, qkv_src, qkv_n, 3));
+      CTRY(pack_umma(c, &ld.o_u, QD, o_src, o_n, 1));
+      CTRY(pack_umma(c, &ld.gu_u, H, gu_src, gu_n, 2));
+      CTRY(pack_umma(c, &ld.down_u, I, d_src, d_n, 1));
+    }
     CTRY(vec_to_float(c, &ld.w_in, lw.input_norm, H));
     CTRY(vec_to_float(c, &ld.w_post, lw.post_norm, H));
     CTRY(vec_to_float(c, &ld.w_qn, lw.q_norm, D));
@@ -584,6 +650,7 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   {
     const void *e_src[1] = {w->embed}; int e_n[1] = {s.vocab};
     CTRY(pack_matrix(c, &c->embed, H, e_src, e_n, 1));
+    if (c->umma_ok) CTRY(pack_umma(c, &c->embed_u, H, e_src, e_n, 1));
     CTRY(vec_to_float(c, &c->w_final, w->final_norm, H));
   }
   {
@@ -620,6 +687,7 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   CTRY(dev_alloc(c, &c->part_o, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * D));
   CTRY(dev_alloc(c, &c->part_ml, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * 2));
   CTRY(dev_alloc(c, &c->rope_tab, (size_t)c->ws_rows * (D / 2)));
+  if (c->umma_ok) CTRY(dev_alloc(c, &c->act_blocks, (size_t)(c->lda / TG_KB) * 8 * TG_MAX_COLS));
   CTRY(setup_fused(c));
   CTRY(dmtd_reset(c));
   CCUDA(cudaStreamSynchronize(c->stream));   // repacking done: the caller may free its weights
@@ -813,6 +881,7 @@ dmtd_status dmtd_set_option(dmtd_ctx *c, const char *name, int64_t value) {
   if (!strcmp(name, "cuda_graph")) { c->use_graph = value != 0; return DMTD_OK; }
   if (!strcmp(name, "literal_sum")) { c->literal_sum = value != 0; drop_graphs(c); return DMTD_OK; }
   if (!strcmp(name, "fused_pass")) { c->use_fused = value != 0; return DMTD_OK; }
+  if (!strcmp(name, "tcgen05_gemm")) { c->use_umma = value != 0; drop_graphs(c); return DMTD_OK; }
   if (!strcmp(name, "tc_attention")) { c->use_tc_attention = value != 0; drop_graphs(c); return DMTD_OK; }
   return fail(c, DMTD_ERR_INVALID_ARG, "unknown option %s", name);
 }

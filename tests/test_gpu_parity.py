@@ -380,3 +380,25 @@ def test_fused_pass_kernel_free_running(dmtd):
     for b in range(B):
         upto = n_new if clear[b].all() else int(np.argmin(clear[b]))
         assert (got[b, :upto] == toks[b, :upto]).all()
+
+
+@pytest.mark.parametrize("B,tau,P,n_new", [(12, 3, 23, 8), (40, 1, 9, 3)])
+def test_tcgen05_projections_many_rows(dmtd, B, tau, P, n_new):
+    """Passes of more than 8 rows run their projections on the tcgen05 GEMM (prefill chunks of up
+    to 256 rows included): against the oracle, and against the mma.sync GEMV on the same inputs."""
+    shape = SHAPES["mid"].with_(intermediate=1856)          # every K a multiple of the 64-wide k block
+    w = make_weights(shape, seed=0, norm_jitter=0.1)
+    prompts = make_prompts(shape.vocab, B, P, seed=1).numpy()
+    toks, _, _, _ = oracle_greedy(shape, w, 2, tau, prompts, n_new)
+    ref_logits, ref_am, o = oracle_forced(shape, w, 2, tau, prompts, toks)
+    wc = to_cuda(w)
+    res = {}
+    for tc in (1, 0):
+        eng = _engine(dmtd, shape, wc, 2, tau, B, P + n_new + 1, kv_dtype="f32")
+        eng.set_option("tcgen05_gemm", tc)
+        got_logits, got_am = gpu_forced(eng, prompts, toks)
+        err, _ = check_logits(got_logits, ref_logits, got_am, ref_am)
+        assert err < 1e-3
+        assert eng.device_state() == o.state()
+        res[tc] = got_logits
+    assert np.abs(res[1] - res[0]).max() < 1e-3
