@@ -15,7 +15,7 @@ constexpr int ATTN_TC_SMEM = PK_AT_ROWS;         // tiles, Q, partial-output ove
 // qkv [B*R][ldq]: q heads already normalised and rotated (not scaled); K and V of the new rows
 // already in the cache.  Cache [b][kv head][max_seq][128] bf16 (PRECISE = false) or fp32.
 template <bool PRECISE>
-__global__ void __launch_bounds__(PK_THREADS)
+__global__ void __launch_bounds__(PK_THREADS, PRECISE ? 1 : 2)      // bf16 cache: two blocks per SM overlap load and math
 attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ kc, const void *__restrict__ vc, int max_seq,
                int nq, int nkv, int R, int RB, int CH, const int *__restrict__ pos0_ptr, float *__restrict__ part_o,
                float *__restrict__ part_ml, int nsplit) {
