@@ -267,6 +267,17 @@ class Oracle:
         return out
 
 
+def _set_kv(self, layer, b, k, v):
+    """Overwrite the first positions of one layer's cache of sequence b: k, v [n_pos, nkv, d]."""
+    nkv, d = self.shape.n_kv_heads, self.shape.head_dim
+    for fn, src in ((self.lib.dll.oracle_k_cache, k), (self.lib.dll.oracle_v_cache, v)):
+        a = np.ctypeslib.as_array(fn(self._ctx, layer, b), shape=(self.max_seq, nkv, d))
+        a[: src.shape[0]] = src
+
+
+Oracle.set_kv = _set_kv
+
+
 def vanilla_generate(shape, weights, prompt, n_new, forced=None):
     """Plain full-recompute autoregressive decoding of one sequence.
     Returns (tokens [P+n_new], logits [n_new, V], argmax [n_new])."""

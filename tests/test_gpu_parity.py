@@ -402,3 +402,35 @@ def test_tcgen05_projections_many_rows(dmtd, B, tau, P, n_new):
         assert eng.device_state() == o.state()
         res[tc] = got_logits
     assert np.abs(res[1] - res[0]).max() < 1e-3
+
+
+@pytest.mark.parametrize("B,S", [(8, 2048), (64, 300), (1, 4100)])
+def test_single_layer_cell_random_hidden_and_kv(dmtd, oracle_lib, B, S):
+    """A cell of the single-layer microbenchmark (4B layer geometry, random N(0,1) hidden states and
+    KV cache, one decode step) against the oracle's layer on the same values."""
+    import ctypes
+    import oracle
+    shape = SHAPES["qwen3_4b"].with_(n_layers=1, vocab=512)
+    w = make_weights(shape, seed=2)
+    g = torch.Generator().manual_seed(7)
+    k = torch.randn(B, shape.n_kv_heads, S, shape.head_dim, generator=g).to(torch.bfloat16)
+    v = torch.randn(B, shape.n_kv_heads, S, shape.head_dim, generator=g).to(torch.bfloat16)
+    hidden = torch.randn(B, 1, shape.hidden, generator=g)
+    o = oracle.Oracle(shape, w, L_d=1, tau=1, max_batch=B, max_seq=S + 1)
+    for b in range(B):
+        o.set_kv(0, b, k[b].double().permute(1, 0, 2).numpy(), v[b].double().permute(1, 0, 2).numpy())
+    ref = o.step_layers(0, 1, hidden.double().numpy(), S)
+    eng = _engine(dmtd, shape, to_cuda(w), 1, 1, B, S + 1, kv_dtype="bf16")
+    kp, vp = eng.kv(0)
+    rt = ctypes.CDLL("libcudart.so")
+    per_seq = shape.n_kv_heads * (S + 1) * shape.head_dim
+    for ptr, src in ((kp, k), (vp, v)):
+        full = torch.zeros(B, shape.n_kv_heads, S + 1, shape.head_dim, dtype=torch.bfloat16)
+        full[:, :, :S] = src
+        dev = full.cuda()
+        rt.cudaMemcpy(ctypes.c_void_p(ptr), ctypes.c_void_p(dev.data_ptr()), ctypes.c_size_t(B * per_seq * 2), 3)
+    got = eng.step_layers(0, 1, hidden.cuda().contiguous(), S)
+    torch.cuda.synchronize()
+    scale = np.abs(ref).max()
+    # bf16 cache on the tensor cores: Q, P and the appended K, V rounded to bf16 (2^-9 relative)
+    assert np.abs(got.double().cpu().numpy() - ref).max() <= 4e-3 * max(1.0, scale)
