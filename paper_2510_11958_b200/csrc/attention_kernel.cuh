@@ -60,38 +60,80 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
   for (int dt = 0; dt < 16; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
   uint4 qh[4][2];
   const int n_keys = j1 - j0;
-  for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
-    const int n_t = min(PK_TK, n_keys - tile0);
-    __syncthreads();                                      // Q written / previous tile consumed
-    if (!PRECISE) {
-      const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(kc) + head_off;
-      const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(vc) + head_off;
+  if (!PRECISE) {
+    // bf16 cache: two tile buffers (the lo-part areas are free here), tile i+1 in flight while
+    // tile i is multiplied
+    const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(kc) + head_off;
+    const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(vc) + head_off;
+    auto fetch = [&](int tile0, int buf) {
+      const int n_t = min(PK_TK, n_keys - tile0);
+      const uint32_t k_t = smem_u32(sc + (buf ? PK_AT_KL : PK_AT_KH)), v_t = smem_u32(sc + (buf ? PK_AT_VL : PK_AT_VH));
       for (int c = threadIdx.x; c < n_t * 32; c += PK_THREADS) {
         const int row = c >> 5, part = c & 31;
-        const uint32_t dst = part < 16 ? kh_tile + row * PK_KROW + part * 16 : vh_tile + row * PK_VROW + (part - 16) * 16;
+        const uint32_t dst = part < 16 ? k_t + row * PK_KROW + part * 16 : v_t + row * PK_VROW + (part - 16) * 16;
         cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
       }
-    } else {
-      attn_fetch_f32(reinterpret_cast<const float *>(kc) + head_off + (size_t)(j0 + tile0) * PK_D,
-                     reinterpret_cast<const float *>(vc) + head_off + (size_t)(j0 + tile0) * PK_D, n_t, sc);
-    }
-    const int n16 = min(PK_TK, (n_t + 15) & ~15);
-    for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS) {      // P = 0 times stale bits must stay 0
-      const uint32_t off = (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16;
-      sts128(vh_tile + off, make_uint4(0u, 0u, 0u, 0u));
-      if (PRECISE) sts128(vl_tile + off, make_uint4(0u, 0u, 0u, 0u));
-    }
-    cp_async_wait_all();
-    __syncthreads();
-    if (tile0 == 0) {
-#pragma unroll
-      for (int kb = 0; kb < 4; ++kb) {
-        qh[kb][0] = lds128(qh_tile + g * PK_QROW + kb * 64 + t * 16);
-        qh[kb][1] = lds128(qh_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
+      const int n16 = min(PK_TK, (n_t + 15) & ~15);
+      for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS)      // P = 0 times stale bits must stay 0
+        sts128(v_t + (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16, make_uint4(0u, 0u, 0u, 0u));
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    fetch(0, 0);
+    int buf = 0;
+    for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK, buf ^= 1) {
+      const int n_t = min(PK_TK, n_keys - tile0);
+      if (tile0 + PK_TK < n_keys) {
+        fetch(tile0 + PK_TK, buf ^ 1);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+      } else {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
       }
+      __syncthreads();                                    // tile (and, the first time, Q) visible to all
+      if (tile0 == 0) {
+#pragma unroll
+        for (int kbk = 0; kbk < 4; ++kbk) {
+          qh[kbk][0] = lds128(qh_tile + g * PK_QROW + kbk * 64 + t * 16);
+          qh[kbk][1] = lds128(qh_tile + (g + 8) * PK_QROW + kbk * 64 + t * 16);
+        }
+      }
+      attn_tile_compute<false>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH,
+                               buf ? PK_AT_VL : PK_AT_VH);
+      __syncthreads();                                    // done with this buffer before it is refilled
     }
-    // every key comes from the cache: key index i sits at position j0 + i
-    attn_tile_compute<PRECISE>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G);
+  } else {
+    for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
+      const int n_t = min(PK_TK, n_keys - tile0);
+      __syncthreads();                                      // Q written / previous tile consumed
+      if (!PRECISE) {
+        const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(kc) + head_off;
+        const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(vc) + head_off;
+        for (int c = threadIdx.x; c < n_t * 32; c += PK_THREADS) {
+          const int row = c >> 5, part = c & 31;
+          const uint32_t dst = part < 16 ? kh_tile + row * PK_KROW + part * 16 : vh_tile + row * PK_VROW + (part - 16) * 16;
+          cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
+        }
+      } else {
+        attn_fetch_f32(reinterpret_cast<const float *>(kc) + head_off + (size_t)(j0 + tile0) * PK_D,
+                       reinterpret_cast<const float *>(vc) + head_off + (size_t)(j0 + tile0) * PK_D, n_t, sc);
+      }
+      const int n16 = min(PK_TK, (n_t + 15) & ~15);
+      for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS) {      // P = 0 times stale bits must stay 0
+        const uint32_t off = (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16;
+        sts128(vh_tile + off, make_uint4(0u, 0u, 0u, 0u));
+        if (PRECISE) sts128(vl_tile + off, make_uint4(0u, 0u, 0u, 0u));
+      }
+      cp_async_wait_all();
+      __syncthreads();
+      if (tile0 == 0) {
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          qh[kb][0] = lds128(qh_tile + g * PK_QROW + kb * 64 + t * 16);
+          qh[kb][1] = lds128(qh_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
+        }
+      }
+      // every key comes from the cache: key index i sits at position j0 + i
+      attn_tile_compute<PRECISE>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G);
+    }
   }
   attn_combine_store(A, sc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
 }

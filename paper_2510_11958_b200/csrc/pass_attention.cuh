@@ -147,12 +147,14 @@ struct AttnAcc {
 
 // Keys of the tile are key_idx0 + row; key index i sits at position (i < n_cached ? j0 + i :
 // pos_new + i - n_cached); query row q may see positions up to row_pos0 + q / G.
+// k_off / v_off: where the tile's K and V (hi parts) sit in the scratch.
 template <bool PRECISE>
 __device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc, const uint4 (&qh)[4][2], int n_t, int tile0,
-                                                  int n_cached, int j0, int pos_new, int row_pos0, int G) {
+                                                  int n_cached, int j0, int pos_new, int row_pos0, int G,
+                                                  int k_off = PK_AT_KH, int v_off = PK_AT_VH) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-  const uint32_t kh_tile = smem_u32(sc + PK_AT_KH), kl_tile = smem_u32(sc + PK_AT_KL);
-  const uint32_t vh_tile = smem_u32(sc + PK_AT_VH), vl_tile = smem_u32(sc + PK_AT_VL);
+  const uint32_t kh_tile = smem_u32(sc + k_off), kl_tile = smem_u32(sc + PK_AT_KL);
+  const uint32_t vh_tile = smem_u32(sc + v_off), vl_tile = smem_u32(sc + PK_AT_VL);
   const uint32_t ql_tile = smem_u32(sc + PK_AT_QL);
   float (&m_run)[2] = A.m_run;
   float (&l_part)[2] = A.l_part;

@@ -12,7 +12,9 @@
 //    with 16 KiB per warp in flight a barrier poll or an activation load waited 3-4 us behind
 //    the block's own weight traffic, with 8 KiB about half of that, at the same stream rate;
 //    asking for the next projection's weights to be prefetched into L2 at a stage boundary made
-//    the following projection slower, not faster, so nothing is requested beyond the ring.
+//    the following projection slower, not faster, so nothing is requested beyond the ring;
+//  * the grid barrier is one counter (release-add, acquire-poll by one thread per block): 2-3 us.
+//    A flag per block polled by a warp (no atomic serialisation) took 5-6 us.
 #pragma once
 
 #include "common.cuh"
