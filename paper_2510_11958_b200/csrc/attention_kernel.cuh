@@ -20,7 +20,7 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
                int nq, int nkv, int R, int RB, int CH, const int *__restrict__ pos0_ptr, float *__restrict__ part_o,
                float *__restrict__ part_ml, int nsplit) {
   extern __shared__ __align__(1024) unsigned char sc[];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = nq / nkv, n_rb = (R + RB - 1) / RB;
   const int split = blockIdx.x, kvh = blockIdx.y / n_rb, rb = blockIdx.y % n_rb, b = blockIdx.z;
   const int r0 = rb * RB, r1 = min(R, r0 + RB), nQ = (r1 - r0) * G;
@@ -57,8 +57,7 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
   A.m_run[0] = A.m_run[1] = -INFINITY;
   A.l_part[0] = A.l_part[1] = 0.f;
 #pragma unroll
-  for (int dt = 0; dt < 16; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
-  uint4 qh[4][2];
+  for (int dt = 0; dt < 8; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
   const int n_keys = j1 - j0;
   if (!PRECISE) {
     // bf16 cache: two tile buffers (the lo-part areas are free here), tile i+1 in flight while
@@ -89,14 +88,7 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
         asm volatile("cp.async.wait_group 0;" ::: "memory");
       }
       __syncthreads();                                    // tile (and, the first time, Q) visible to all
-      if (tile0 == 0) {
-#pragma unroll
-        for (int kbk = 0; kbk < 4; ++kbk) {
-          qh[kbk][0] = lds128(qh_tile + g * PK_QROW + kbk * 64 + t * 16);
-          qh[kbk][1] = lds128(qh_tile + (g + 8) * PK_QROW + kbk * 64 + t * 16);
-        }
-      }
-      attn_tile_compute<false>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH,
+      attn_tile_compute<false>(A, sc, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH,
                                buf ? PK_AT_VL : PK_AT_VH);
       __syncthreads();                                    // done with this buffer before it is refilled
     }
@@ -124,15 +116,8 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
       }
       cp_async_wait_all();
       __syncthreads();
-      if (tile0 == 0) {
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          qh[kb][0] = lds128(qh_tile + g * PK_QROW + kb * 64 + t * 16);
-          qh[kb][1] = lds128(qh_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
-        }
-      }
       // every key comes from the cache: key index i sits at position j0 + i
-      attn_tile_compute<PRECISE>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G);
+      attn_tile_compute<PRECISE>(A, sc, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G);
     }
   }
   attn_combine_store(A, sc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);

@@ -12,6 +12,17 @@
 
 namespace dmtd {
 
+// Profiling builds: clock64() of thread 0 of the first block at points inside the attention
+// stage (the last layer's values stay), in the 16 slots before the wall-clock slots.
+#ifdef DMTD_PASS_TIMING
+#define PK_SUBSTAMP(i)                                                                     \
+  do {                                                                                     \
+    if (threadIdx.x == 0 && blockIdx.x == 0 && P.timing) P.timing[4096 - 4 - 16 + (i)] = clock64(); \
+  } while (0)
+#else
+#define PK_SUBSTAMP(i) do {} while (0)
+#endif
+
 constexpr int PK_FETCH = 10;                                  // float4 units of an fp32 tile a thread loads at once
 constexpr int PK_TK = 64;                                     // keys per shared-memory tile
 constexpr int PK_KROW = 320;                                  // bytes per K row: 256 + 64, conflict-free 16-byte operand loads
@@ -82,6 +93,7 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
   const int G = P.nq / P.nkv, nQ = R * G;
   const float *rows = reinterpret_cast<const float *>(sc + PK_AT_ROWS);
   const float scale = rsqrtf((float)PK_D);
+#pragma unroll 1
   for (int task = warp; task < nQ + 2 * R; task += PK_WARPS) {
     int r, col, kind;                                   // kind 0 q, 1 k, 2 v
     if (task < nQ) { r = task / G; col = (task % G) * PK_D; kind = 0; }
@@ -138,168 +150,173 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
   }
 }
 
-// One 64-key tile against the 16 query rows: this warp's 16 keys.  acc holds the warp's running
-// max, running sum (per lane, summed over the four lanes of a row at the end) and output.
+// One 64-key tile against the 16 query rows.  Warp w takes keys 16 (w & 3) .. + 15 of the tile
+// and output dimensions 64 (w >> 2) .. + 63: the two warps of a key group compute the same
+// scores and each multiplies them with its half of V.  acc holds the warp's running max, running
+// sum (per lane, summed over the four lanes of a row at the end) and output.
 struct AttnAcc {
   float m_run[2], l_part[2];
-  float o[16][4];
+  float o[8][4];
 };
 
 // Keys of the tile are key_idx0 + row; key index i sits at position (i < n_cached ? j0 + i :
 // pos_new + i - n_cached); query row q may see positions up to row_pos0 + q / G.
-// k_off / v_off: where the tile's K and V (hi parts) sit in the scratch.
+// k_off / v_off: where the tile's K and V (hi parts) sit in the scratch.  The Q fragments are
+// read from shared memory in a rolled loop: the code stays short (instruction fetch, not
+// arithmetic, bounds a stage that runs once per layer).
 template <bool PRECISE>
-__device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc, const uint4 (&qh)[4][2], int n_t, int tile0,
-                                                  int n_cached, int j0, int pos_new, int row_pos0, int G,
-                                                  int k_off = PK_AT_KH, int v_off = PK_AT_VH) {
+__device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc, int n_t, int tile0, int n_cached, int j0,
+                                                  int pos_new, int row_pos0, int G, int k_off = PK_AT_KH,
+                                                  int v_off = PK_AT_VH) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int kg = warp & 3, dh = warp >> 2;
   const uint32_t kh_tile = smem_u32(sc + k_off), kl_tile = smem_u32(sc + PK_AT_KL);
   const uint32_t vh_tile = smem_u32(sc + v_off), vl_tile = smem_u32(sc + PK_AT_VL);
-  const uint32_t ql_tile = smem_u32(sc + PK_AT_QL);
+  const uint32_t qh_tile = smem_u32(sc + PK_AT_QH), ql_tile = smem_u32(sc + PK_AT_QL);
   float (&m_run)[2] = A.m_run;
   float (&l_part)[2] = A.l_part;
-  float (&o)[16][4] = A.o;
-  if (warp * 16 < n_t) {
-        float c[2][4];
+  float (&o)[8][4] = A.o;
+  if (kg * 16 >= n_t) return;
+  float c[2][4];
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-          c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+  for (int nt = 0; nt < 2; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+#pragma unroll 1
+  for (int kb = 0; kb < 4; ++kb) {
+    const uint32_t q_off = g * PK_QROW + kb * 64 + t * 16;
+    const uint4 q0 = lds128(qh_tile + q_off), q1 = lds128(qh_tile + q_off + 8 * PK_QROW);
+    uint4 p0 = make_uint4(0u, 0u, 0u, 0u), p1 = p0;
+    if (PRECISE) { p0 = lds128(ql_tile + q_off); p1 = lds128(ql_tile + q_off + 8 * PK_QROW); }
 #pragma unroll
-          for (int kb = 0; kb < 4; ++kb) {
-            const uint32_t off = (warp * 16 + nt * 8 + g) * PK_KROW + kb * 64 + t * 16;
-            const uint4 Kh = lds128(kh_tile + off);
-            mma_bf16_16816(c[nt], qh[kb][0].x, qh[kb][1].x, qh[kb][0].y, qh[kb][1].y, Kh.x, Kh.y);
-            mma_bf16_16816(c[nt], qh[kb][0].z, qh[kb][1].z, qh[kb][0].w, qh[kb][1].w, Kh.z, Kh.w);
-            if (PRECISE) {
-              // the lo parts of Q stay in shared memory: registers are short here
-              const uint4 Kl = lds128(kl_tile + off);
-              const uint4 q0 = lds128(ql_tile + g * PK_QROW + kb * 64 + t * 16);
-              const uint4 q1 = lds128(ql_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
-              mma_bf16_16816(c[nt], qh[kb][0].x, qh[kb][1].x, qh[kb][0].y, qh[kb][1].y, Kl.x, Kl.y);
-              mma_bf16_16816(c[nt], qh[kb][0].z, qh[kb][1].z, qh[kb][0].w, qh[kb][1].w, Kl.z, Kl.w);
-              mma_bf16_16816(c[nt], q0.x, q1.x, q0.y, q1.y, Kh.x, Kh.y);
-              mma_bf16_16816(c[nt], q0.z, q1.z, q0.w, q1.w, Kh.z, Kh.w);
-            }
-          }
-        }
-        // causal / range mask: lane holds rows g (e = 0, 1) and g + 8 (e = 2, 3), keys 2t, 2t + 1 of each n-tile
-        float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int kl = warp * 16 + nt * 8 + 2 * t + (e & 1), idx = tile0 + kl, row = g + (e >> 1) * 8;
-            const int key_pos = idx < n_cached ? j0 + idx : pos_new + (idx - n_cached);
-            const bool ok = kl < n_t && key_pos <= row_pos0 + row / G;
-            c[nt][e] = ok ? c[nt][e] : -INFINITY;
-            mx[e >> 1] = fmaxf(mx[e >> 1], c[nt][e]);
-          }
-        }
-        float corr[2];
-#pragma unroll
-        for (int hr = 0; hr < 2; ++hr) {
-          mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 1));
-          mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 2));
-          const float m_new = fmaxf(m_run[hr], mx[hr]);
-          corr[hr] = m_new > -INFINITY ? __expf(m_run[hr] - m_new) : 1.f;
-          m_run[hr] = m_new;
-        }
-        float psum[2] = {0.f, 0.f};
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float p = c[nt][e] > -INFINITY ? __expf(c[nt][e] - m_run[e >> 1]) : 0.f;
-            c[nt][e] = p;
-            psum[e >> 1] += p;
-          }
-        }
-        l_part[0] = l_part[0] * corr[0] + psum[0];
-        l_part[1] = l_part[1] * corr[1] + psum[1];
-        // P as the A operand: hi parts and (fp32 cache) lo parts
-        uint32_t ah[4], al[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float p0 = c[i >> 1][(i & 1) * 2], p1 = c[i >> 1][(i & 1) * 2 + 1];
-          ah[i] = pack_bf16x2(p0, p1);
-          if (PRECISE) al[i] = pack_bf16x2(p0 - __uint_as_float(ah[i] << 16), p1 - __uint_as_float(ah[i] & 0xffff0000u));
-        }
-        const int mi = lane >> 3, rr = lane & 7;
-        const uint32_t v_off = (warp * 16 + (mi & 1) * 8 + rr) * PK_VROW + (mi >> 1) * 16;
-#pragma unroll
-        for (int d2 = 0; d2 < 8; ++d2) {
-          uint32_t b0, b1, b2, b3;
-          ldmatrix_x4_trans(vh_tile + v_off + d2 * 32, b0, b1, b2, b3);
-          o[2 * d2][0] *= corr[0]; o[2 * d2][1] *= corr[0]; o[2 * d2][2] *= corr[1]; o[2 * d2][3] *= corr[1];
-          o[2 * d2 + 1][0] *= corr[0]; o[2 * d2 + 1][1] *= corr[0]; o[2 * d2 + 1][2] *= corr[1]; o[2 * d2 + 1][3] *= corr[1];
-          mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
-          mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
-          if (PRECISE) {
-            mma_bf16_16816(o[2 * d2], al[0], al[1], al[2], al[3], b0, b1);
-            mma_bf16_16816(o[2 * d2 + 1], al[0], al[1], al[2], al[3], b2, b3);
-            ldmatrix_x4_trans(vl_tile + v_off + d2 * 32, b0, b1, b2, b3);
-            mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
-            mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
-          }
-        }
+    for (int nt = 0; nt < 2; ++nt) {
+      const uint32_t off = (kg * 16 + nt * 8 + g) * PK_KROW + kb * 64 + t * 16;
+      const uint4 Kh = lds128(kh_tile + off);
+      mma_bf16_16816(c[nt], q0.x, q1.x, q0.y, q1.y, Kh.x, Kh.y);
+      mma_bf16_16816(c[nt], q0.z, q1.z, q0.w, q1.w, Kh.z, Kh.w);
+      if (PRECISE) {
+        const uint4 Kl = lds128(kl_tile + off);
+        mma_bf16_16816(c[nt], q0.x, q1.x, q0.y, q1.y, Kl.x, Kl.y);
+        mma_bf16_16816(c[nt], q0.z, q1.z, q0.w, q1.w, Kl.z, Kl.w);
+        mma_bf16_16816(c[nt], p0.x, p1.x, p0.y, p1.y, Kh.x, Kh.y);
+        mma_bf16_16816(c[nt], p0.z, p1.z, p0.w, p1.w, Kh.z, Kh.w);
       }
+    }
+  }
+  // causal / range mask: lane holds rows g (e = 0, 1) and g + 8 (e = 2, 3), keys 2t, 2t + 1 of each n-tile
+  float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int kl = kg * 16 + nt * 8 + 2 * t + (e & 1), idx = tile0 + kl, row = g + (e >> 1) * 8;
+      const int key_pos = idx < n_cached ? j0 + idx : pos_new + (idx - n_cached);
+      const bool ok = kl < n_t && key_pos <= row_pos0 + row / G;
+      c[nt][e] = ok ? c[nt][e] : -INFINITY;
+      mx[e >> 1] = fmaxf(mx[e >> 1], c[nt][e]);
+    }
+  }
+  float corr[2];
+#pragma unroll
+  for (int hr = 0; hr < 2; ++hr) {
+    mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 1));
+    mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 2));
+    const float m_new = fmaxf(m_run[hr], mx[hr]);
+    corr[hr] = m_new > -INFINITY ? __expf(m_run[hr] - m_new) : 1.f;
+    m_run[hr] = m_new;
+  }
+  float psum[2] = {0.f, 0.f};
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float p = c[nt][e] > -INFINITY ? __expf(c[nt][e] - m_run[e >> 1]) : 0.f;
+      c[nt][e] = p;
+      psum[e >> 1] += p;
+    }
+  }
+  l_part[0] = l_part[0] * corr[0] + psum[0];
+  l_part[1] = l_part[1] * corr[1] + psum[1];
+  // P as the A operand: hi parts and (fp32 cache) lo parts
+  uint32_t ah[4], al[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float p0 = c[i >> 1][(i & 1) * 2], p1 = c[i >> 1][(i & 1) * 2 + 1];
+    ah[i] = pack_bf16x2(p0, p1);
+    if (PRECISE) al[i] = pack_bf16x2(p0 - __uint_as_float(ah[i] << 16), p1 - __uint_as_float(ah[i] & 0xffff0000u));
+  }
+  const int mi = lane >> 3, rr = lane & 7;
+  const uint32_t v_row = (kg * 16 + (mi & 1) * 8 + rr) * PK_VROW + (mi >> 1) * 16 + dh * 128;
+#pragma unroll
+  for (int d2 = 0; d2 < 4; ++d2) {
+    uint32_t b0, b1, b2, b3;
+    ldmatrix_x4_trans(vh_tile + v_row + d2 * 32, b0, b1, b2, b3);
+    o[2 * d2][0] *= corr[0]; o[2 * d2][1] *= corr[0]; o[2 * d2][2] *= corr[1]; o[2 * d2][3] *= corr[1];
+    o[2 * d2 + 1][0] *= corr[0]; o[2 * d2 + 1][1] *= corr[0]; o[2 * d2 + 1][2] *= corr[1]; o[2 * d2 + 1][3] *= corr[1];
+    mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
+    mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+    if (PRECISE) {
+      mma_bf16_16816(o[2 * d2], al[0], al[1], al[2], al[3], b0, b1);
+      mma_bf16_16816(o[2 * d2 + 1], al[0], al[1], al[2], al[3], b2, b3);
+      ldmatrix_x4_trans(vl_tile + v_row + d2 * 32, b0, b1, b2, b3);
+      mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
+      mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+    }
+  }
 }
 
-// Combine the warps of the block into the slice's partial result: unnormalised output with its
-// max and sum, written to part_o / part_ml at slot (row0 + q / G, head0 + q % G, split), where a
-// (row, head) owns `slot_stride` consecutive slots.
+// Combine the key groups of the block into the slice's partial result: unnormalised output with
+// its max and sum, written to part_o / part_ml at slot (row0 + q / G, head0 + q % G, split),
+// where a (row, head) owns `slot_stride` consecutive slots.
+constexpr int PK_KGROUPS = 4;
 __device__ __forceinline__ void attn_combine_store(AttnAcc &A, unsigned char *sc, int nQ, int G, int row0, int head0, int nq,
                                                    int slot_stride, int split, float *part_o, float *part_ml) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int kg = warp & 3, dh = warp >> 2;
   float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
   float *const red_m = reinterpret_cast<float *>(sc + PK_AT_RED);
   float *const red_l = red_m + PK_WARPS * PK_QR;
   float (&m_run)[2] = A.m_run;
   float (&l_part)[2] = A.l_part;
-  float (&o)[16][4] = A.o;
-  // combine the warps into this slice's partial result
+  float (&o)[8][4] = A.o;
   pk_sync();                                            // tiles consumed: their space becomes o_s
 #pragma unroll
   for (int hr = 0; hr < 2; ++hr) {
     l_part[hr] += __shfl_xor_sync(0xffffffffu, l_part[hr], 1);
     l_part[hr] += __shfl_xor_sync(0xffffffffu, l_part[hr], 2);
-    if (t == 0) { red_m[warp * PK_QR + g + 8 * hr] = m_run[hr]; red_l[warp * PK_QR + g + 8 * hr] = l_part[hr]; }
+    if (t == 0 && dh == 0) { red_m[kg * PK_QR + g + 8 * hr] = m_run[hr]; red_l[kg * PK_QR + g + 8 * hr] = l_part[hr]; }
   }
-  if (g < nQ) {
 #pragma unroll
-    for (int dt = 0; dt < 16; ++dt)
-      *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][0], o[dt][1]);
-  }
-  if (g + 8 < nQ) {
+  for (int hr = 0; hr < 2; ++hr) {
+    if (g + 8 * hr < nQ) {
+      float *dst = o_s + (kg * PK_QR + g + 8 * hr) * PK_OROW + dh * 64 + 2 * t;
 #pragma unroll
-    for (int dt = 0; dt < 16; ++dt)
-      *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g + 8) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][2], o[dt][3]);
+      for (int dt = 0; dt < 8; ++dt) *reinterpret_cast<float2 *>(dst + dt * 8) = make_float2(o[dt][2 * hr], o[dt][2 * hr + 1]);
+    }
   }
   pk_sync();
-  // per query row: the slice's max and sum, and the factor each warp's share is scaled by
+  // per query row: the slice's max and sum, and the factor each key group's share is scaled by
   if ((int)threadIdx.x < nQ) {
     const int qi = threadIdx.x;
     float m = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < PK_WARPS; ++w) m = fmaxf(m, red_m[w * PK_QR + qi]);
+    for (int w = 0; w < PK_KGROUPS; ++w) m = fmaxf(m, red_m[w * PK_QR + qi]);
     float l = 0.f;
 #pragma unroll
-    for (int w = 0; w < PK_WARPS; ++w) {
+    for (int w = 0; w < PK_KGROUPS; ++w) {
       const float mw = red_m[w * PK_QR + qi];
       const float f = mw > -INFINITY ? __expf(mw - m) : 0.f;
       l += red_l[w * PK_QR + qi] * f;
       red_l[w * PK_QR + qi] = f;
     }
     const size_t slot = ((size_t)(row0 + qi / G) * nq + head0 + qi % G) * slot_stride + split;
-    part_ml[slot * 2] = m;
-    part_ml[slot * 2 + 1] = l;
+    *reinterpret_cast<float2 *>(part_ml + slot * 2) = make_float2(m, l);
   }
   pk_sync();
+#pragma unroll 1
   for (int idx = threadIdx.x; idx < nQ * (PK_D / 4); idx += PK_THREADS) {
     const int qi = idx / (PK_D / 4), d4 = idx % (PK_D / 4);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int w = 0; w < PK_WARPS; ++w) {
+    for (int w = 0; w < PK_KGROUPS; ++w) {
       const float f = red_l[w * PK_QR + qi];
       const float4 v = *reinterpret_cast<const float4 *>(o_s + (w * PK_QR + qi) * PK_OROW + d4 * 4);
       acc.x += v.x * f; acc.y += v.y * f; acc.z += v.z * f; acc.w += v.w * f;
@@ -314,6 +331,7 @@ __device__ __forceinline__ void attn_combine_store(AttnAcc &A, unsigned char *sc
 // that its registers are not counted against the attention loop's.
 __device__ __noinline__ void attn_fetch_f32(const float *k_rows, const float *v_rows, int n_rows, unsigned char *sc) {
   const int total = n_rows * 64;                          // float4 units: 32 of K and 32 of V per row
+#pragma unroll 1
   for (int base = 0; base < total; base += PK_FETCH * PK_THREADS) {
     float4 v[PK_FETCH];
 #pragma unroll
@@ -348,7 +366,6 @@ __device__ __noinline__ void attn_fetch_f32(const float *k_rows, const float *v_
 template <bool PRECISE>
 __device__ __noinline__ void attention_stage(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
   const PassShared S = pass_shared();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int G = P.nq / P.nkv, nQ = R * G;
   int nsplit, CH;
   attn_plan_device(P, pos0, nsplit, CH);
@@ -358,7 +375,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
   unsigned char *const sc = S.bstage;
   const uint32_t kh_tile = smem_u32(sc + PK_AT_KH), kl_tile = smem_u32(sc + PK_AT_KL);
   const uint32_t vh_tile = smem_u32(sc + PK_AT_VH), vl_tile = smem_u32(sc + PK_AT_VL);
-  const uint32_t qh_tile = smem_u32(sc + PK_AT_QH), ql_tile = smem_u32(sc + PK_AT_QL);
+  const uint32_t qh_tile = smem_u32(sc + PK_AT_QH);
   // a 16-byte part (8 values) of a tile row: parts 0..15 are K, 16..31 are V
   auto put_part = [&](int row, int part, const float (&f)[8]) {
     uint4 hi, lo;
@@ -368,6 +385,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     if (PRECISE) sts128((part < 16 ? kl_tile : vl_tile) + off, lo);
   };
 
+#pragma unroll 1
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
     const int split = item % nsplit, kvh = (item / nsplit) % P.nkv, b = item / (nsplit * P.nkv);
     // keys [j0, j1) of the cache, then (last slice) the R keys of the pass
@@ -382,6 +400,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
         // bf16 cache: asynchronous copies, 16 bytes each
         const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(Ly.kc) + head_off;
         const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(Ly.vc) + head_off;
+#pragma unroll 1
         for (int c = threadIdx.x; c < n_c * 32; c += PK_THREADS) {
           const int row = c >> 5, part = c & 31;
           const uint32_t dst = part < 16 ? kh_tile + row * PK_KROW + part * 16 : vh_tile + row * PK_VROW + (part - 16) * 16;
@@ -392,11 +411,13 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
                        reinterpret_cast<const float *>(Ly.vc) + head_off + (size_t)(j0 + tile0) * PK_D, n_c, sc);
       }
     };
+    PK_SUBSTAMP(0);
     pk_sync();                                            // the previous item is done with the scratch
     if (threadIdx.x == 0) {
       // the pass's own q | k | v vectors of this kv head: three bulk copies per row
       const int ldq = (P.nq + 2 * P.nkv) * PK_D;
       stage_begin(S, (uint32_t)(R * (G + 2) * PK_D * 4));
+#pragma unroll 1
       for (int r = 0; r < R; ++r) {
         const float *src = P.qkv + (size_t)(b * R + r) * ldq;
         float *dst = reinterpret_cast<float *>(sc + PK_AT_ROWS) + r * PK_AT_ROW_FLOATS;
@@ -405,22 +426,28 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
         stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
       }
     }
+    PK_SUBSTAMP(1);
     fetch_cached(0);                                      // in flight while the pass's own rows arrive
+    PK_SUBSTAMP(2);
     // query rows beyond nQ are zero (the previous item's partial outputs lay over the Q tiles)
+#pragma unroll 1
     for (int i = threadIdx.x; i < 2 * PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(qh_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
     stage_wait(P, S);
+    PK_SUBSTAMP(3);
     attn_new_rows<PRECISE>(P, Ly, sc, b, kvh, R, pos0, split == 0);
+    PK_SUBSTAMP(4);
 
     AttnAcc A;
     A.m_run[0] = A.m_run[1] = -INFINITY;
     A.l_part[0] = A.l_part[1] = 0.f;
 #pragma unroll
-    for (int dt = 0; dt < 16; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
-    uint4 qh[4][2];
+    for (int dt = 0; dt < 8; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
+#pragma unroll 1
     for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
       const int n_t = min(PK_TK, n_keys - tile0);
       pk_sync();                                          // new rows written / previous tile consumed
       if (tile0 > 0) fetch_cached(tile0);
+#pragma unroll 1
       for (int c = threadIdx.x + max(0, n_cached - tile0) * 32; c < n_t * 32; c += PK_THREADS) {
         const int row = c >> 5, part = c & 31, r = tile0 + row - n_cached;
         const float *src = reinterpret_cast<const float *>(sc + PK_AT_NEW) + ((part < 16 ? 0 : PK_MAX_ROWS) + r) * PK_D + (part & 15) * 8;
@@ -428,6 +455,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
         put_part(row, part, f);
       }
       const int n16 = min(PK_TK, (n_t + 15) & ~15);
+#pragma unroll 1
       for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS) {    // P = 0 times stale bits must stay 0
         const uint32_t off = (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16;
         sts128(vh_tile + off, make_uint4(0u, 0u, 0u, 0u));
@@ -435,20 +463,14 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
       }
       cp_async_wait_all();
       pk_sync();
-      if (tile0 == 0) {
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          qh[kb][0] = lds128(qh_tile + g * PK_QROW + kb * 64 + t * 16);
-          qh[kb][1] = lds128(qh_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
-        }
-      }
-      attn_tile_compute<PRECISE>(A, sc, qh, n_t, tile0, n_cached, j0, pos0, pos0, G);
+      attn_tile_compute<PRECISE>(A, sc, n_t, tile0, n_cached, j0, pos0, pos0, G);
     }
-
-
+    PK_SUBSTAMP(5);
     attn_combine_store(A, sc, nQ, G, b * R, kvh * G, P.nq, PK_NSPLIT_CAP, split, P.part_o, P.part_ml);
+    PK_SUBSTAMP(6);
   }
   pk_sync();
+  PK_SUBSTAMP(7);
 }
 
 }  // namespace dmtd

@@ -16,17 +16,30 @@
 namespace dmtd {
 
 // Profiling builds (-DDMTD_PASS_TIMING) record clock64() of thread 0 of the first and the last
-// block after every prologue, projection and barrier.
+// block after every prologue, projection and barrier; the last four slots of each block hold
+// clock64() and the nanosecond wall clock at kernel entry and at kernel exit, which give the
+// SM clock rate of the launch and the time outside the stamped stages.
 #ifdef DMTD_PASS_TIMING
 constexpr int PK_TIMING_SLOTS = 4096;
 #define PK_STAMP()                                                                                   \
   do {                                                                                               \
     if (threadIdx.x == 0 && P.timing && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) &&          \
-        stamp_n < PK_TIMING_SLOTS)                                                                   \
+        stamp_n < PK_TIMING_SLOTS - 4)                                                               \
       P.timing[(blockIdx.x ? PK_TIMING_SLOTS : 0) + stamp_n++] = clock64();                          \
+  } while (0)
+#define PK_STAMP_WALL(i)                                                                             \
+  do {                                                                                               \
+    if (threadIdx.x == 0 && P.timing && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) {          \
+      long long ns;                                                                                  \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));                                         \
+      long long *t = P.timing + (blockIdx.x ? PK_TIMING_SLOTS : 0) + PK_TIMING_SLOTS - 4 + 2 * (i);  \
+      t[0] = clock64();                                                                              \
+      t[1] = ns;                                                                                     \
+    }                                                                                                \
   } while (0)
 #else
 #define PK_STAMP() do {} while (0)
+#define PK_STAMP_WALL(i) do {} while (0)
 #endif
 
 // out[m][n] += sum_k W[n][k] act[m][k] over this warp's share of W, streamed through its ring.
@@ -161,6 +174,7 @@ __device__ __noinline__ void argmax_final(const PassParams &P) {
 }
 
 __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_constant__ PassParams P) {
+  PK_STAMP_WALL(0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const PassShared S = pass_shared();
   const int nL = P.l_end - P.l_begin;
@@ -284,6 +298,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
       if (clock64() - t0 > P.wait_limit) break;
     pp.consumed += 1;
   }
+  PK_STAMP_WALL(1);
 }
 
 }  // namespace dmtd

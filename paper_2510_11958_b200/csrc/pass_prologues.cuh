@@ -38,6 +38,7 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, H = P.H;
   if (threadIdx.x == 0) {
     stage_begin(S, (uint32_t)(M * H * 4));
+#pragma unroll 1
     for (int m = 0; m < M; ++m) stage_copy(S, S.xs + m * H, x + (size_t)m * row_stride, (uint32_t)(H * 4));
   }
   const SlabSpan sp = slab_span(W);
@@ -50,8 +51,10 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
     if (u < nu) wv[j] = __ldg(reinterpret_cast<const float4 *>(w_norm + sp.first * sp.KS) + u);
   }
   stage_wait(P, S);
+#pragma unroll 1
   for (int m = 0; m < M; ++m) {
     float ss = 0.f;
+#pragma unroll 1
     for (int k4 = threadIdx.x; k4 < H / 4; k4 += PK_THREADS) {
       const float4 v = reinterpret_cast<const float4 *>(S.xs)[m * (H / 4) + k4];
       ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
@@ -60,6 +63,7 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
     if (lane == 0) S.red[warp * PK_MAX_ROWS + m] = ss;
   }
   pk_sync();
+#pragma unroll 1
   for (int m = 0; m < M; ++m) {
     float v = 0.f;
 #pragma unroll
@@ -86,6 +90,7 @@ __device__ __noinline__ void swiglu_prologue(const PassParams &P, int M, const P
   const int ks4 = sp.KS / 4, ldgu = 2 * P.I, total = sp.count * M * ks4;
   if (threadIdx.x == 0) {
     stage_begin(S, (uint32_t)(sp.count * M * 2 * sp.KS * 4));
+#pragma unroll 1
     for (int i = 0; i < sp.count * M; ++i) {             // i = sl * M + m: gate values, then up values
       const float *src = P.gu + (size_t)(i % M) * ldgu + (sp.first + i / M) * sp.KS;
       stage_copy(S, S.xs + (size_t)i * 2 * sp.KS, src, (uint32_t)(sp.KS * 4));
@@ -93,6 +98,7 @@ __device__ __noinline__ void swiglu_prologue(const PassParams &P, int M, const P
     }
   }
   stage_wait(P, S);
+#pragma unroll 1
   for (int idx = threadIdx.x; idx < total; idx += PK_THREADS) {
     const int i = idx / ks4, u4 = idx - i * ks4;
     const float4 g = reinterpret_cast<const float4 *>(S.xs + (size_t)i * 2 * sp.KS)[u4];
@@ -115,6 +121,7 @@ __device__ __noinline__ void merge_prologue(const PassParams &P, int M, int nspl
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const SlabSpan sp = slab_span(W);
   const int heads_per_slab = sp.KS / PK_D, n_heads = sp.count * heads_per_slab;
+#pragma unroll 1
   for (int pair = warp; pair < M * n_heads; pair += PK_WARPS) {
     const int m = pair / n_heads, hh = pair - m * n_heads;
     const int sl = hh / heads_per_slab, h = sp.first * heads_per_slab + hh;
@@ -123,6 +130,7 @@ __device__ __noinline__ void merge_prologue(const PassParams &P, int M, int nspl
     if (lane < nsplit) ml = __ldcg(reinterpret_cast<const float2 *>(P.part_ml) + slot0 + lane);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float wgt = 0.f;
+#pragma unroll 1
     for (int s0 = 0; s0 < nsplit; s0 += PK_MERGE_BATCH) {
       float4 po[PK_MERGE_BATCH];
 #pragma unroll
@@ -148,6 +156,7 @@ __device__ __noinline__ void merge_prologue(const PassParams &P, int M, int nspl
 // grid (row m = b*R + r sits at position pos0 + r).  Readers wait for the next grid barrier.
 __device__ __noinline__ void embed_rows(const PassParams &P, float *x, int M, int R, int pos0) {
   const int units = P.H / 8;
+#pragma unroll 1
   for (int i = blockIdx.x * PK_THREADS + threadIdx.x; i < M * units; i += gridDim.x * PK_THREADS) {
     const int m = i / units, u = i - m * units;
     int tok = P.tokens[(size_t)(m / R) * P.max_seq + pos0 + m % R];
@@ -167,6 +176,7 @@ __device__ __noinline__ void embed_rows(const PassParams &P, float *x, int M, in
 // row of the decoding layers (Section 2.2: only that row goes on); spread over the grid.
 __device__ __forceinline__ void select_rows(const PassParams &P) {
   const int h4 = P.H / 4;
+#pragma unroll 1
   for (int i = blockIdx.x * PK_THREADS + threadIdx.x; i < P.B * h4; i += gridDim.x * PK_THREADS) {
     const int b = i / h4, k4 = i - b * h4;
     reinterpret_cast<float4 *>(P.x_up)[(size_t)b * h4 + k4] =

@@ -175,6 +175,7 @@ __device__ __forceinline__ SlabSpan slab_span(const PackedMat &W) {
 
 // Clear `n` floats, the work spread over the grid.
 __device__ __forceinline__ void grid_zero(float *p, int n) {
+#pragma unroll 1
   for (int i = (blockIdx.x * PK_THREADS + threadIdx.x) * 4; i < n; i += gridDim.x * PK_THREADS * 4) {
     if (i + 4 <= n) {
       *reinterpret_cast<float4 *>(p + i) = make_float4(0.f, 0.f, 0.f, 0.f);

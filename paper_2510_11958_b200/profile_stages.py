@@ -80,6 +80,13 @@ def main():
               " ".join(f"{nm}={per[1:, i].mean():.1f}" for i, nm in enumerate(NAMES) if nm != "-") +
               f" | sum {per[1:].mean(0).sum():.1f}")
         print("  head: prologue %.1f, projection %.1f, barrier %.1f" % tuple(d[n_layers * 15: n_layers * 15 + 3]))
+        if blk == 0:
+            a = s[SLOTS - 20:SLOTS - 12]
+            print("  inside the last layer's attention stage (entry, rows requested, cached tile fetched, rows landed, "
+                  "rows normed, tiles done, partials stored, exit): " + " ".join(f"{v / (args.ghz * 1e3):.2f}" for v in np.diff(a)))
+        c0, w0, c1, w1 = (int(v) for v in s[SLOTS - 4:])
+        print(f"  kernel entry to exit: {(w1 - w0) / 1e3:.1f} us by the wall clock, SM clock {(c1 - c0) / max(w1 - w0, 1):.3f} GHz; "
+              f"entry to first stamp {(s[0] - c0) / (args.ghz * 1e3):.1f} us, last stamp to exit {(c1 - s[n - 1]) / (args.ghz * 1e3):.1f} us")
 
 
 if __name__ == "__main__":
