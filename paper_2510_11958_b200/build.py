@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libdmtd_b200.so")
 SOURCES = ["engine.cu"]
 HEADERS = ["common.cuh", "kernels.cuh", "pass_common.cuh", "pass_stream.cuh", "pass_prologues.cuh",
-           "pass_attention.cuh", "pass_kernel.cuh", "attention_kernel.cuh", "gemm_tc05.cuh"]
+           "pass_attention.cuh", "pass_attention_f32.cuh", "pass_kernel.cuh", "attention_kernel.cuh", "gemm_tc05.cuh"]
 
 
 def _stale() -> bool:

@@ -446,6 +446,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
       const int n_t = min(PK_TK, n_keys - tile0);
       pk_sync();                                          // new rows written / previous tile consumed
+      PK_SUBSTAMP(8);
       if (tile0 > 0) fetch_cached(tile0);
 #pragma unroll 1
       for (int c = threadIdx.x + max(0, n_cached - tile0) * 32; c < n_t * 32; c += PK_THREADS) {
@@ -461,8 +462,10 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
         sts128(vh_tile + off, make_uint4(0u, 0u, 0u, 0u));
         if (PRECISE) sts128(vl_tile + off, make_uint4(0u, 0u, 0u, 0u));
       }
+      PK_SUBSTAMP(9);
       cp_async_wait_all();
       pk_sync();
+      PK_SUBSTAMP(10);
       attn_tile_compute<PRECISE>(A, sc, n_t, tile0, n_cached, j0, pos0, pos0, G);
     }
     PK_SUBSTAMP(5);

@@ -1,0 +1,276 @@
+// Attention stage of the pass kernel for an fp32 KV cache: steps a3 (QK-norm, rotary embedding,
+// KV append) and a4 (split-KV attention) in plain fp32 FMAs.
+//
+// With an fp32 cache the tensor-core form needs three mma.sync per product (bf16 hi/lo pairs),
+// and mma.sync issues slowly on this GPU (measured: about 30 cycles per m16n8k16 per SM
+// sub-partition, 2.2 us for one 64-key tile); the same tile is 0.26 M FMAs at most, the K and V
+// tiles stay fp32 in shared memory (no splitting, so they arrive by asynchronous copies), and the
+// result is exact fp32 arithmetic.
+#pragma once
+
+#include "pass_attention.cuh"
+
+namespace dmtd {
+
+constexpr int PK_F_KROW = 576;                                   // bytes per K row: 512 + 64, conflict-free 16-byte reads by (key, part) lanes
+constexpr int PK_F_K = 0;                                        // K tile [PK_TK][PK_F_KROW]
+constexpr int PK_F_V = PK_F_K + PK_TK * PK_F_KROW;               // V tile [PK_TK][128] floats
+constexpr int PK_F_Q = PK_F_V + PK_TK * PK_D * 4;                // Q [PK_QR][128] floats, scaled by 1/sqrt(d)
+constexpr int PK_F_S = PK_F_Q + PK_QR * PK_D * 4;                // scores, then probabilities [PK_TK][PK_QR]
+constexpr int PK_F_STAT = PK_F_S + PK_TK * PK_QR * 4;            // running max, running sum, rescale factor [3][PK_QR]
+constexpr int PK_F_NEW = PK_F_STAT + 3 * PK_QR * 4;              // K rows of the pass [4][128], then V rows [4][128]
+constexpr int PK_F_W = PK_F_NEW + 2 * PK_MAX_ROWS * PK_D * 4;    // q-norm weights, k-norm weights (floats), rotary frequencies (doubles)
+constexpr int PK_F_END = PK_F_W + 2 * PK_D * 4 + (PK_D / 2) * 8;
+static_assert(PK_F_END <= PK_AT_ROWS, "fp32 attention scratch overlaps the row staging area");
+static_assert(PK_WARPS * PK_QR * PK_OROW * 4 <= PK_F_Q, "partial-output overlay reaches Q");
+
+// QK-norm (Section 3.1's Qwen3 block) and the half-split rotary embedding of one head vector,
+// one value per lane and quarter: v[j] is element lane + 32 j.
+__device__ __forceinline__ void head_norm_rope(const float *w, const double *inv_freq, float eps, float scale, int pos,
+                                               int lane, float (&v)[4]) {
+  float ss = v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
+  ss = warp_sum(ss);
+  const float inv = rsqrtf(ss / (float)PK_D + eps) * scale;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) v[j] = v[j] * inv * w[lane + 32 * j];
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    // angle reduced to [-pi, pi] in double, then the fast sine and cosine
+    double a = (double)pos * inv_freq[lane + 32 * j];
+    a -= 6.283185307179586 * rint(a * 0.15915494309189535);
+    float sn, cs;
+    __sincosf((float)a, &sn, &cs);
+    const float x0 = v[j], x1 = v[j + 2];
+    v[j] = x0 * cs - x1 * sn;
+    v[j + 2] = x1 * cs + x0 * sn;
+  }
+}
+
+// Step a3 for one (sequence, kv head): one warp per head vector of the pass's rows.
+__device__ __forceinline__ void attn_new_rows_f32(const PassParams &P, const PassLayer &Ly, unsigned char *sc, int b, int kvh,
+                                                  int R, int pos0, bool write_cache) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = P.nq / P.nkv, nQ = R * G;
+  const float *rows = reinterpret_cast<const float *>(sc + PK_AT_ROWS);
+  const float *w_q = reinterpret_cast<const float *>(sc + PK_F_W), *w_k = w_q + PK_D;
+  const double *inv_freq = reinterpret_cast<const double *>(sc + PK_F_W + 2 * PK_D * 4);
+  const float scale = rsqrtf((float)PK_D);
+#pragma unroll 1
+  for (int task = warp; task < nQ + 2 * R; task += PK_WARPS) {
+    int r, col, kind;                                   // kind 0 q, 1 k, 2 v
+    if (task < nQ) { r = task / G; col = (task % G) * PK_D; kind = 0; }
+    else if (task < nQ + R) { r = task - nQ; col = G * PK_D; kind = 1; }
+    else { r = task - nQ - R; col = (G + 1) * PK_D; kind = 2; }
+    const float *src = rows + r * PK_AT_ROW_FLOATS + col;
+    float v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = src[lane + 32 * j];
+    if (kind != 2) head_norm_rope(kind == 0 ? w_q : w_k, inv_freq, P.eps, kind == 0 ? scale : 1.f, pos0 + r, lane, v);
+    float *dst;
+    if (kind == 0) dst = reinterpret_cast<float *>(sc + PK_F_Q) + task * PK_D;
+    else dst = reinterpret_cast<float *>(sc + PK_F_NEW) + ((kind == 2 ? PK_MAX_ROWS : 0) + r) * PK_D;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) dst[lane + 32 * j] = v[j];
+    if (kind != 0 && write_cache) {
+      float *cache = reinterpret_cast<float *>(kind == 1 ? Ly.kc : Ly.vc) +
+                     (((size_t)b * P.nkv + kvh) * P.max_seq + pos0 + r) * PK_D;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) cache[lane + 32 * j] = v[j];
+    }
+  }
+}
+
+__device__ __forceinline__ float4 lds_f4(const unsigned char *p) { return *reinterpret_cast<const float4 *>(p); }
+
+// Steps a3 + a4 for the items (sequence, kv head, key slice) of this block, fp32 cache.
+// Per 64-key tile: scores by (key, quarter-of-d) threads with the K row in registers; softmax
+// statistics by one warp per query row; P V by (key group = warp, 4 output dims = lane) threads.
+__device__ __noinline__ void attention_stage_f32(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
+  const PassShared S = pass_shared();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = P.nq / P.nkv, nQ = R * G;
+  int nsplit, CH;
+  attn_plan_device(P, pos0, nsplit, CH);
+  const int items = P.B * P.nkv * nsplit;
+  if ((int)blockIdx.x >= items) return;
+  unsigned char *const sc = S.bstage;
+  float *const sm_s = reinterpret_cast<float *>(sc + PK_F_S);
+  float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR, *const corr = l_run + PK_QR;
+
+#pragma unroll 1
+  for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    const int split = item % nsplit, kvh = (item / nsplit) % P.nkv, b = item / (nsplit * P.nkv);
+    // keys [j0, j1) of the cache, then (last slice) the R keys of the pass
+    const int j0 = split * CH, j1 = min(j0 + CH, pos0);
+    const int n_cached = max(0, j1 - j0);
+    const int n_keys = n_cached + (split == nsplit - 1 ? R : 0);
+    const float *kc = reinterpret_cast<const float *>(Ly.kc) + (((size_t)b * P.nkv + kvh) * P.max_seq + j0) * PK_D;
+    const float *vc = reinterpret_cast<const float *>(Ly.vc) + (((size_t)b * P.nkv + kvh) * P.max_seq + j0) * PK_D;
+    PK_SUBSTAMP(0);
+    pk_sync();                                            // the previous item is done with the scratch
+    if (threadIdx.x == 0) {
+      // the pass's own q | k | v vectors of this kv head, the two norm weights and the rotary frequencies
+      const int ldq = (P.nq + 2 * P.nkv) * PK_D;
+      stage_begin(S, (uint32_t)(R * (G + 2) * PK_D * 4 + 2 * PK_D * 4 + (PK_D / 2) * 8));
+#pragma unroll 1
+      for (int r = 0; r < R; ++r) {
+        const float *src = P.qkv + (size_t)(b * R + r) * ldq;
+        float *dst = reinterpret_cast<float *>(sc + PK_AT_ROWS) + r * PK_AT_ROW_FLOATS;
+        stage_copy(S, dst, src + kvh * G * PK_D, (uint32_t)(G * PK_D * 4));
+        stage_copy(S, dst + G * PK_D, src + (P.nq + kvh) * PK_D, PK_D * 4);
+        stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
+      }
+      stage_copy(S, sc + PK_F_W, Ly.w_qn, PK_D * 4);
+      stage_copy(S, sc + PK_F_W + PK_D * 4, Ly.w_kn, PK_D * 4);
+      stage_copy(S, sc + PK_F_W + 2 * PK_D * 4, P.inv_freq, (PK_D / 2) * 8);
+    }
+    PK_SUBSTAMP(1);
+    // cached rows of a tile: asynchronous 16-byte copies, 32 of K and 32 of V per row
+    auto fetch_cached = [&](int tile0) {
+      const int n_c = min(PK_TK, n_cached - tile0);
+#pragma unroll 1
+      for (int c = threadIdx.x; c < n_c * 64; c += PK_THREADS) {
+        const int row = c >> 6, u = c & 63;
+        const uint32_t dst = smem_u32(sc) + (u < 32 ? PK_F_K + row * PK_F_KROW + u * 16 : PK_F_V + row * PK_D * 4 + (u - 32) * 16);
+        cp_async16(dst, (u < 32 ? kc : vc) + (size_t)(tile0 + row) * PK_D + (u & 31) * 4);
+      }
+    };
+    fetch_cached(0);                                      // in flight while the pass's own rows arrive
+    PK_SUBSTAMP(2);
+    if ((int)threadIdx.x < PK_QR) { m_run[threadIdx.x] = -INFINITY; l_run[threadIdx.x] = 0.f; }
+    stage_wait(P, S);
+    PK_SUBSTAMP(3);
+    attn_new_rows_f32(P, Ly, sc, b, kvh, R, pos0, split == 0);
+    PK_SUBSTAMP(4);
+
+    float acc[PK_QR][4];
+#pragma unroll
+    for (int q = 0; q < PK_QR; ++q) acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f;
+#pragma unroll 1
+    for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
+      const int n_t = min(PK_TK, n_keys - tile0);
+      pk_sync();                                          // new rows written / previous tile consumed
+      PK_SUBSTAMP(8);
+      if (tile0 > 0) fetch_cached(tile0);
+      // the pass's own rows that fall into this tile
+#pragma unroll 1
+      for (int c = threadIdx.x + max(0, n_cached - tile0) * 64; c < n_t * 64; c += PK_THREADS) {
+        const int row = c >> 6, u = c & 63, r = tile0 + row - n_cached;
+        const float4 val = lds_f4(sc + PK_F_NEW + (((u < 32 ? 0 : PK_MAX_ROWS) + r) * PK_D + (u & 31) * 4) * 4);
+        *reinterpret_cast<float4 *>(sc + (u < 32 ? PK_F_K + row * PK_F_KROW + u * 16 : PK_F_V + row * PK_D * 4 + (u - 32) * 16)) = val;
+      }
+      PK_SUBSTAMP(9);
+      cp_async_wait_all();
+      pk_sync();
+      PK_SUBSTAMP(10);
+      {
+        // scores: thread = (key, part); part p holds the 16-byte units p, p + 4, .. of the K row
+        // (every lane runs the loop, since the four parts of a key meet in warp shuffles; keys
+        // beyond the tile read row 0 and store nothing)
+        const int key = threadIdx.x >> 2, part = threadIdx.x & 3;
+        const bool live = key < n_t;
+        {
+          float4 kr[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) kr[j] = lds_f4(sc + PK_F_K + (live ? key : 0) * PK_F_KROW + (part + 4 * j) * 16);
+          const int idx = tile0 + key;
+          const int key_pos = idx < n_cached ? j0 + idx : pos0 + (idx - n_cached);
+          int r = 0, h = 0;
+#pragma unroll 1
+          for (int q = 0; q < nQ; ++q) {
+            const unsigned char *qp = sc + PK_F_Q + q * PK_D * 4 + part * 16;
+            float s = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float4 qv = lds_f4(qp + j * 64);
+              s += kr[j].x * qv.x + kr[j].y * qv.y + kr[j].z * qv.z + kr[j].w * qv.w;
+            }
+            s += __shfl_xor_sync(0xffffffffu, s, 1);
+            s += __shfl_xor_sync(0xffffffffu, s, 2);
+            if (live && part == 0) sm_s[key * PK_QR + q] = key_pos <= pos0 + r ? s : -INFINITY;
+            if (++h == G) { h = 0; ++r; }
+          }
+        }
+      }
+      PK_SUBSTAMP(11);
+      pk_sync();
+      PK_SUBSTAMP(12);
+      // per query row: the tile's max joins the running max; scores become probabilities
+#pragma unroll 1
+      for (int q = warp; q < nQ; q += PK_WARPS) {
+        const float v0 = lane < n_t ? sm_s[lane * PK_QR + q] : -INFINITY;
+        const float v1 = lane + 32 < n_t ? sm_s[(lane + 32) * PK_QR + q] : -INFINITY;
+        const float m_old = m_run[q];
+        const float m_new = fmaxf(m_old, warp_max(fmaxf(v0, v1)));
+        const float p0 = v0 > -INFINITY ? __expf(v0 - m_new) : 0.f;
+        const float p1 = v1 > -INFINITY ? __expf(v1 - m_new) : 0.f;
+        sm_s[lane * PK_QR + q] = p0;
+        sm_s[(lane + 32) * PK_QR + q] = p1;
+        const float ps = warp_sum(p0 + p1);
+        if (lane == 0) {
+          const float f = m_old > -INFINITY ? __expf(m_old - m_new) : 0.f;
+          corr[q] = f;
+          l_run[q] = l_run[q] * f + ps;
+          m_run[q] = m_new;
+        }
+      }
+      PK_SUBSTAMP(13);
+      pk_sync();
+      PK_SUBSTAMP(14);
+      // O += P V: warp = key group (keys warp, warp + 8, ..), lane = 4 output dimensions
+#pragma unroll
+      for (int q = 0; q < PK_QR; ++q) {
+        if (q < nQ) {
+          const float f = corr[q];
+          acc[q][0] *= f; acc[q][1] *= f; acc[q][2] *= f; acc[q][3] *= f;
+        }
+      }
+#pragma unroll 1
+      for (int key = warp; key < n_t; key += PK_WARPS) {
+        const float4 vv = lds_f4(sc + PK_F_V + (key * PK_D + lane * 4) * 4);
+#pragma unroll
+        for (int q4 = 0; q4 < PK_QR / 4; ++q4) {
+          if (q4 * 4 < nQ) {
+            const float4 pv = lds_f4(sc + PK_F_S + (key * PK_QR + q4 * 4) * 4);
+            const float pq[4] = {pv.x, pv.y, pv.z, pv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              acc[q4 * 4 + e][0] += pq[e] * vv.x; acc[q4 * 4 + e][1] += pq[e] * vv.y;
+              acc[q4 * 4 + e][2] += pq[e] * vv.z; acc[q4 * 4 + e][3] += pq[e] * vv.w;
+            }
+          }
+        }
+      }
+    }
+    PK_SUBSTAMP(5);
+    // the slice's partial result: the key groups' outputs summed, with the running max and sum
+    float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
+    pk_sync();                                            // tiles consumed: their space becomes o_s
+#pragma unroll
+    for (int q = 0; q < PK_QR; ++q)
+      if (q < nQ) *reinterpret_cast<float4 *>(o_s + (warp * PK_QR + q) * PK_OROW + lane * 4) = make_float4(acc[q][0], acc[q][1], acc[q][2], acc[q][3]);
+    pk_sync();
+    if ((int)threadIdx.x < nQ) {
+      const int qi = threadIdx.x;
+      const size_t slot = ((size_t)(b * R + qi / G) * P.nq + kvh * G + qi % G) * PK_NSPLIT_CAP + split;
+      *reinterpret_cast<float2 *>(P.part_ml + slot * 2) = make_float2(m_run[qi], l_run[qi]);
+    }
+#pragma unroll 1
+    for (int idx = threadIdx.x; idx < nQ * (PK_D / 4); idx += PK_THREADS) {
+      const int qi = idx / (PK_D / 4), d4 = idx % (PK_D / 4);
+      float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int w = 0; w < PK_WARPS; ++w) {
+        const float4 v = *reinterpret_cast<const float4 *>(o_s + (w * PK_QR + qi) * PK_OROW + d4 * 4);
+        sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+      }
+      const size_t slot = ((size_t)(b * R + qi / G) * P.nq + kvh * G + qi % G) * PK_NSPLIT_CAP + split;
+      *reinterpret_cast<float4 *>(P.part_o + slot * PK_D + d4 * 4) = sum;
+    }
+    PK_SUBSTAMP(6);
+  }
+  pk_sync();
+  PK_SUBSTAMP(7);
+}
+
+}  // namespace dmtd

@@ -39,6 +39,7 @@ def main():
     ap.add_argument("--kind", default="full", choices=["full", "upper"])
     ap.add_argument("--ghz", type=float, default=1.965)
     ap.add_argument("--kv", default=None, choices=["bf16", "f32"], help="KV cache type (default: the workload's)")
+    ap.add_argument("--prompt-len", type=int, default=None, help="prompt length (default: the workload's)")
     ap.add_argument("--build-only", action="store_true")
     args = ap.parse_args()
     build_timing_library()
@@ -50,6 +51,9 @@ def main():
     from synthetic import SHAPES, WORKLOADS, make_prompts, make_weights
     bd.library_path = lambda: LIB
     wl = WORKLOADS[args.workload]
+    if args.prompt_len:
+        import dataclasses
+        wl = dataclasses.replace(wl, prompt_len=args.prompt_len)
     shape = SHAPES[wl.shape]
     w = make_weights(shape, seed=wl.weight_seed, device="cuda")
     eng = bd.Dmtd(shape, w, L_d=wl.L_d, tau=wl.tau, max_batch=wl.batch, max_seq=wl.prompt_len + 64,
@@ -84,6 +88,12 @@ def main():
             a = s[SLOTS - 20:SLOTS - 12]
             print("  inside the last layer's attention stage (entry, rows requested, cached tile fetched, rows landed, "
                   "rows normed, tiles done, partials stored, exit): " + " ".join(f"{v / (args.ghz * 1e3):.2f}" for v in np.diff(a)))
+            t = s[SLOTS - 12:SLOTS - 5]
+            print("  last tile: sync %.2f, new rows placed %.2f, copies landed + sync %.2f, multiplied %.2f" %
+                  tuple(v / (args.ghz * 1e3) for v in (t[0] - a[4], t[1] - t[0], t[2] - t[1], a[5] - t[2])))
+            if t[6] > t[2]:
+                print("  multiplied = scores %.2f, sync %.2f, softmax %.2f, sync %.2f, P V %.2f (fp32 cache only)" %
+                      tuple(v / (args.ghz * 1e3) for v in (t[3] - t[2], t[4] - t[3], t[5] - t[4], t[6] - t[5], a[5] - t[6])))
         c0, w0, c1, w1 = (int(v) for v in s[SLOTS - 4:])
         print(f"  kernel entry to exit: {(w1 - w0) / 1e3:.1f} us by the wall clock, SM clock {(c1 - c0) / max(w1 - w0, 1):.3f} GHz; "
               f"entry to first stamp {(s[0] - c0) / (args.ghz * 1e3):.1f} us, last stamp to exit {(c1 - s[n - 1]) / (args.ghz * 1e3):.1f} us")
