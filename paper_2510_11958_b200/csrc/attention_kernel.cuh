@@ -10,6 +10,183 @@
 
 namespace dmtd {
 
+// Work layout of this kernel's tiles: each of the first four warps takes 16 keys of a 64-key tile
+// against all 128 output dimensions, with the Q fragments in registers.  (The pass kernel's
+// attention stage spreads one tile over all eight warps, two per key group, which halves the
+// latency of its single tile but repeats the Q K^T products; here, where tiles follow one another
+// and mma.sync issue is the limit, the repeated products cost 10 % of the throughput.)
+// One 64-key tile against the 16 query rows: this warp's 16 keys.  acc holds the warp's running
+// max, running sum (per lane, summed over the four lanes of a row at the end) and output.
+struct AttnAccW {
+  float m_run[2], l_part[2];
+  float o[16][4];
+};
+
+// Keys of the tile are key_idx0 + row; key index i sits at position (i < n_cached ? j0 + i :
+// pos_new + i - n_cached); query row q may see positions up to row_pos0 + q / G.
+// k_off / v_off: where the tile's K and V (hi parts) sit in the scratch.
+template <bool PRECISE>
+__device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *sc, const uint4 (&qh)[4][2], int n_t, int tile0,
+                                                  int n_cached, int j0, int pos_new, int row_pos0, int G,
+                                                  int k_off = PK_AT_KH, int v_off = PK_AT_VH) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const uint32_t kh_tile = smem_u32(sc + k_off), kl_tile = smem_u32(sc + PK_AT_KL);
+  const uint32_t vh_tile = smem_u32(sc + v_off), vl_tile = smem_u32(sc + PK_AT_VL);
+  const uint32_t ql_tile = smem_u32(sc + PK_AT_QL);
+  float (&m_run)[2] = A.m_run;
+  float (&l_part)[2] = A.l_part;
+  float (&o)[16][4] = A.o;
+  if (warp * 16 < n_t) {
+        float c[2][4];
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+          c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+#pragma unroll
+          for (int kb = 0; kb < 4; ++kb) {
+            const uint32_t off = (warp * 16 + nt * 8 + g) * PK_KROW + kb * 64 + t * 16;
+            const uint4 Kh = lds128(kh_tile + off);
+            mma_bf16_16816(c[nt], qh[kb][0].x, qh[kb][1].x, qh[kb][0].y, qh[kb][1].y, Kh.x, Kh.y);
+            mma_bf16_16816(c[nt], qh[kb][0].z, qh[kb][1].z, qh[kb][0].w, qh[kb][1].w, Kh.z, Kh.w);
+            if (PRECISE) {
+              // the lo parts of Q stay in shared memory: registers are short here
+              const uint4 Kl = lds128(kl_tile + off);
+              const uint4 q0 = lds128(ql_tile + g * PK_QROW + kb * 64 + t * 16);
+              const uint4 q1 = lds128(ql_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
+              mma_bf16_16816(c[nt], qh[kb][0].x, qh[kb][1].x, qh[kb][0].y, qh[kb][1].y, Kl.x, Kl.y);
+              mma_bf16_16816(c[nt], qh[kb][0].z, qh[kb][1].z, qh[kb][0].w, qh[kb][1].w, Kl.z, Kl.w);
+              mma_bf16_16816(c[nt], q0.x, q1.x, q0.y, q1.y, Kh.x, Kh.y);
+              mma_bf16_16816(c[nt], q0.z, q1.z, q0.w, q1.w, Kh.z, Kh.w);
+            }
+          }
+        }
+        // causal / range mask: lane holds rows g (e = 0, 1) and g + 8 (e = 2, 3), keys 2t, 2t + 1 of each n-tile
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int kl = warp * 16 + nt * 8 + 2 * t + (e & 1), idx = tile0 + kl, row = g + (e >> 1) * 8;
+            const int key_pos = idx < n_cached ? j0 + idx : pos_new + (idx - n_cached);
+            const bool ok = kl < n_t && key_pos <= row_pos0 + row / G;
+            c[nt][e] = ok ? c[nt][e] : -INFINITY;
+            mx[e >> 1] = fmaxf(mx[e >> 1], c[nt][e]);
+          }
+        }
+        float corr[2];
+#pragma unroll
+        for (int hr = 0; hr < 2; ++hr) {
+          mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 1));
+          mx[hr] = fmaxf(mx[hr], __shfl_xor_sync(0xffffffffu, mx[hr], 2));
+          const float m_new = fmaxf(m_run[hr], mx[hr]);
+          corr[hr] = m_new > -INFINITY ? __expf(m_run[hr] - m_new) : 1.f;
+          m_run[hr] = m_new;
+        }
+        float psum[2] = {0.f, 0.f};
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float p = c[nt][e] > -INFINITY ? __expf(c[nt][e] - m_run[e >> 1]) : 0.f;
+            c[nt][e] = p;
+            psum[e >> 1] += p;
+          }
+        }
+        l_part[0] = l_part[0] * corr[0] + psum[0];
+        l_part[1] = l_part[1] * corr[1] + psum[1];
+        // P as the A operand: hi parts and (fp32 cache) lo parts
+        uint32_t ah[4], al[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float p0 = c[i >> 1][(i & 1) * 2], p1 = c[i >> 1][(i & 1) * 2 + 1];
+          ah[i] = pack_bf16x2(p0, p1);
+          if (PRECISE) al[i] = pack_bf16x2(p0 - __uint_as_float(ah[i] << 16), p1 - __uint_as_float(ah[i] & 0xffff0000u));
+        }
+        const int mi = lane >> 3, rr = lane & 7;
+        const uint32_t v_off = (warp * 16 + (mi & 1) * 8 + rr) * PK_VROW + (mi >> 1) * 16;
+#pragma unroll
+        for (int d2 = 0; d2 < 8; ++d2) {
+          uint32_t b0, b1, b2, b3;
+          ldmatrix_x4_trans(vh_tile + v_off + d2 * 32, b0, b1, b2, b3);
+          o[2 * d2][0] *= corr[0]; o[2 * d2][1] *= corr[0]; o[2 * d2][2] *= corr[1]; o[2 * d2][3] *= corr[1];
+          o[2 * d2 + 1][0] *= corr[0]; o[2 * d2 + 1][1] *= corr[0]; o[2 * d2 + 1][2] *= corr[1]; o[2 * d2 + 1][3] *= corr[1];
+          mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
+          mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+          if (PRECISE) {
+            mma_bf16_16816(o[2 * d2], al[0], al[1], al[2], al[3], b0, b1);
+            mma_bf16_16816(o[2 * d2 + 1], al[0], al[1], al[2], al[3], b2, b3);
+            ldmatrix_x4_trans(vl_tile + v_off + d2 * 32, b0, b1, b2, b3);
+            mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
+            mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+          }
+        }
+      }
+}
+
+// Combine the warps of the block into the slice's partial result: unnormalised output with its
+// max and sum, written to part_o / part_ml at slot (row0 + q / G, head0 + q % G, split), where a
+// (row, head) owns `slot_stride` consecutive slots.
+__device__ __forceinline__ void attn_combine_store_w(AttnAccW &A, unsigned char *sc, int nQ, int G, int row0, int head0, int nq,
+                                                   int slot_stride, int split, float *part_o, float *part_ml) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
+  float *const red_m = reinterpret_cast<float *>(sc + PK_AT_RED);
+  float *const red_l = red_m + PK_WARPS * PK_QR;
+  float (&m_run)[2] = A.m_run;
+  float (&l_part)[2] = A.l_part;
+  float (&o)[16][4] = A.o;
+  // combine the warps into this slice's partial result
+  pk_sync();                                            // tiles consumed: their space becomes o_s
+#pragma unroll
+  for (int hr = 0; hr < 2; ++hr) {
+    l_part[hr] += __shfl_xor_sync(0xffffffffu, l_part[hr], 1);
+    l_part[hr] += __shfl_xor_sync(0xffffffffu, l_part[hr], 2);
+    if (t == 0) { red_m[warp * PK_QR + g + 8 * hr] = m_run[hr]; red_l[warp * PK_QR + g + 8 * hr] = l_part[hr]; }
+  }
+  if (g < nQ) {
+#pragma unroll
+    for (int dt = 0; dt < 16; ++dt)
+      *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][0], o[dt][1]);
+  }
+  if (g + 8 < nQ) {
+#pragma unroll
+    for (int dt = 0; dt < 16; ++dt)
+      *reinterpret_cast<float2 *>(o_s + (warp * PK_QR + g + 8) * PK_OROW + dt * 8 + 2 * t) = make_float2(o[dt][2], o[dt][3]);
+  }
+  pk_sync();
+  // per query row: the slice's max and sum, and the factor each warp's share is scaled by
+  if ((int)threadIdx.x < nQ) {
+    const int qi = threadIdx.x;
+    float m = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < PK_WARPS; ++w) m = fmaxf(m, red_m[w * PK_QR + qi]);
+    float l = 0.f;
+#pragma unroll
+    for (int w = 0; w < PK_WARPS; ++w) {
+      const float mw = red_m[w * PK_QR + qi];
+      const float f = mw > -INFINITY ? __expf(mw - m) : 0.f;
+      l += red_l[w * PK_QR + qi] * f;
+      red_l[w * PK_QR + qi] = f;
+    }
+    const size_t slot = ((size_t)(row0 + qi / G) * nq + head0 + qi % G) * slot_stride + split;
+    part_ml[slot * 2] = m;
+    part_ml[slot * 2 + 1] = l;
+  }
+  pk_sync();
+  for (int idx = threadIdx.x; idx < nQ * (PK_D / 4); idx += PK_THREADS) {
+    const int qi = idx / (PK_D / 4), d4 = idx % (PK_D / 4);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int w = 0; w < PK_WARPS; ++w) {
+      const float f = red_l[w * PK_QR + qi];
+      const float4 v = *reinterpret_cast<const float4 *>(o_s + (w * PK_QR + qi) * PK_OROW + d4 * 4);
+      acc.x += v.x * f; acc.y += v.y * f; acc.z += v.z * f; acc.w += v.w * f;
+    }
+    const size_t slot = ((size_t)(row0 + qi / G) * nq + head0 + qi % G) * slot_stride + split;
+    *reinterpret_cast<float4 *>(part_o + slot * PK_D + d4 * 4) = acc;
+  }
+}
+
+
 constexpr int ATTN_TC_SMEM = PK_AT_ROWS;         // tiles, Q, partial-output overlay, reduction arrays
 
 // qkv [B*R][ldq]: q heads already normalised and rotated (not scaled); K and V of the new rows
@@ -20,7 +197,7 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
                int nq, int nkv, int R, int RB, int CH, const int *__restrict__ pos0_ptr, float *__restrict__ part_o,
                float *__restrict__ part_ml, int nsplit) {
   extern __shared__ __align__(1024) unsigned char sc[];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int G = nq / nkv, n_rb = (R + RB - 1) / RB;
   const int split = blockIdx.x, kvh = blockIdx.y / n_rb, rb = blockIdx.y % n_rb, b = blockIdx.z;
   const int r0 = rb * RB, r1 = min(R, r0 + RB), nQ = (r1 - r0) * G;
@@ -53,11 +230,12 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
     }
   }
   const size_t head_off = ((size_t)b * nkv + kvh) * max_seq * PK_D;
-  AttnAcc A;
+  AttnAccW A;
   A.m_run[0] = A.m_run[1] = -INFINITY;
   A.l_part[0] = A.l_part[1] = 0.f;
 #pragma unroll
-  for (int dt = 0; dt < 8; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
+  for (int dt = 0; dt < 16; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
+  uint4 qh[4][2];
   const int n_keys = j1 - j0;
   if (!PRECISE) {
     // bf16 cache: two tile buffers (the lo-part areas are free here), tile i+1 in flight while
@@ -88,7 +266,14 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
         asm volatile("cp.async.wait_group 0;" ::: "memory");
       }
       __syncthreads();                                    // tile (and, the first time, Q) visible to all
-      attn_tile_compute<false>(A, sc, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH,
+      if (tile0 == 0) {
+#pragma unroll
+        for (int kbk = 0; kbk < 4; ++kbk) {
+          qh[kbk][0] = lds128(qh_tile + g * PK_QROW + kbk * 64 + t * 16);
+          qh[kbk][1] = lds128(qh_tile + (g + 8) * PK_QROW + kbk * 64 + t * 16);
+        }
+      }
+      attn_tile_compute_w<false>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH,
                                buf ? PK_AT_VL : PK_AT_VH);
       __syncthreads();                                    // done with this buffer before it is refilled
     }
@@ -116,11 +301,18 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
       }
       cp_async_wait_all();
       __syncthreads();
+      if (tile0 == 0) {
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          qh[kb][0] = lds128(qh_tile + g * PK_QROW + kb * 64 + t * 16);
+          qh[kb][1] = lds128(qh_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
+        }
+      }
       // every key comes from the cache: key index i sits at position j0 + i
-      attn_tile_compute<PRECISE>(A, sc, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G);
+      attn_tile_compute_w<PRECISE>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G);
     }
   }
-  attn_combine_store(A, sc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
+  attn_combine_store_w(A, sc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
 }
 
 }  // namespace dmtd

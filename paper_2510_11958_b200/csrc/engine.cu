@@ -146,7 +146,7 @@ int choose_aps(int K, int cap) {
 
 // Build one packed matrix from up to three row blocks (e.g. q, k, v) of equal K.
 dmtd_status pack_matrix(dmtd_ctx *c, PackedMat *out, int K, const void *const *srcs, const int *Ns, int n_src,
-                        int aps_cap = 40) {
+                        int aps_cap) {
   int N = 0;
   for (int i = 0; i < n_src; ++i) N += Ns[i];
   PackedMat m{};
@@ -619,6 +619,10 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   c->umma_ok = s.weight_dtype == DMTD_BF16 && (long long)max_batch * std::max(tau, 1) > 8 && H % TG_KB == 0 &&
                QD % TG_KB == 0 && I % TG_KB == 0;
   c->layers.resize(s.n_layers);
+  // k-slab width of the packed matrices: contexts small enough for the pass kernel (which stages
+  // only the slabs a block's share touches, and gains from short ones) get 256-wide slabs;
+  // larger batches run the per-step GEMV, which is faster with 1280-wide slabs
+  const int aps = max_batch <= PK_MAX_ROWS ? 8 : 40;
   for (int l = 0; l < s.n_layers; ++l) {
     const dmtd_layer_weights &lw = w->layers[l];
     const void *ptrs[] = {lw.input_norm, lw.q_proj, lw.k_proj, lw.v_proj, lw.q_norm, lw.k_norm, lw.o_proj,
@@ -628,14 +632,14 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
     LayerDev &ld = c->layers[l];
     const void *qkv_src[3] = {lw.q_proj, lw.k_proj, lw.v_proj};
     int qkv_n[3] = {QD, KVD, KVD};
-    CTRY(pack_matrix(c, &ld.qkv, H, qkv_src, qkv_n, 3));
+    CTRY(pack_matrix(c, &ld.qkv, H, qkv_src, qkv_n, 3, aps));
     const void *o_src[1] = {lw.o_proj}; int o_n[1] = {H};
     // k-slabs of two heads: a block of the pass kernel then merges the attention slices of few heads
     CTRY(pack_matrix(c, &ld.o, QD, o_src, o_n, 1, D == 128 ? 8 : 40));
     const void *gu_src[2] = {lw.gate_proj, lw.up_proj}; int gu_n[2] = {I, I};
-    CTRY(pack_matrix(c, &ld.gu, H, gu_src, gu_n, 2));
+    CTRY(pack_matrix(c, &ld.gu, H, gu_src, gu_n, 2, aps));
     const void *d_src[1] = {lw.down_proj}; int d_n[1] = {H};
-    CTRY(pack_matrix(c, &ld.down, I, d_src, d_n, 1));
+    CTRY(pack_matrix(c, &ld.down, I, d_src, d_n, 1, aps));
     if (c->umma_ok) {
       CTRY(pack_umma(c, &ld.qkv_u, H, qkv_src, qkv_n, 3));
       CTRY(pack_umma(c, &ld.o_u, QD, o_src, o_n, 1));
@@ -649,7 +653,7 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   }
   {
     const void *e_src[1] = {w->embed}; int e_n[1] = {s.vocab};
-    CTRY(pack_matrix(c, &c->embed, H, e_src, e_n, 1));
+    CTRY(pack_matrix(c, &c->embed, H, e_src, e_n, 1, aps));
     if (c->umma_ok) CTRY(pack_umma(c, &c->embed_u, H, e_src, e_n, 1));
     CTRY(vec_to_float(c, &c->w_final, w->final_norm, H));
   }

@@ -175,20 +175,30 @@ __device__ __noinline__ void attention_stage_f32(const PassParams &P, const Pass
           for (int j = 0; j < 8; ++j) kr[j] = lds_f4(sc + PK_F_K + (live ? key : 0) * PK_F_KROW + (part + 4 * j) * 16);
           const int idx = tile0 + key;
           const int key_pos = idx < n_cached ? j0 + idx : pos0 + (idx - n_cached);
-          int r = 0, h = 0;
+          // four query rows at a time: four independent chains of FMAs (rows beyond nQ hold
+          // whatever the scratch held; their sums are not stored)
 #pragma unroll 1
-          for (int q = 0; q < nQ; ++q) {
-            const unsigned char *qp = sc + PK_F_Q + q * PK_D * 4 + part * 16;
-            float s = 0.f;
+          for (int q0 = 0; q0 < nQ; q0 += 4) {
+            const unsigned char *qp = sc + PK_F_Q + q0 * PK_D * 4 + part * 16;
+            float s[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-              const float4 qv = lds_f4(qp + j * 64);
-              s += kr[j].x * qv.x + kr[j].y * qv.y + kr[j].z * qv.z + kr[j].w * qv.w;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float4 qv = lds_f4(qp + e * PK_D * 4 + j * 64);
+                s[e] += kr[j].x * qv.x + kr[j].y * qv.y + kr[j].z * qv.z + kr[j].w * qv.w;
+              }
             }
-            s += __shfl_xor_sync(0xffffffffu, s, 1);
-            s += __shfl_xor_sync(0xffffffffu, s, 2);
-            if (live && part == 0) sm_s[key * PK_QR + q] = key_pos <= pos0 + r ? s : -INFINITY;
-            if (++h == G) { h = 0; ++r; }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              s[e] += __shfl_xor_sync(0xffffffffu, s[e], 1);
+              s[e] += __shfl_xor_sync(0xffffffffu, s[e], 2);
+            }
+            if (live && part == 0) {
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                if (q0 + e < nQ) sm_s[key * PK_QR + q0 + e] = key_pos <= pos0 + (q0 + e) / G ? s[e] : -INFINITY;
+            }
           }
         }
       }

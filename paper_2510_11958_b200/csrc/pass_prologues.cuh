@@ -8,7 +8,7 @@
 
 namespace dmtd {
 
-constexpr int PK_MERGE_BATCH = 8;    // partial outputs (float4 per lane) in flight per warp in the merge
+constexpr int PK_MERGE_BATCH = 16;   // partial outputs (float4 per lane) in flight per warp in the merge
 constexpr int PK_SPAN_UNITS = 3;     // float4 units of a block's k-slab span per thread: span <= 3072 values
 
 // Inputs of a prologue come into shared memory as bulk copies issued by one thread: no load

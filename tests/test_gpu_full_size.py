@@ -43,3 +43,27 @@ def test_two_layers_qwen3_4b_geometry_benchmark_context():
     shape = SHAPES["qwen3_4b"].with_(n_layers=2)
     err, clear, eng = _run(shape, 1, 3, 512, 10, seed=3)
     print(f"two layers, P=512: max|dlogit|={err:.2e}, clear-margin steps {clear:.0%}")
+
+
+def test_repeated_runs_agree():
+    """The same forced decode twenty times through one context (reset in between): every run's
+    logits stay within 1e-3 of the first run's.  The order in which partial sums meet in fp32
+    moves them by about 5e-5; a stage that read a buffer another block was still writing, or
+    had already cleared, would move single steps by far more."""
+    import paper_2510_11958_b200 as pkg
+    shape = SHAPES["qwen3_4b"].with_(n_layers=2)
+    P = 512
+    wc = to_cuda(make_weights(shape, seed=3))
+    prompts = make_prompts(shape.vocab, 1, P, seed=1).numpy()
+    forced = make_prompts(shape.vocab, 1, 10, seed=2).numpy()
+    eng = pkg.Dmtd(shape, wc, L_d=1, tau=3, max_batch=1, max_seq=P + 12, kv_dtype="f32")
+    del wc
+    first, worst = None, 0.0
+    for _ in range(20):
+        eng.reset()
+        logits, _ = gpu_forced(eng, prompts, forced)
+        if first is None:
+            first = logits
+        else:
+            worst = max(worst, float(np.abs(logits - first).max()))
+    assert worst <= 1e-3, f"runs differ by {worst:.3e}"
