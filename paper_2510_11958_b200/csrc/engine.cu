@@ -614,10 +614,9 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   const dmtd_model_shape &s = c->s;
   const int H = s.hidden, D = s.head_dim, QD = s.n_q_heads * D, KVD = s.n_kv_heads * D, I = s.intermediate;
 
-  // weights; contexts whose passes can hold more than 8 rows (batch x cycle length) also get the
-  // copy the tcgen05 GEMM reads
-  c->umma_ok = s.weight_dtype == DMTD_BF16 && (long long)max_batch * std::max(tau, 1) > 8 && H % TG_KB == 0 &&
-               QD % TG_KB == 0 && I % TG_KB == 0;
+  // weights; every bf16 context whose dimensions fit also gets the copy the tcgen05 GEMM reads:
+  // passes of more than 8 rows (batch x cycle length) and the prefill of every context use it
+  c->umma_ok = s.weight_dtype == DMTD_BF16 && H % TG_KB == 0 && QD % TG_KB == 0 && I % TG_KB == 0;
   c->layers.resize(s.n_layers);
   // k-slab width of the packed matrices: contexts small enough for the pass kernel (which stages
   // only the slabs a block's share touches, and gains from short ones) get 256-wide slabs;

@@ -331,7 +331,6 @@ __device__ __forceinline__ void attn_combine_store(AttnAcc &A, unsigned char *sc
 // that its registers are not counted against the attention loop's.
 __device__ __noinline__ void attn_fetch_f32(const float *k_rows, const float *v_rows, int n_rows, unsigned char *sc) {
   const int total = n_rows * 64;                          // float4 units: 32 of K and 32 of V per row
-#pragma unroll 1
   for (int base = 0; base < total; base += PK_FETCH * PK_THREADS) {
     float4 v[PK_FETCH];
 #pragma unroll

@@ -6,7 +6,8 @@ Builds a profiling variant of the library (-DDMTD_PASS_TIMING, written beside th
 libdmtd_b200_timing.so), runs a few decode cycles of the workload and prints, for the first and
 the last block of the grid, how long thread 0 spent in every prologue, projection and grid
 barrier of one pass, averaged over the layers.  Times are clock64() ticks converted with
---ghz (the SM clock under load; 1.965 GHz on B200 when the kernel is memory-bound).
+the SM clock the launch itself measured (ticks between kernel entry and exit over the wall clock's
+nanoseconds; about 1.86 GHz under this load), or with --ghz.
 """
 import argparse
 import ctypes as C
@@ -37,7 +38,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="qwen3_4b_b1")
     ap.add_argument("--kind", default="full", choices=["full", "upper"])
-    ap.add_argument("--ghz", type=float, default=1.965)
+    ap.add_argument("--ghz", type=float, default=None, help="SM clock for tick -> us (default: measured in the launch itself)")
     ap.add_argument("--kv", default=None, choices=["bf16", "f32"], help="KV cache type (default: the workload's)")
     ap.add_argument("--prompt-len", type=int, default=None, help="prompt length (default: the workload's)")
     ap.add_argument("--build-only", action="store_true")
@@ -74,6 +75,9 @@ def main():
     eng.dll.dmtd_debug_pass_timing.argtypes = [C.c_void_p, C.c_void_p]
     assert eng.dll.dmtd_debug_pass_timing(eng._ctx, buf.ctypes.data_as(C.c_void_p)) == 0
     n_layers = shape.n_layers if args.kind == "full" else wl.L_d
+    if args.ghz is None:
+        c0, w0, c1, w1 = (int(v) for v in buf[SLOTS - 4:SLOTS])
+        args.ghz = (c1 - c0) / max(w1 - w0, 1)           # clock64 ticks per nanosecond of the wall clock
     for blk, label in ((0, "first block"), (1, "last block")):
         s = buf[blk * SLOTS:(blk + 1) * SLOTS]
         n = 1 + n_layers * 15 + 3
