@@ -15,6 +15,17 @@
 //    the following projection slower, not faster, so nothing is requested beyond the ring;
 //  * the grid barrier is one counter (release-add, acquire-poll by one thread per block): 2-3 us.
 //    A flag per block polled by a warp (no atomic serialisation) took 5-6 us.
+//  * handing a stage's outputs over without barriers was tried: every partial sum added with one
+//    64-bit reduction to a word that carries a fixed-point sum and a count of the atoms summed in,
+//    the next stage polling the words it needs.  It ran at the speed of the barrier version (what
+//    a stage waits for is the slowest block's share, 1 - 2.5 us behind the median and a different
+//    block every time, not the barrier's own 1.2 us), and a block's inputs come from only some of
+//    the blocks, so nothing tells it when a buffer may be cleared or reused: one run in ten had a
+//    pass with logits off by 1e-2.  Dropped.  (atomicAdd on unsigned long long compiled to the
+//    returning form and slowed the weight loop by 15 %; red.global.add.u64 in PTX did not.)
+//  * mma.sync issues about once per 30 cycles per SM sub-partition here: enough for the weight
+//    loop (one atom per ~90 cycles), too slow for attention with bf16 hi/lo pairs, which is
+//    why the fp32-cache attention stage uses FMAs.
 #pragma once
 
 #include "common.cuh"
