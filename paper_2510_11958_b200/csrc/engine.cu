@@ -244,13 +244,24 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
     P.rows = std::min(TG_MAX_COLS / 2, M - m0);
     P.n_cols = (2 * P.rows + 15) / 16 * 16;
     P.out = out + (size_t)m0 * ldo; P.ldo = ldo;
-    P.ksplit = std::max(1, std::min(W.n_kb, (c->n_sms + W.n_tiles - 1) / W.n_tiles));
     P.error = &c->dstate->error; P.wait_limit = 2000000000ll;
+    // Every block of a launch should be resident at once (a block streams at the rate its own
+    // stages allow, so a second round of blocks doubles the time): blocks per SM follow from
+    // shared memory and tensor memory; with more row tiles than that, two-stage blocks make room
+    // for two per SM.  Row tiles are then split along k over as many blocks as still fit.
+    int tmem_cols = 32;
+    while (tmem_cols < P.n_cols) tmem_cols <<= 1;
+    auto smem_of = [&](int st) { return st * (TG_WBLOCK + P.n_cols * 128) + 128; };
+    auto per_sm_of = [&](int st) { return std::max(1, std::min((227 * 1024) / (smem_of(st) + 1024), 512 / tmem_cols)); };
+    P.stages = TG_STAGES;
+    if (W.n_tiles > c->n_sms * per_sm_of(TG_STAGES) && W.n_tiles <= c->n_sms * per_sm_of(2)) P.stages = 2;
+    const int slots = c->n_sms * per_sm_of(P.stages);
+    P.ksplit = std::max(1, std::min(W.n_kb, slots / W.n_tiles));
     long long units = (long long)W.n_kb * 8 * P.n_cols;
     act_blocks_kernel<<<(int)std::min<long long>((units + 255) / 256, 4096), 256, 0, c->stream>>>(
         act + (size_t)m0 * lda, lda, P.rows, W.K, P.n_cols, c->act_blocks);
     LAUNCH_OK(c, "act_blocks_kernel");
-    int smem = TG_STAGES * (TG_WBLOCK + P.n_cols * 128) + 128;
+    int smem = smem_of(P.stages);
     static int configured = 0;
     if (configured < smem) {
       CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -679,7 +690,13 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   c->ws_rows = std::max(256, max_batch * std::max(tau, 8));
   c->lda = std::max(H, std::max(QD, I));
   c->ldqkv = QD + 2 * KVD; c->ldgu = 2 * I; c->ldl = (s.vocab + 15) / 16 * 16;
-  c->CH = max_seq <= 2048 ? 64 : 256;
+  // Keys per slice of the split-KV attention: enough slices that a decode step of max_batch
+  // sequences fills the SMs about four times over, and no more (every slice costs a block its
+  // set-up, a partial result and a share of the merge); whole 64-key tiles.
+  {
+    const int want = std::max(1, std::min(64, 4 * c->n_sms / std::max(1, max_batch * s.n_kv_heads)));
+    c->CH = std::max(64, ((max_seq + want - 1) / want + 63) / 64 * 64);
+  }
   c->nsplit_max = (max_seq + c->CH - 1) / c->CH;
   CTRY(dev_alloc(c, &c->x_lo, (size_t)c->ws_rows * H));
   CTRY(dev_alloc(c, &c->x_up, (size_t)max_batch * H));

@@ -44,6 +44,7 @@ struct GemmTcParams {
   float *out;                // [rows][ldo], accumulated into
   int ldo;
   int ksplit;                // blocks per row tile, each taking a share of the k blocks
+  int stages;                // pipeline stages of a block, 2 .. TG_STAGES
   int *error;
   long long wait_limit;
 };
@@ -76,9 +77,10 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
   extern __shared__ __align__(1024) unsigned char tg_smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int act_block = P.n_cols * 128, stage_bytes = TG_WBLOCK + act_block;
-  uint64_t *bars = reinterpret_cast<uint64_t *>(tg_smem + TG_STAGES * stage_bytes);    // full[S], empty[S], done
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * TG_STAGES + 1);
-  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + TG_STAGES), done = smem_u32(bars + 2 * TG_STAGES);
+  const int S = P.stages;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(tg_smem + S * stage_bytes);    // full[S], empty[S], done
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * S + 1);
+  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + S), done = smem_u32(bars + 2 * S);
 
   const int tile = blockIdx.x / P.ksplit, ks = blockIdx.x % P.ksplit;
   const int kb0 = P.W.n_kb * ks / P.ksplit, kb1 = P.W.n_kb * (ks + 1) / P.ksplit, n_it = kb1 - kb0;
@@ -86,7 +88,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
   while (tmem_cols < P.n_cols) tmem_cols <<= 1;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 2 * TG_STAGES + 1; ++s) mbar_init(smem_u32(bars + s), 1);
+    for (int s = 0; s < 2 * S + 1; ++s) mbar_init(smem_u32(bars + s), 1);
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -101,8 +103,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
   if (warp == 0 && lane == 0) {
     // ---- producer: two bulk copies per k block
     for (int i = 0; i < n_it; ++i) {
-      const int st = i % TG_STAGES;
-      if (i >= TG_STAGES && !tg_wait(empty0 + st * 8, ((i / TG_STAGES) - 1) & 1, P)) break;
+      const int st = i % S;
+      if (i >= S && !tg_wait(empty0 + st * 8, ((i / S) - 1) & 1, P)) break;
       const uint32_t dst = smem_u32(tg_smem + st * stage_bytes);
       mbar_expect_tx(full0 + st * 8, (uint32_t)stage_bytes);
       bulk_g2s(dst, P.W.w + ((size_t)tile * P.W.n_kb + kb0 + i) * (TG_WBLOCK / 16), TG_WBLOCK, full0 + st * 8);
@@ -114,8 +116,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
     const uint32_t b_lbo = (uint32_t)(P.n_cols / 8) * 128;
     bool ok = true;
     for (int i = 0; i < n_it && ok; ++i) {
-      const int st = i % TG_STAGES;
-      ok = tg_wait(full0 + st * 8, (i / TG_STAGES) & 1, P);
+      const int st = i % S;
+      ok = tg_wait(full0 + st * 8, (i / S) & 1, P);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t a_base = smem_u32(tg_smem + st * stage_bytes), b_base = a_base + TG_WBLOCK;
