@@ -948,7 +948,10 @@ struct AttnPlan { int CH, nsplit; size_t ml_off, o_off, bytes; };
 // pairs, then the unnormalised partial outputs, one set per (row, head, key slice).
 AttnPlan attn_plan(int B, int R, int nq, int D, int n_keys) {
   AttnPlan p{};
-  p.CH = n_keys <= 2048 ? 64 : 256;
+  // slices enough to fill a GPU of about 150 SMs four times over (the call does not know the
+  // number of kv heads: a quarter of the query heads is assumed), each of whole 64-key tiles
+  const int want = std::max(1, std::min(64, 600 / std::max(1, B * std::max(1, nq / 4))));
+  p.CH = std::max(64, ((n_keys + want - 1) / want + 63) / 64 * 64);
   p.nsplit = std::max(1, (n_keys + p.CH - 1) / p.CH);
   size_t slots = (size_t)B * R * nq * p.nsplit;
   p.ml_off = 256;
