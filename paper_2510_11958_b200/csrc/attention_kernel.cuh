@@ -6,7 +6,7 @@
 // the slices are merged by attn_merge_kernel.
 #pragma once
 
-#include "pass_attention.cuh"
+#include "pass_attention_f32.cuh"
 
 namespace dmtd {
 
@@ -313,6 +313,65 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
     }
   }
   attn_combine_store_w(A, sc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
+}
+
+// The same step for an fp32 cache in plain FMAs (three mma.sync per product would be needed for
+// fp32 accuracy, and they issue too slowly): the tile arithmetic of the pass kernel's fp32
+// attention stage, one 64-key tile in shared memory per block and two blocks per SM, so that one
+// block's copies run under the other's arithmetic.
+constexpr int ATTN_F32_SMEM = PK_F_NEW;           // K and V tile, Q, scores, running max / sum / rescale factor
+
+__global__ void __launch_bounds__(PK_THREADS, 2)
+attn_f32_kernel(const float *__restrict__ qkv, int ldq, const float *__restrict__ kc, const float *__restrict__ vc, int max_seq,
+                int nq, int nkv, int R, int RB, int CH, const int *__restrict__ pos0_ptr, float *__restrict__ part_o,
+                float *__restrict__ part_ml, int nsplit) {
+  extern __shared__ __align__(1024) unsigned char sc[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = nq / nkv, n_rb = (R + RB - 1) / RB;
+  const int split = blockIdx.x, kvh = blockIdx.y / n_rb, rb = blockIdx.y % n_rb, b = blockIdx.z;
+  const int r0 = rb * RB, r1 = min(R, r0 + RB), nQ = (r1 - r0) * G;
+  const int pos0 = *pos0_ptr;
+  const int j0 = split * CH, j1 = min(j0 + CH, pos0 + r1);      // the last row of the block sees position pos0 + r1 - 1
+  if (j0 >= j1) {                                                 // empty slice: mark and leave
+    for (int qi = threadIdx.x; qi < nQ; qi += PK_THREADS) {
+      const size_t slot = ((size_t)(b * R + r0 + qi / G) * nq + kvh * G + qi % G) * nsplit + split;
+      part_ml[slot * 2] = -INFINITY;
+      part_ml[slot * 2 + 1] = 0.f;
+    }
+    return;
+  }
+  // Q rows, scaled by 1/sqrt(d): row qi = (position r0 + qi / G, head kvh*G + qi % G)
+  const float scale = rsqrtf((float)PK_D);
+  for (int qi = warp; qi < nQ; qi += PK_WARPS) {
+    const float *src = qkv + (size_t)(b * R + r0 + qi / G) * ldq + (size_t)(kvh * G + qi % G) * PK_D;
+    float *dst = reinterpret_cast<float *>(sc + PK_F_Q) + qi * PK_D;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) dst[lane + 32 * j] = src[lane + 32 * j] * scale;
+  }
+  float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR;
+  if ((int)threadIdx.x < PK_QR) { m_run[threadIdx.x] = -INFINITY; l_run[threadIdx.x] = 0.f; }
+  const float *kb = kc + (((size_t)b * nkv + kvh) * max_seq + j0) * PK_D;
+  const float *vb = vc + (((size_t)b * nkv + kvh) * max_seq + j0) * PK_D;
+  float acc[PK_QR][4];
+#pragma unroll
+  for (int q = 0; q < PK_QR; ++q) acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f;
+  const int n_keys = j1 - j0;
+#pragma unroll 1
+  for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
+    const int n_t = min(PK_TK, n_keys - tile0);
+    __syncthreads();                                      // Q and the statistics written / previous tile consumed
+#pragma unroll 1
+    for (int c = threadIdx.x; c < n_t * 64; c += PK_THREADS) {
+      const int row = c >> 6, u = c & 63;
+      const uint32_t dst = smem_u32(sc) + (u < 32 ? PK_F_K + row * PK_F_KROW + u * 16 : PK_F_V + row * PK_D * 4 + (u - 32) * 16);
+      cp_async16(dst, (u < 32 ? kb : vb) + (size_t)(tile0 + row) * PK_D + (u & 31) * 4);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+    // every key comes from the cache: key index i sits at position j0 + i
+    attn_f32_tile(sc, acc, nQ, G, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0);
+  }
+  attn_f32_combine(sc, acc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
 }
 
 }  // namespace dmtd

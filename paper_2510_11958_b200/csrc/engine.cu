@@ -301,15 +301,23 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
   LAUNCH_OK(c, "qk_norm_rope_append_kernel");
   int RB = std::max(1, ATTN_QR / G), n_rb = (R + RB - 1) / RB;
   if (D == PK_D && c->use_tc_attention) {
-    // tensor-core kernel (head_dim 128): hi+lo operands with an fp32 cache, plain bf16 otherwise
-    constexpr bool kPrecise = std::is_same<KVT, float>::value;
+    // head_dim 128: the tensor-core kernel with a bf16 cache, the FMA kernel with an fp32 cache
     static bool tc_configured = false;
-    if (!tc_configured) {
-      CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<kPrecise>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM));
-      tc_configured = true;
+    if constexpr (std::is_same<KVT, float>::value) {
+      if (!tc_configured) {
+        CUDA_TRY(c, cudaFuncSetAttribute(attn_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_F32_SMEM));
+        tc_configured = true;
+      }
+      attn_f32_kernel<<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_F32_SMEM, c->stream>>>(
+          c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
+    } else {
+      if (!tc_configured) {
+        CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM));
+        tc_configured = true;
+      }
+      attn_tc_kernel<false><<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
+          c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
     }
-    attn_tc_kernel<kPrecise><<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
-        c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
   } else {
   size_t smem = (size_t)ATTN_WARPS * ATTN_QR * D * sizeof(float);
   static bool configured = false;
@@ -982,11 +990,18 @@ dmtd_status attention_launch_t(const float *q, const void *k, const void *v, int
   set_int_kernel<<<1, 1, 0, stream>>>(pos_dev, pos0);
   cudaError_t e;
   if (D == PK_D) {
-    constexpr bool kPrecise = std::is_same<KVT, float>::value;
-    e = cudaFuncSetAttribute(attn_tc_kernel<kPrecise>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM);
-    if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention: %s", cudaGetErrorString(e));
-    attn_tc_kernel<kPrecise><<<dim3(p.nsplit, nkv * n_rb, B), PK_THREADS, ATTN_TC_SMEM, stream>>>(
-        q, ld, k, v, max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o, part_ml, p.nsplit);
+    if constexpr (std::is_same<KVT, float>::value) {
+      e = cudaFuncSetAttribute(attn_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_F32_SMEM);
+      if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention: %s", cudaGetErrorString(e));
+      attn_f32_kernel<<<dim3(p.nsplit, nkv * n_rb, B), PK_THREADS, ATTN_F32_SMEM, stream>>>(
+          q, ld, static_cast<const float *>(k), static_cast<const float *>(v), max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o,
+          part_ml, p.nsplit);
+    } else {
+      e = cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM);
+      if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention: %s", cudaGetErrorString(e));
+      attn_tc_kernel<false><<<dim3(p.nsplit, nkv * n_rb, B), PK_THREADS, ATTN_TC_SMEM, stream>>>(
+          q, ld, k, v, max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o, part_ml, p.nsplit);
+    }
   } else {
     size_t smem = (size_t)ATTN_WARPS * ATTN_QR * D * sizeof(float);
     e = cudaFuncSetAttribute(attn_partial_kernel<D, KVT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);

@@ -2,10 +2,12 @@
 // (split-KV attention on the tensor cores; the key slices are merged by the O projection's
 // prologue).
 //
-// Two precisions, chosen by the KV cache's storage type.  With a bf16 cache, Q, K, P and V enter
-// the MMAs as single bf16 values.  With an fp32 cache every operand is a bf16 hi + lo pair and
-// each product is three MMAs (hi*hi + hi*lo + lo*hi), which keeps the attention at fp32 accuracy:
-// on the 36-layer model the bf16 cache alone moves the logits by up to 0.05, an fp32 cache by 1e-4.
+// This file is the tensor-core form, used with a bf16 cache: Q, K, P and V enter the MMAs as
+// single bf16 values.  The PRECISE = true variants below (every operand a bf16 hi + lo pair,
+// three MMAs per product, fp32 accuracy with an fp32 cache) are kept for comparison, but nothing
+// instantiates them any more: mma.sync issues too slowly for three per product, and fp32 caches
+// run the FMA form (pass_attention_f32.cuh).  On the 36-layer model a bf16 cache alone moves the
+// logits by up to 0.05, an fp32 cache by 1e-4.
 #pragma once
 
 #include "pass_prologues.cuh"

@@ -82,20 +82,144 @@ __device__ __forceinline__ void attn_new_rows_f32(const PassParams &P, const Pas
 
 __device__ __forceinline__ float4 lds_f4(const unsigned char *p) { return *reinterpret_cast<const float4 *>(p); }
 
+// One tile that is complete in shared memory: scores, the softmax step, O += P V.  Key index i of
+// the slice sits at position (i < n_cached ? j0 + i : pos_new + i - n_cached); query row q may see
+// positions up to row_pos0 + q / G.  Two block syncs inside; the caller syncs before the tile's
+// space is written again.
+__device__ __forceinline__ void attn_f32_tile(unsigned char *sc, float (&acc)[PK_QR][4], int nQ, int G, int n_t, int tile0,
+                                              int n_cached, int j0, int pos_new, int row_pos0) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float *const sm_s = reinterpret_cast<float *>(sc + PK_F_S);
+  float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR, *const corr = l_run + PK_QR;
+      {
+        // scores: thread = (key, part); part p holds the 16-byte units p, p + 4, .. of the K row
+        // (every lane runs the loop, since the four parts of a key meet in warp shuffles; keys
+        // beyond the tile read row 0 and store nothing)
+        const int key = threadIdx.x >> 2, part = threadIdx.x & 3;
+        const bool live = key < n_t;
+        {
+          float4 kr[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) kr[j] = lds_f4(sc + PK_F_K + (live ? key : 0) * PK_F_KROW + (part + 4 * j) * 16);
+          const int idx = tile0 + key;
+          const int key_pos = idx < n_cached ? j0 + idx : pos_new + (idx - n_cached);
+          // four query rows at a time: four independent chains of FMAs (rows beyond nQ hold
+          // whatever the scratch held; their sums are not stored)
+#pragma unroll 1
+          for (int q0 = 0; q0 < nQ; q0 += 4) {
+            const unsigned char *qp = sc + PK_F_Q + q0 * PK_D * 4 + part * 16;
+            float s[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float4 qv = lds_f4(qp + e * PK_D * 4 + j * 64);
+                s[e] += kr[j].x * qv.x + kr[j].y * qv.y + kr[j].z * qv.z + kr[j].w * qv.w;
+              }
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              s[e] += __shfl_xor_sync(0xffffffffu, s[e], 1);
+              s[e] += __shfl_xor_sync(0xffffffffu, s[e], 2);
+            }
+            if (live && part == 0) {
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                if (q0 + e < nQ) sm_s[key * PK_QR + q0 + e] = key_pos <= row_pos0 + (q0 + e) / G ? s[e] : -INFINITY;
+            }
+          }
+        }
+      }
+      pk_sync();
+      // per query row: the tile's max joins the running max; scores become probabilities
+#pragma unroll 1
+      for (int q = warp; q < nQ; q += PK_WARPS) {
+        const float v0 = lane < n_t ? sm_s[lane * PK_QR + q] : -INFINITY;
+        const float v1 = lane + 32 < n_t ? sm_s[(lane + 32) * PK_QR + q] : -INFINITY;
+        const float m_old = m_run[q];
+        const float m_new = fmaxf(m_old, warp_max(fmaxf(v0, v1)));
+        const float p0 = v0 > -INFINITY ? __expf(v0 - m_new) : 0.f;
+        const float p1 = v1 > -INFINITY ? __expf(v1 - m_new) : 0.f;
+        sm_s[lane * PK_QR + q] = p0;
+        sm_s[(lane + 32) * PK_QR + q] = p1;
+        const float ps = warp_sum(p0 + p1);
+        if (lane == 0) {
+          const float f = m_old > -INFINITY ? __expf(m_old - m_new) : 0.f;
+          corr[q] = f;
+          l_run[q] = l_run[q] * f + ps;
+          m_run[q] = m_new;
+        }
+      }
+      pk_sync();
+      // O += P V: warp = key group (keys warp, warp + 8, ..), lane = 4 output dimensions
+#pragma unroll
+      for (int q = 0; q < PK_QR; ++q) {
+        if (q < nQ) {
+          const float f = corr[q];
+          acc[q][0] *= f; acc[q][1] *= f; acc[q][2] *= f; acc[q][3] *= f;
+        }
+      }
+#pragma unroll 1
+      for (int key = warp; key < n_t; key += PK_WARPS) {
+        const float4 vv = lds_f4(sc + PK_F_V + (key * PK_D + lane * 4) * 4);
+#pragma unroll
+        for (int q4 = 0; q4 < PK_QR / 4; ++q4) {
+          if (q4 * 4 < nQ) {
+            const float4 pv = lds_f4(sc + PK_F_S + (key * PK_QR + q4 * 4) * 4);
+            const float pq[4] = {pv.x, pv.y, pv.z, pv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              acc[q4 * 4 + e][0] += pq[e] * vv.x; acc[q4 * 4 + e][1] += pq[e] * vv.y;
+              acc[q4 * 4 + e][2] += pq[e] * vv.z; acc[q4 * 4 + e][3] += pq[e] * vv.w;
+            }
+          }
+        }
+      }
+}
+
+// The slice's partial result: the key groups' outputs summed, with the running max and sum, at
+// slot (row0 + q / G, head0 + q % G, split), where a (row, head) owns `slot_stride` slots.
+__device__ __forceinline__ void attn_f32_combine(unsigned char *sc, float (&acc)[PK_QR][4], int nQ, int G, int row0, int head0,
+                                                 int nq, int slot_stride, int split, float *part_o, float *part_ml) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float *const m_run = reinterpret_cast<const float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR;
+    float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
+    pk_sync();                                            // tiles consumed: their space becomes o_s
+#pragma unroll
+    for (int q = 0; q < PK_QR; ++q)
+      if (q < nQ) *reinterpret_cast<float4 *>(o_s + (warp * PK_QR + q) * PK_OROW + lane * 4) = make_float4(acc[q][0], acc[q][1], acc[q][2], acc[q][3]);
+    pk_sync();
+    if ((int)threadIdx.x < nQ) {
+      const int qi = threadIdx.x;
+      const size_t slot = ((size_t)(row0 + qi / G) * nq + head0 + qi % G) * slot_stride + split;
+      *reinterpret_cast<float2 *>(part_ml + slot * 2) = make_float2(m_run[qi], l_run[qi]);
+    }
+#pragma unroll 1
+    for (int idx = threadIdx.x; idx < nQ * (PK_D / 4); idx += PK_THREADS) {
+      const int qi = idx / (PK_D / 4), d4 = idx % (PK_D / 4);
+      float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int w = 0; w < PK_WARPS; ++w) {
+        const float4 v = *reinterpret_cast<const float4 *>(o_s + (w * PK_QR + qi) * PK_OROW + d4 * 4);
+        sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+      }
+      const size_t slot = ((size_t)(row0 + qi / G) * nq + head0 + qi % G) * slot_stride + split;
+      *reinterpret_cast<float4 *>(part_o + slot * PK_D + d4 * 4) = sum;
+    }
+}
+
 // Steps a3 + a4 for the items (sequence, kv head, key slice) of this block, fp32 cache.
 // Per 64-key tile: scores by (key, quarter-of-d) threads with the K row in registers; softmax
 // statistics by one warp per query row; P V by (key group = warp, 4 output dims = lane) threads.
 __device__ __noinline__ void attention_stage_f32(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
   const PassShared S = pass_shared();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = P.nq / P.nkv, nQ = R * G;
   int nsplit, CH;
   attn_plan_device(P, pos0, nsplit, CH);
   const int items = P.B * P.nkv * nsplit;
   if ((int)blockIdx.x >= items) return;
   unsigned char *const sc = S.bstage;
-  float *const sm_s = reinterpret_cast<float *>(sc + PK_F_S);
-  float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR, *const corr = l_run + PK_QR;
+  float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR;
 
 #pragma unroll 1
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
@@ -163,120 +287,10 @@ __device__ __noinline__ void attention_stage_f32(const PassParams &P, const Pass
       cp_async_wait_all();
       pk_sync();
       PK_SUBSTAMP(10);
-      {
-        // scores: thread = (key, part); part p holds the 16-byte units p, p + 4, .. of the K row
-        // (every lane runs the loop, since the four parts of a key meet in warp shuffles; keys
-        // beyond the tile read row 0 and store nothing)
-        const int key = threadIdx.x >> 2, part = threadIdx.x & 3;
-        const bool live = key < n_t;
-        {
-          float4 kr[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) kr[j] = lds_f4(sc + PK_F_K + (live ? key : 0) * PK_F_KROW + (part + 4 * j) * 16);
-          const int idx = tile0 + key;
-          const int key_pos = idx < n_cached ? j0 + idx : pos0 + (idx - n_cached);
-          // four query rows at a time: four independent chains of FMAs (rows beyond nQ hold
-          // whatever the scratch held; their sums are not stored)
-#pragma unroll 1
-          for (int q0 = 0; q0 < nQ; q0 += 4) {
-            const unsigned char *qp = sc + PK_F_Q + q0 * PK_D * 4 + part * 16;
-            float s[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float4 qv = lds_f4(qp + e * PK_D * 4 + j * 64);
-                s[e] += kr[j].x * qv.x + kr[j].y * qv.y + kr[j].z * qv.z + kr[j].w * qv.w;
-              }
-            }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              s[e] += __shfl_xor_sync(0xffffffffu, s[e], 1);
-              s[e] += __shfl_xor_sync(0xffffffffu, s[e], 2);
-            }
-            if (live && part == 0) {
-#pragma unroll
-              for (int e = 0; e < 4; ++e)
-                if (q0 + e < nQ) sm_s[key * PK_QR + q0 + e] = key_pos <= pos0 + (q0 + e) / G ? s[e] : -INFINITY;
-            }
-          }
-        }
-      }
-      PK_SUBSTAMP(11);
-      pk_sync();
-      PK_SUBSTAMP(12);
-      // per query row: the tile's max joins the running max; scores become probabilities
-#pragma unroll 1
-      for (int q = warp; q < nQ; q += PK_WARPS) {
-        const float v0 = lane < n_t ? sm_s[lane * PK_QR + q] : -INFINITY;
-        const float v1 = lane + 32 < n_t ? sm_s[(lane + 32) * PK_QR + q] : -INFINITY;
-        const float m_old = m_run[q];
-        const float m_new = fmaxf(m_old, warp_max(fmaxf(v0, v1)));
-        const float p0 = v0 > -INFINITY ? __expf(v0 - m_new) : 0.f;
-        const float p1 = v1 > -INFINITY ? __expf(v1 - m_new) : 0.f;
-        sm_s[lane * PK_QR + q] = p0;
-        sm_s[(lane + 32) * PK_QR + q] = p1;
-        const float ps = warp_sum(p0 + p1);
-        if (lane == 0) {
-          const float f = m_old > -INFINITY ? __expf(m_old - m_new) : 0.f;
-          corr[q] = f;
-          l_run[q] = l_run[q] * f + ps;
-          m_run[q] = m_new;
-        }
-      }
-      PK_SUBSTAMP(13);
-      pk_sync();
-      PK_SUBSTAMP(14);
-      // O += P V: warp = key group (keys warp, warp + 8, ..), lane = 4 output dimensions
-#pragma unroll
-      for (int q = 0; q < PK_QR; ++q) {
-        if (q < nQ) {
-          const float f = corr[q];
-          acc[q][0] *= f; acc[q][1] *= f; acc[q][2] *= f; acc[q][3] *= f;
-        }
-      }
-#pragma unroll 1
-      for (int key = warp; key < n_t; key += PK_WARPS) {
-        const float4 vv = lds_f4(sc + PK_F_V + (key * PK_D + lane * 4) * 4);
-#pragma unroll
-        for (int q4 = 0; q4 < PK_QR / 4; ++q4) {
-          if (q4 * 4 < nQ) {
-            const float4 pv = lds_f4(sc + PK_F_S + (key * PK_QR + q4 * 4) * 4);
-            const float pq[4] = {pv.x, pv.y, pv.z, pv.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              acc[q4 * 4 + e][0] += pq[e] * vv.x; acc[q4 * 4 + e][1] += pq[e] * vv.y;
-              acc[q4 * 4 + e][2] += pq[e] * vv.z; acc[q4 * 4 + e][3] += pq[e] * vv.w;
-            }
-          }
-        }
-      }
+      attn_f32_tile(sc, acc, nQ, G, n_t, tile0, n_cached, j0, pos0, pos0);
     }
     PK_SUBSTAMP(5);
-    // the slice's partial result: the key groups' outputs summed, with the running max and sum
-    float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
-    pk_sync();                                            // tiles consumed: their space becomes o_s
-#pragma unroll
-    for (int q = 0; q < PK_QR; ++q)
-      if (q < nQ) *reinterpret_cast<float4 *>(o_s + (warp * PK_QR + q) * PK_OROW + lane * 4) = make_float4(acc[q][0], acc[q][1], acc[q][2], acc[q][3]);
-    pk_sync();
-    if ((int)threadIdx.x < nQ) {
-      const int qi = threadIdx.x;
-      const size_t slot = ((size_t)(b * R + qi / G) * P.nq + kvh * G + qi % G) * PK_NSPLIT_CAP + split;
-      *reinterpret_cast<float2 *>(P.part_ml + slot * 2) = make_float2(m_run[qi], l_run[qi]);
-    }
-#pragma unroll 1
-    for (int idx = threadIdx.x; idx < nQ * (PK_D / 4); idx += PK_THREADS) {
-      const int qi = idx / (PK_D / 4), d4 = idx % (PK_D / 4);
-      float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int w = 0; w < PK_WARPS; ++w) {
-        const float4 v = *reinterpret_cast<const float4 *>(o_s + (w * PK_QR + qi) * PK_OROW + d4 * 4);
-        sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
-      }
-      const size_t slot = ((size_t)(b * R + qi / G) * P.nq + kvh * G + qi % G) * PK_NSPLIT_CAP + split;
-      *reinterpret_cast<float4 *>(P.part_o + slot * PK_D + d4 * 4) = sum;
-    }
+    attn_f32_combine(sc, acc, nQ, G, b * R, kvh * G, P.nq, PK_NSPLIT_CAP, split, P.part_o, P.part_ml);
     PK_SUBSTAMP(6);
   }
   pk_sync();
