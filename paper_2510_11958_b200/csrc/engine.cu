@@ -76,6 +76,8 @@ struct dmtd_ctx {
   float *f_part_o = nullptr, *f_part_ml = nullptr, *amax_val = nullptr;
   int *amax_idx = nullptr;
   unsigned int *grid_bar = nullptr;
+  float *pick_val = nullptr;                // per-step greedy pick: best of every vocabulary slice, [max_batch][ARGMAX_SLICES]
+  int *pick_idx = nullptr;
   long long *pass_timing = nullptr;         // profiling builds only
 
   // graphs: [kind 1 = full, 2 = upper-only]
@@ -373,13 +375,15 @@ dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos
   const dmtd_model_shape &s = c->s;
   const LayerDev &lw = c->layers[l];
   int M = B * R, H = s.hidden, I = s.intermediate, QD = s.n_q_heads * s.head_dim;
-  prep_norm_kernel<<<M, 256, 0, c->stream>>>(x, H, lw.w_in, H, s.rms_eps, c->act, c->lda, c->qkv, c->ldqkv, c->ldqkv);
+  prep_norm_kernel<<<dim3(M, (c->ldqkv + PREP_ZERO_COLS - 1) / PREP_ZERO_COLS), 256, 0, c->stream>>>(
+      x, H, lw.w_in, H, s.rms_eps, c->act, c->lda, c->qkv, c->ldqkv, c->ldqkv);
   LAUNCH_OK(c, "prep_norm_kernel");
   TRY(launch_gemv(c, lw.qkv, lw.qkv_u, c->act, c->lda, M, c->qkv, c->ldqkv));
   TRY(launch_attention(c, l, B, R, pos0, splits_for(c, pos_end)));
   (void)QD;
   TRY(launch_gemv(c, lw.o, lw.o_u, c->act, c->lda, M, x, H));
-  prep_norm_kernel<<<M, 256, 0, c->stream>>>(x, H, lw.w_post, H, s.rms_eps, c->act, c->lda, c->gu, c->ldgu, c->ldgu);
+  prep_norm_kernel<<<dim3(M, (c->ldgu + PREP_ZERO_COLS - 1) / PREP_ZERO_COLS), 256, 0, c->stream>>>(
+      x, H, lw.w_post, H, s.rms_eps, c->act, c->lda, c->gu, c->ldgu, c->ldgu);
   LAUNCH_OK(c, "prep_norm_kernel");
   TRY(launch_gemv(c, lw.gu, lw.gu_u, c->act, c->lda, M, c->gu, c->ldgu));
   prep_swiglu_kernel<<<dim3((I + 255) / 256, M), 256, 0, c->stream>>>(c->gu, c->ldgu, I, c->act, c->lda);
@@ -391,16 +395,19 @@ dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos
 // Step a9/a10: final norm, tied LM head, greedy pick, token feedback.
 dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, float *out_logits) {
   const dmtd_model_shape &s = c->s;
-  prep_norm_kernel<<<B, 256, 0, c->stream>>>(c->x_up, s.hidden, c->w_final, s.hidden, s.rms_eps, c->act, c->lda,
+  prep_norm_kernel<<<dim3(B, (c->ldl + PREP_ZERO_COLS - 1) / PREP_ZERO_COLS), 256, 0, c->stream>>>(
+      c->x_up, s.hidden, c->w_final, s.hidden, s.rms_eps, c->act, c->lda,
                                              c->logits, c->ldl, c->ldl);
   LAUNCH_OK(c, "prep_norm_kernel");
   TRY(launch_gemv(c, c->embed, c->embed_u, c->act, c->lda, B, c->logits, c->ldl));
   if (out_logits)
     CUDA_TRY(c, cudaMemcpy2DAsync(out_logits, (size_t)s.vocab * 4, c->logits, (size_t)c->ldl * 4, (size_t)s.vocab * 4, B,
                                   cudaMemcpyDeviceToDevice, c->stream));
-  argmax_kernel<<<B, 1024, 0, c->stream>>>(c->logits, c->ldl, s.vocab, c->tokens, c->max_seq, c->dstate,
-                                           write_token ? 1 : 0, out_argmax);
-  LAUNCH_OK(c, "argmax_kernel");
+  argmax_slices_kernel<<<dim3(B, ARGMAX_SLICES), 256, 0, c->stream>>>(c->logits, c->ldl, s.vocab, c->pick_val, c->pick_idx);
+  LAUNCH_OK(c, "argmax_slices_kernel");
+  argmax_pick_kernel<<<B, 32, 0, c->stream>>>(c->pick_val, c->pick_idx, ARGMAX_SLICES, c->tokens, c->max_seq, c->dstate,
+                                              write_token ? 1 : 0, out_argmax);
+  LAUNCH_OK(c, "argmax_pick_kernel");
   return DMTD_OK;
 }
 
@@ -712,6 +719,8 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   CTRY(dev_alloc(c, &c->qkv, (size_t)c->ws_rows * c->ldqkv));
   CTRY(dev_alloc(c, &c->gu, (size_t)c->ws_rows * c->ldgu));
   CTRY(dev_alloc(c, &c->logits, (size_t)max_batch * c->ldl));
+  CTRY(dev_alloc(c, &c->pick_val, (size_t)max_batch * ARGMAX_SLICES));
+  CTRY(dev_alloc(c, &c->pick_idx, (size_t)max_batch * ARGMAX_SLICES));
   CTRY(dev_alloc(c, &c->part_o, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * D));
   CTRY(dev_alloc(c, &c->part_ml, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * 2));
   CTRY(dev_alloc(c, &c->rope_tab, (size_t)c->ws_rows * (D / 2)));

@@ -81,12 +81,24 @@ __global__ void embed_kernel(PackedMat E, const int *__restrict__ tokens, int ma
 
 // ------------------------------------------------------------------------------------
 // Activation preparation for a projection: act[m][:] = x[m][:] / rms(x[m]) * w, and clear
-// the accumulator row the projection will add into.  One block per row.
+// the accumulator row the projection will add into.  Grid (rows, slices): every block clears
+// PREP_ZERO_COLS columns of its row's accumulator, the first block of a row also does the norm.
 // ------------------------------------------------------------------------------------
+constexpr int PREP_ZERO_COLS = 4096;
 __global__ void prep_norm_kernel(const float *__restrict__ x, int ldx, const float *__restrict__ w,
                                  int K, float eps, float *__restrict__ act, int lda,
                                  float *__restrict__ zero_buf, int zero_ld, int zero_cols) {
-  int m = blockIdx.x;
+  const int m = blockIdx.x;
+  if (zero_buf) {
+    const int c0 = blockIdx.y * PREP_ZERO_COLS, c1 = min(zero_cols, c0 + PREP_ZERO_COLS);
+    float *row = zero_buf + (size_t)m * zero_ld;
+    const bool aligned = (zero_ld & 3) == 0;              // then every row starts on a 16-byte boundary
+    for (int k = c0 + threadIdx.x * 4; k < c1; k += blockDim.x * 4) {
+      if (aligned && k + 4 <= c1) *reinterpret_cast<float4 *>(row + k) = make_float4(0.f, 0.f, 0.f, 0.f);
+      else for (int j = k; j < c1; ++j) row[j] = 0.f;
+    }
+  }
+  if (blockIdx.y != 0) return;
   const float *xr = x + (size_t)m * ldx;
   float ss = 0.f;
   for (int k = threadIdx.x; k < K; k += blockDim.x) ss += xr[k] * xr[k];
@@ -102,8 +114,6 @@ __global__ void prep_norm_kernel(const float *__restrict__ x, int ldx, const flo
   __syncthreads();
   float inv = rsqrtf(red[0] / (float)K + eps);
   for (int k = threadIdx.x; k < K; k += blockDim.x) act[(size_t)m * lda + k] = xr[k] * inv * w[k];
-  if (zero_buf)
-    for (int k = threadIdx.x; k < zero_cols; k += blockDim.x) zero_buf[(size_t)m * zero_ld + k] = 0.f;
 }
 
 // act[m][i] = silu(g) * u with g = gu[m][i], u = gu[m][I + i]  (the SwiGLU gate).
@@ -516,22 +526,14 @@ __global__ void select_last_kernel(const float *__restrict__ x_lo, int R, int H,
 
 // ------------------------------------------------------------------------------------
 // a9 (second half): greedy pick, lowest index on ties; a10: feed the token back.
-// One block per sequence.  The token goes to position n_known of the token buffer unless a
-// forced token already sits there (teacher forcing), and to out_argmax if given.
+// Two levels: ARGMAX_SLICES blocks per sequence each find the best of their slice of the
+// vocabulary, then one block per sequence picks among them.  The token goes to position
+// n_known of the token buffer unless a forced token already sits there (teacher forcing), and
+// to out_argmax if given.
 // ------------------------------------------------------------------------------------
-__global__ void argmax_kernel(const float *__restrict__ logits, int ldl, int V, int *__restrict__ tokens,
-                              int max_seq, const DevState *__restrict__ st, int write_token,
-                              int *__restrict__ out_argmax) {
-  int b = blockIdx.x;
-  const float *z = logits + (size_t)b * ldl;
-  float best = -INFINITY;
-  int bi = 0x7fffffff;
-  for (int i = threadIdx.x; i < V; i += blockDim.x) {
-    float v = z[i];
-    if (v > best) { best = v; bi = i; }
-  }
-  __shared__ float sv[1024];
-  __shared__ int si[1024];
+constexpr int ARGMAX_SLICES = 16;
+
+__device__ __forceinline__ void argmax_block_reduce(float best, int bi, float *sv, int *si) {
   sv[threadIdx.x] = best; si[threadIdx.x] = bi;
   __syncthreads();
   for (int s = blockDim.x >> 1; s > 0; s >>= 1) {
@@ -543,6 +545,44 @@ __global__ void argmax_kernel(const float *__restrict__ logits, int ldl, int V, 
     }
     __syncthreads();
   }
+}
+
+// grid (sequences, ARGMAX_SLICES), 256 threads
+__global__ void argmax_slices_kernel(const float *__restrict__ logits, int ldl, int V, float *__restrict__ part_val,
+                                     int *__restrict__ part_idx) {
+  const int b = blockIdx.x, per = (V + gridDim.y - 1) / gridDim.y;
+  const int i0 = blockIdx.y * per, i1 = min(V, i0 + per);
+  const float *z = logits + (size_t)b * ldl;
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int i = i0 + threadIdx.x; i < i1; i += blockDim.x) {
+    float v = z[i];
+    if (v > best) { best = v; bi = i; }
+  }
+  __shared__ float sv[256];
+  __shared__ int si[256];
+  argmax_block_reduce(best, bi, sv, si);
+  if (threadIdx.x == 0) {
+    part_val[b * gridDim.y + blockIdx.y] = sv[0];
+    part_idx[b * gridDim.y + blockIdx.y] = si[0];
+  }
+}
+
+// grid (sequences), 32 threads
+__global__ void argmax_pick_kernel(const float *__restrict__ part_val, const int *__restrict__ part_idx, int n_slices,
+                                   int *__restrict__ tokens, int max_seq, const DevState *__restrict__ st, int write_token,
+                                   int *__restrict__ out_argmax) {
+  const int b = blockIdx.x;
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int i = threadIdx.x; i < n_slices; i += blockDim.x) {
+    float v = part_val[b * n_slices + i];
+    int ix = part_idx[b * n_slices + i];
+    if (v > best || (v == best && ix < bi)) { best = v; bi = ix; }
+  }
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  argmax_block_reduce(best, bi, sv, si);
   if (threadIdx.x == 0) {
     int pick = si[0] == 0x7fffffff ? 0 : si[0];
     if (write_token) tokens[(size_t)b * max_seq + st->n_known] = pick;

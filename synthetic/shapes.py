@@ -80,6 +80,9 @@ WORKLOADS = {
                                gen_len=64, kv_dtype="f32"),
     "qwen3_4b_b32": Workload("qwen3_4b_b32", "qwen3_4b", L_d=8, tau=3, batch=32, prompt_len=1024,
                              gen_len=512, kv_dtype="f32"),
+    # the same batch on the 4-layer model: small enough to list every launch under a profiler
+    "qwen3_4b_l4_b32": Workload("qwen3_4b_l4_b32", "qwen3_4b_l4", L_d=2, tau=3, batch=32, prompt_len=1024,
+                                gen_len=48, kv_dtype="f32"),
     "qwen3_4b_long": Workload("qwen3_4b_long", "qwen3_4b", L_d=8, tau=3, batch=8,
                               prompt_len=16384, gen_len=256),
 }
