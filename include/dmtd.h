@@ -198,12 +198,15 @@ dmtd_status dmtd_set_tau(dmtd_ctx *ctx, int32_t tau);
  *   "literal_sum"  0/1  upper-layer input of a full pass = embedding + lower-stack output, the
  *                       literal sum of Eq. 4, instead of the lower-stack output alone (default 0)
  *   "fused_pass"   0/1  run each decode pass as one persistent kernel where the model and batch
- *                       allow it (bf16 weights and KV, head_dim 128, at most 4 rows per pass);
+ *                       allow it (bf16 weights, bf16 or fp32 KV, head_dim 128, at most 4 rows per pass);
  *                       0 = always the per-step kernels (default 1)
- *   "tc_attention" 0/1  attention of the per-step kernels on the tensor cores (head_dim 128; default 1)
- *   "tcgen05_gemm" 0/1  projections of more than 8 rows on the tcgen05 tensor cores; only contexts
- *                       created with max_batch * tau > 8 hold the second weight copy it reads
- *                       (default 1)
+ *   "tc_attention" 0/1  attention of the per-step kernels by the tiled split-KV kernels for
+ *                       head_dim 128 (tensor cores with a bf16 cache, FMAs with an fp32 cache)
+ *                       instead of the one-warp-per-key-group kernel (default 1)
+ *   "tcgen05_gemm" 0/1  projections of more than 8 rows (prefill chunks included) on the tcgen05
+ *                       tensor cores; bf16 contexts whose hidden, query and intermediate sizes
+ *                       are multiples of 64 hold the second weight copy it reads, which doubles
+ *                       the weight memory of the context (default 1)
  * Errors: INVALID_ARG for an unknown name or value. */
 dmtd_status dmtd_set_option(dmtd_ctx *ctx, const char *name, int64_t value);
 
