@@ -270,7 +270,16 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
                                        TG_STAGES * (TG_WBLOCK + TG_MAX_COLS * 128) + 128));
       configured = TG_STAGES * (TG_WBLOCK + TG_MAX_COLS * 128) + 128;
     }
-    gemm_tc05_kernel<<<W.n_tiles * P.ksplit, TG_THREADS, smem, c->stream>>>(P);
+    // launched with programmatic stream serialisation: its blocks may start (allocate tensor
+    // memory, request their first weight blocks) while act_blocks_kernel is still running
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(W.n_tiles * P.ksplit); cfg.blockDim = dim3(TG_THREADS);
+    cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = c->stream;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    CUDA_TRY(c, cudaLaunchKernelEx(&cfg, gemm_tc05_kernel, P));
     LAUNCH_OK(c, "gemm_tc05_kernel");
   }
   return DMTD_OK;

@@ -101,10 +101,23 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
   const uint32_t tmem = *tmem_slot;
 
   if (warp == 0 && lane == 0) {
-    // ---- producer: two bulk copies per k block
-    for (int i = 0; i < n_it; ++i) {
+    // ---- producer: two bulk copies per k block.  The kernel is launched so that it may start
+    // while the kernel before it (which writes the activation blocks) is still running: the
+    // weight blocks of the first stages are requested at once, the activation blocks only after
+    // that kernel has completed and its writes are visible.
+    const int n_first = min(S, n_it);
+    for (int i = 0; i < n_first; ++i) {
+      mbar_expect_tx(full0 + i * 8, (uint32_t)stage_bytes);
+      bulk_g2s(smem_u32(tg_smem + i * stage_bytes), P.W.w + ((size_t)tile * P.W.n_kb + kb0 + i) * (TG_WBLOCK / 16), TG_WBLOCK,
+               full0 + i * 8);
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (int i = 0; i < n_first; ++i)
+      bulk_g2s(smem_u32(tg_smem + i * stage_bytes) + TG_WBLOCK, P.act_blocks + (size_t)(kb0 + i) * (act_block / 16),
+               (uint32_t)act_block, full0 + i * 8);
+    for (int i = n_first; i < n_it; ++i) {
       const int st = i % S;
-      if (i >= S && !tg_wait(empty0 + st * 8, ((i / S) - 1) & 1, P)) break;
+      if (!tg_wait(empty0 + st * 8, ((i / S) - 1) & 1, P)) break;
       const uint32_t dst = smem_u32(tg_smem + st * stage_bytes);
       mbar_expect_tx(full0 + st * 8, (uint32_t)stage_bytes);
       bulk_g2s(dst, P.W.w + ((size_t)tile * P.W.n_kb + kb0 + i) * (TG_WBLOCK / 16), TG_WBLOCK, full0 + st * 8);
@@ -170,6 +183,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
 // column 2m is the hi part of row m, column 2m + 1 its lo part; columns beyond 2 * rows are zero.
 __global__ void act_blocks_kernel(const float *__restrict__ act, int lda, int rows, int K, int n_cols,
                                   uint4 *__restrict__ blocks) {
+  // the GEMM that follows may be scheduled already: it waits for this grid before it reads the blocks
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int n_kb = K / TG_KB;
   const long long total = (long long)n_kb * 8 * n_cols;            // 16-byte units
   for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (long long)gridDim.x * blockDim.x) {
