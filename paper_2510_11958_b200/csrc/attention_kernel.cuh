@@ -319,7 +319,7 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
 // fp32 accuracy, and they issue too slowly): the tile arithmetic of the pass kernel's fp32
 // attention stage, one 64-key tile in shared memory per block and two blocks per SM, so that one
 // block's copies run under the other's arithmetic.
-constexpr int ATTN_F32_SMEM = PK_F_NEW;           // K and V tile, Q, scores, running max / sum / rescale factor
+constexpr int ATTN_F32_SMEM = PK_F_NEW;           // K and V tile, Q, partial scores, running max / sum / rescale factor
 
 __global__ void __launch_bounds__(PK_THREADS, 2)
 attn_f32_kernel(const float *__restrict__ qkv, int ldq, const float *__restrict__ kc, const float *__restrict__ vc, int max_seq,

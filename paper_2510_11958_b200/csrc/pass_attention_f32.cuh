@@ -12,17 +12,19 @@
 
 namespace dmtd {
 
-constexpr int PK_F_KROW = 576;                                   // bytes per K row: 512 + 64, conflict-free 16-byte reads by (key, part) lanes
+constexpr int PK_F_KROW = 528;                                   // bytes per K row: 512 + 16, conflict-free 16-byte reads by 8 lanes on 8 rows
+constexpr int PK_F_PARTS = 4;                                    // a score is the sum of 4 partial dot products over 32 dimensions each
 constexpr int PK_F_K = 0;                                        // K tile [PK_TK][PK_F_KROW]
 constexpr int PK_F_V = PK_F_K + PK_TK * PK_F_KROW;               // V tile [PK_TK][128] floats
 constexpr int PK_F_Q = PK_F_V + PK_TK * PK_D * 4;                // Q [PK_QR][128] floats, scaled by 1/sqrt(d)
-constexpr int PK_F_S = PK_F_Q + PK_QR * PK_D * 4;                // scores, then probabilities [PK_TK][PK_QR]
-constexpr int PK_F_STAT = PK_F_S + PK_TK * PK_QR * 4;            // running max, running sum, rescale factor [3][PK_QR]
+constexpr int PK_F_S = PK_F_Q + PK_QR * PK_D * 4;                // partial scores [part][PK_TK][PK_QR]; part 0's area then holds the probabilities
+constexpr int PK_F_STAT = PK_F_S + PK_F_PARTS * PK_TK * PK_QR * 4;   // running max, running sum, rescale factor [3][PK_QR]
 constexpr int PK_F_NEW = PK_F_STAT + 3 * PK_QR * 4;              // K rows of the pass [4][128], then V rows [4][128]
 constexpr int PK_F_W = PK_F_NEW + 2 * PK_MAX_ROWS * PK_D * 4;    // q-norm weights, k-norm weights (floats), rotary frequencies (doubles)
-constexpr int PK_F_END = PK_F_W + 2 * PK_D * 4 + (PK_D / 2) * 8;
-static_assert(PK_F_END <= PK_AT_ROWS, "fp32 attention scratch overlaps the row staging area");
-static_assert(PK_WARPS * PK_QR * PK_OROW * 4 <= PK_F_Q, "partial-output overlay reaches Q");
+constexpr int PK_F_ROWS = PK_F_W + 2 * PK_D * 4 + (PK_D / 2) * 8;    // the pass's q | k | v vectors of one kv head, fp32, per row
+constexpr int PK_F_END = PK_F_ROWS + PK_MAX_ROWS * PK_AT_ROW_FLOATS * 4;
+static_assert(PK_F_END <= PK_BSTAGE_BYTES + PK_XS_BYTES, "fp32 attention scratch does not fit");
+static_assert(PK_WARPS * PK_QR * PK_OROW * 4 <= PK_F_S, "partial-output overlay (over K, V and Q, all consumed by then) reaches the scores");
 
 // QK-norm (Section 3.1's Qwen3 block) and the half-split rotary embedding of one head vector,
 // one value per lane and quarter: v[j] is element lane + 32 j.
@@ -51,7 +53,7 @@ __device__ __forceinline__ void attn_new_rows_f32(const PassParams &P, const Pas
                                                   int R, int pos0, bool write_cache) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = P.nq / P.nkv, nQ = R * G;
-  const float *rows = reinterpret_cast<const float *>(sc + PK_AT_ROWS);
+  const float *rows = reinterpret_cast<const float *>(sc + PK_F_ROWS);
   const float *w_q = reinterpret_cast<const float *>(sc + PK_F_W), *w_k = w_q + PK_D;
   const double *inv_freq = reinterpret_cast<const double *>(sc + PK_F_W + 2 * PK_D * 4);
   const float scale = rsqrtf((float)PK_D);
@@ -91,51 +93,51 @@ __device__ __forceinline__ void attn_f32_tile(unsigned char *sc, float (&acc)[PK
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   float *const sm_s = reinterpret_cast<float *>(sc + PK_F_S);
   float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR, *const corr = l_run + PK_QR;
-      {
-        // scores: thread = (key, part); part p holds the 16-byte units p, p + 4, .. of the K row
-        // (every lane runs the loop, since the four parts of a key meet in warp shuffles; keys
-        // beyond the tile read row 0 and store nothing)
-        const int key = threadIdx.x >> 2, part = threadIdx.x & 3;
-        const bool live = key < n_t;
-        {
-          float4 kr[8];
+  {
+    // partial scores: warp = (part, half of the tile's keys), lane = key.  Part p is dimensions
+    // 32 p .. 32 p + 31; the lanes of a warp read the same Q values (one broadcast each) and
+    // their own K rows (row stride 528 bytes: no bank conflicts); the four parts of a score meet
+    // in the softmax step.
+    const int part = warp & 3, key = (warp >> 2) * 32 + lane;
+    if (key < n_t) {
+      float4 kr[8];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) kr[j] = lds_f4(sc + PK_F_K + (live ? key : 0) * PK_F_KROW + (part + 4 * j) * 16);
-          const int idx = tile0 + key;
-          const int key_pos = idx < n_cached ? j0 + idx : pos_new + (idx - n_cached);
-          // four query rows at a time: four independent chains of FMAs (rows beyond nQ hold
-          // whatever the scratch held; their sums are not stored)
+      for (int j = 0; j < 8; ++j) kr[j] = lds_f4(sc + PK_F_K + key * PK_F_KROW + (part * 8 + j) * 16);
+      // four query rows at a time: four independent chains of FMAs (rows beyond nQ hold whatever
+      // the scratch held; nobody reads their sums)
 #pragma unroll 1
-          for (int q0 = 0; q0 < nQ; q0 += 4) {
-            const unsigned char *qp = sc + PK_F_Q + q0 * PK_D * 4 + part * 16;
-            float s[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int q0 = 0; q0 < nQ; q0 += 4) {
+        const unsigned char *qp = sc + PK_F_Q + q0 * PK_D * 4 + part * 128;
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < 8; ++j) {
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float4 qv = lds_f4(qp + e * PK_D * 4 + j * 64);
-                s[e] += kr[j].x * qv.x + kr[j].y * qv.y + kr[j].z * qv.z + kr[j].w * qv.w;
-              }
-            }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              s[e] += __shfl_xor_sync(0xffffffffu, s[e], 1);
-              s[e] += __shfl_xor_sync(0xffffffffu, s[e], 2);
-            }
-            if (live && part == 0) {
-#pragma unroll
-              for (int e = 0; e < 4; ++e)
-                if (q0 + e < nQ) sm_s[key * PK_QR + q0 + e] = key_pos <= row_pos0 + (q0 + e) / G ? s[e] : -INFINITY;
-            }
+          for (int e = 0; e < 4; ++e) {
+            const float4 qv = lds_f4(qp + e * PK_D * 4 + j * 16);
+            s[e] += kr[j].x * qv.x + kr[j].y * qv.y + kr[j].z * qv.z + kr[j].w * qv.w;
           }
         }
+        *reinterpret_cast<float4 *>(sm_s + (part * PK_TK + key) * PK_QR + q0) = make_float4(s[0], s[1], s[2], s[3]);
       }
+    }
+  }
       pk_sync();
       // per query row: the tile's max joins the running max; scores become probabilities
 #pragma unroll 1
       for (int q = warp; q < nQ; q += PK_WARPS) {
-        const float v0 = lane < n_t ? sm_s[lane * PK_QR + q] : -INFINITY;
-        const float v1 = lane + 32 < n_t ? sm_s[(lane + 32) * PK_QR + q] : -INFINITY;
+        float v[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int key = lane + 32 * h, idx = tile0 + key;
+          const int key_pos = idx < n_cached ? j0 + idx : pos_new + (idx - n_cached);
+          v[h] = -INFINITY;
+          if (key < n_t && key_pos <= row_pos0 + q / G) {
+            v[h] = 0.f;
+#pragma unroll
+            for (int p = 0; p < PK_F_PARTS; ++p) v[h] += sm_s[(p * PK_TK + key) * PK_QR + q];
+          }
+        }
+        const float v0 = v[0], v1 = v[1];
         const float m_old = m_run[q];
         const float m_new = fmaxf(m_old, warp_max(fmaxf(v0, v1)));
         const float p0 = v0 > -INFINITY ? __expf(v0 - m_new) : 0.f;
@@ -239,7 +241,7 @@ __device__ __noinline__ void attention_stage_f32(const PassParams &P, const Pass
 #pragma unroll 1
       for (int r = 0; r < R; ++r) {
         const float *src = P.qkv + (size_t)(b * R + r) * ldq;
-        float *dst = reinterpret_cast<float *>(sc + PK_AT_ROWS) + r * PK_AT_ROW_FLOATS;
+        float *dst = reinterpret_cast<float *>(sc + PK_F_ROWS) + r * PK_AT_ROW_FLOATS;
         stage_copy(S, dst, src + kvh * G * PK_D, (uint32_t)(G * PK_D * 4));
         stage_copy(S, dst + G * PK_D, src + (P.nq + kvh) * PK_D, PK_D * 4);
         stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
