@@ -161,7 +161,7 @@ __device__ __forceinline__ void attn_f32_tile(unsigned char *sc, float (&acc)[PK
           acc[q][0] *= f; acc[q][1] *= f; acc[q][2] *= f; acc[q][3] *= f;
         }
       }
-#pragma unroll 1
+#pragma unroll 2
       for (int key = warp; key < n_t; key += PK_WARPS) {
         const float4 vv = lds_f4(sc + PK_F_V + (key * PK_D + lane * 4) * 4);
 #pragma unroll
