@@ -123,7 +123,7 @@ __device__ __forceinline__ void attn_f32_tile(unsigned char *sc, float (&acc)[PK
   }
       pk_sync();
       // per query row: the tile's max joins the running max; scores become probabilities
-#pragma unroll 1
+#pragma unroll 2
       for (int q = warp; q < nQ; q += PK_WARPS) {
         float v[2];
 #pragma unroll
