@@ -356,21 +356,37 @@ attn_f32_kernel(const float *__restrict__ qkv, int ldq, const float *__restrict_
 #pragma unroll
   for (int q = 0; q < PK_QR; ++q) acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f;
   const int n_keys = j1 - j0;
+  // The K and the V tile are loaded as two groups of asynchronous copies, each re-issued for the
+  // next tile as soon as the step that reads it is over: K of tile i + 1 arrives under the
+  // softmax step and P V of tile i, V of tile i + 1 under the scores of tile i + 1.
+  auto fetch = [&](const float *rows, int tile0, int dst_off, int row_bytes) {
+    const int n_t = min(PK_TK, n_keys - tile0);
+#pragma unroll 1
+    for (int c = threadIdx.x; c < n_t * 32; c += PK_THREADS) {
+      const int row = c >> 5, u = c & 31;
+      if (tile0 < n_keys) cp_async16(smem_u32(sc) + dst_off + row * row_bytes + u * 16, rows + (size_t)(tile0 + row) * PK_D + u * 4);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");      // an empty group past the last tile keeps the counts uniform
+  };
+  fetch(kb, 0, PK_F_K, PK_F_KROW);
+  fetch(vb, 0, PK_F_V, PK_D * 4);
 #pragma unroll 1
   for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
     const int n_t = min(PK_TK, n_keys - tile0);
-    __syncthreads();                                      // Q and the statistics written / previous tile consumed
-#pragma unroll 1
-    for (int c = threadIdx.x; c < n_t * 64; c += PK_THREADS) {
-      const int row = c >> 6, u = c & 63;
-      const uint32_t dst = smem_u32(sc) + (u < 32 ? PK_F_K + row * PK_F_KROW + u * 16 : PK_F_V + row * PK_D * 4 + (u - 32) * 16);
-      cp_async16(dst, (u < 32 ? kb : vb) + (size_t)(tile0 + row) * PK_D + (u & 31) * 4);
-    }
-    cp_async_wait_all();
-    __syncthreads();
+    asm volatile("cp.async.wait_group 1;" ::: "memory");      // K of this tile (V may still be on its way)
+    __syncthreads();                                      // ... from every thread; the first time also Q and the statistics
+    attn_f32_scores(sc, nQ, n_t);
+    __syncthreads();                                      // K consumed
+    fetch(kb, tile0 + PK_TK, PK_F_K, PK_F_KROW);
     // every key comes from the cache: key index i sits at position j0 + i
-    attn_f32_tile(sc, acc, nQ, G, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0);
+    attn_f32_softmax(sc, nQ, G, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0);
+    asm volatile("cp.async.wait_group 1;" ::: "memory");      // V of this tile (the next K may still be on its way)
+    __syncthreads();                                      // probabilities and V from every thread
+    attn_f32_pv(sc, acc, nQ, n_t);
+    __syncthreads();                                      // V and the probabilities consumed
+    fetch(vb, tile0 + PK_TK, PK_F_V, PK_D * 4);
   }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
   attn_f32_combine(sc, acc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
 }
 

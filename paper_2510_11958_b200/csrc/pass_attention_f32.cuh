@@ -84,15 +84,13 @@ __device__ __forceinline__ void attn_new_rows_f32(const PassParams &P, const Pas
 
 __device__ __forceinline__ float4 lds_f4(const unsigned char *p) { return *reinterpret_cast<const float4 *>(p); }
 
-// One tile that is complete in shared memory: scores, the softmax step, O += P V.  Key index i of
-// the slice sits at position (i < n_cached ? j0 + i : pos_new + i - n_cached); query row q may see
-// positions up to row_pos0 + q / G.  Two block syncs inside; the caller syncs before the tile's
-// space is written again.
-__device__ __forceinline__ void attn_f32_tile(unsigned char *sc, float (&acc)[PK_QR][4], int nQ, int G, int n_t, int tile0,
-                                              int n_cached, int j0, int pos_new, int row_pos0) {
+// One tile in shared memory, in three steps with a block sync between them: partial scores
+// (reads K and Q), the softmax step (scores to probabilities, running max and sum), O += P V
+// (reads V).  Key index i of the slice sits at position (i < n_cached ? j0 + i : pos_new + i -
+// n_cached); query row q may see positions up to row_pos0 + q / G.
+__device__ __forceinline__ void attn_f32_scores(unsigned char *sc, int nQ, int n_t) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   float *const sm_s = reinterpret_cast<float *>(sc + PK_F_S);
-  float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR, *const corr = l_run + PK_QR;
   {
     // partial scores: warp = (part, half of the tile's keys), lane = key.  Part p is dimensions
     // 32 p .. 32 p + 31; the lanes of a warp read the same Q values (one broadcast each) and
@@ -121,7 +119,13 @@ __device__ __forceinline__ void attn_f32_tile(unsigned char *sc, float (&acc)[PK
       }
     }
   }
-      pk_sync();
+}
+
+__device__ __forceinline__ void attn_f32_softmax(unsigned char *sc, int nQ, int G, int n_t, int tile0, int n_cached, int j0,
+                                                 int pos_new, int row_pos0) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float *const sm_s = reinterpret_cast<float *>(sc + PK_F_S);
+  float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR, *const corr = l_run + PK_QR;
       // per query row: the tile's max joins the running max; scores become probabilities
 #pragma unroll 2
       for (int q = warp; q < nQ; q += PK_WARPS) {
@@ -152,7 +156,11 @@ __device__ __forceinline__ void attn_f32_tile(unsigned char *sc, float (&acc)[PK
           m_run[q] = m_new;
         }
       }
-      pk_sync();
+}
+
+__device__ __forceinline__ void attn_f32_pv(unsigned char *sc, float (&acc)[PK_QR][4], int nQ, int n_t) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float *const corr = reinterpret_cast<const float *>(sc + PK_F_STAT) + 2 * PK_QR;
       // O += P V: warp = key group (keys warp, warp + 8, ..), lane = 4 output dimensions
 #pragma unroll
       for (int q = 0; q < PK_QR; ++q) {
@@ -177,6 +185,17 @@ __device__ __forceinline__ void attn_f32_tile(unsigned char *sc, float (&acc)[PK
           }
         }
       }
+}
+
+// The three steps on a tile that is complete in shared memory; the caller syncs before the tile's
+// space is written again.
+__device__ __forceinline__ void attn_f32_tile(unsigned char *sc, float (&acc)[PK_QR][4], int nQ, int G, int n_t, int tile0,
+                                              int n_cached, int j0, int pos_new, int row_pos0) {
+  attn_f32_scores(sc, nQ, n_t);
+  pk_sync();
+  attn_f32_softmax(sc, nQ, G, n_t, tile0, n_cached, j0, pos_new, row_pos0);
+  pk_sync();
+  attn_f32_pv(sc, acc, nQ, n_t);
 }
 
 // The slice's partial result: the key groups' outputs summed, with the running max and sum, at
