@@ -235,8 +235,11 @@ def test_errors(dmtd):
     ("bf16", 2, 3, 8, 2, 128, 37, 64),           # a refill chunk: causal among the 3 new rows
     ("f32", 3, 4, 4, 2, 64, 0, 8),               # no history at all
     ("bf16", 1, 5, 16, 1, 128, 2300, 2400),      # 16 query heads per KV head, rows split in blocks, long slices
-    ("f32", 2, 3, 8, 2, 128, 300, 512),          # fp32 cache on the tensor cores: hi+lo operands
+    ("f32", 2, 3, 8, 2, 128, 300, 512),          # fp32 cache: the FMA kernel
     ("f32", 1, 1, 32, 8, 128, 3000, 3072),
+    ("f32", 40, 1, 8, 2, 128, 1500, 1536),       # a batch large enough for long slices: 4 tiles per block, ragged
+    ("f32", 24, 3, 8, 2, 128, 1000, 1024),       # the same with a refill chunk (12 query rows per tile)
+    ("bf16", 40, 1, 8, 2, 128, 1500, 1536),      # several double-buffered tiles per block
 ])
 def test_attention_decode_matches_oracle(dmtd, oracle_lib, kvdt, B, R, nq, nkv, D, pos0, max_seq):
     """dmtd_attention_decode against the oracle's attention on the same (rounded) K and V."""
@@ -251,8 +254,8 @@ def test_attention_decode_matches_oracle(dmtd, oracle_lib, kvdt, B, R, nq, nkv, 
     for b in range(B):
         ref = oracle_lib.attention(q[b].double().numpy(), k[b, :, :n].double().permute(1, 0, 2).numpy(),
                                    v[b, :, :n].double().permute(1, 0, 2).numpy(), pos0)
-        # head_dim 128 runs on the tensor cores: with a bf16 cache Q and P are rounded to bf16 as well
-        # (2^-9 relative each); with an fp32 cache the operands are hi+lo pairs and nothing is lost
+        # head_dim 128 with a bf16 cache runs on the tensor cores: Q and P are rounded to bf16 as well
+        # (2^-9 relative each); with an fp32 cache the arithmetic is plain fp32
         tol = 5e-3 if (kvdt == "bf16" and D == 128) else 2e-5
         assert np.abs(got[b].double().cpu().numpy() - ref).max() <= tol * max(1.0, np.abs(ref).max())
 
