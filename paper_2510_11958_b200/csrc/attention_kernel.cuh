@@ -25,14 +25,12 @@ struct AttnAccW {
 // Keys of the tile are key_idx0 + row; key index i sits at position (i < n_cached ? j0 + i :
 // pos_new + i - n_cached); query row q may see positions up to row_pos0 + q / G.
 // k_off / v_off: where the tile's K and V (hi parts) sit in the scratch.
-template <bool PRECISE>
 __device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *sc, const uint4 (&qh)[4][2], int n_t, int tile0,
                                                   int n_cached, int j0, int pos_new, int row_pos0, int G,
                                                   int k_off = PK_AT_KH, int v_off = PK_AT_VH) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-  const uint32_t kh_tile = smem_u32(sc + k_off), kl_tile = smem_u32(sc + PK_AT_KL);
-  const uint32_t vh_tile = smem_u32(sc + v_off), vl_tile = smem_u32(sc + PK_AT_VL);
-  const uint32_t ql_tile = smem_u32(sc + PK_AT_QL);
+  const uint32_t kh_tile = smem_u32(sc + k_off);
+  const uint32_t vh_tile = smem_u32(sc + v_off);
   float (&m_run)[2] = A.m_run;
   float (&l_part)[2] = A.l_part;
   float (&o)[16][4] = A.o;
@@ -47,16 +45,6 @@ __device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *
             const uint4 Kh = lds128(kh_tile + off);
             mma_bf16_16816(c[nt], qh[kb][0].x, qh[kb][1].x, qh[kb][0].y, qh[kb][1].y, Kh.x, Kh.y);
             mma_bf16_16816(c[nt], qh[kb][0].z, qh[kb][1].z, qh[kb][0].w, qh[kb][1].w, Kh.z, Kh.w);
-            if (PRECISE) {
-              // the lo parts of Q stay in shared memory: registers are short here
-              const uint4 Kl = lds128(kl_tile + off);
-              const uint4 q0 = lds128(ql_tile + g * PK_QROW + kb * 64 + t * 16);
-              const uint4 q1 = lds128(ql_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
-              mma_bf16_16816(c[nt], qh[kb][0].x, qh[kb][1].x, qh[kb][0].y, qh[kb][1].y, Kl.x, Kl.y);
-              mma_bf16_16816(c[nt], qh[kb][0].z, qh[kb][1].z, qh[kb][0].w, qh[kb][1].w, Kl.z, Kl.w);
-              mma_bf16_16816(c[nt], q0.x, q1.x, q0.y, q1.y, Kh.x, Kh.y);
-              mma_bf16_16816(c[nt], q0.z, q1.z, q0.w, q1.w, Kh.z, Kh.w);
-            }
           }
         }
         // causal / range mask: lane holds rows g (e = 0, 1) and g + 8 (e = 2, 3), keys 2t, 2t + 1 of each n-tile
@@ -94,12 +82,11 @@ __device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *
         l_part[0] = l_part[0] * corr[0] + psum[0];
         l_part[1] = l_part[1] * corr[1] + psum[1];
         // P as the A operand: hi parts and (fp32 cache) lo parts
-        uint32_t ah[4], al[4] = {0u, 0u, 0u, 0u};
+        uint32_t ah[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float p0 = c[i >> 1][(i & 1) * 2], p1 = c[i >> 1][(i & 1) * 2 + 1];
           ah[i] = pack_bf16x2(p0, p1);
-          if (PRECISE) al[i] = pack_bf16x2(p0 - __uint_as_float(ah[i] << 16), p1 - __uint_as_float(ah[i] & 0xffff0000u));
         }
         const int mi = lane >> 3, rr = lane & 7;
         const uint32_t v_off = (warp * 16 + (mi & 1) * 8 + rr) * PK_VROW + (mi >> 1) * 16;
@@ -111,13 +98,6 @@ __device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *
           o[2 * d2 + 1][0] *= corr[0]; o[2 * d2 + 1][1] *= corr[0]; o[2 * d2 + 1][2] *= corr[1]; o[2 * d2 + 1][3] *= corr[1];
           mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
           mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
-          if (PRECISE) {
-            mma_bf16_16816(o[2 * d2], al[0], al[1], al[2], al[3], b0, b1);
-            mma_bf16_16816(o[2 * d2 + 1], al[0], al[1], al[2], al[3], b2, b3);
-            ldmatrix_x4_trans(vl_tile + v_off + d2 * 32, b0, b1, b2, b3);
-            mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
-            mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
-          }
         }
       }
 }
@@ -190,9 +170,8 @@ __device__ __forceinline__ void attn_combine_store_w(AttnAccW &A, unsigned char 
 constexpr int ATTN_TC_SMEM = PK_AT_ROWS;         // tiles, Q, partial-output overlay, reduction arrays
 
 // qkv [B*R][ldq]: q heads already normalised and rotated (not scaled); K and V of the new rows
-// already in the cache.  Cache [b][kv head][max_seq][128] bf16 (PRECISE = false) or fp32.
-template <bool PRECISE>
-__global__ void __launch_bounds__(PK_THREADS, PRECISE ? 1 : 2)      // bf16 cache: two blocks per SM overlap load and math
+// already in the cache.  Cache [b][kv head][max_seq][128] bf16.
+__global__ void __launch_bounds__(PK_THREADS, 2)      // bf16 cache: two blocks per SM overlap load and math
 attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ kc, const void *__restrict__ vc, int max_seq,
                int nq, int nkv, int R, int RB, int CH, const int *__restrict__ pos0_ptr, float *__restrict__ part_o,
                float *__restrict__ part_ml, int nsplit) {
@@ -211,7 +190,7 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
     }
     return;
   }
-  const uint32_t kh_tile = smem_u32(sc + PK_AT_KH), vh_tile = smem_u32(sc + PK_AT_VH), vl_tile = smem_u32(sc + PK_AT_VL);
+  const uint32_t kh_tile = smem_u32(sc + PK_AT_KH), vh_tile = smem_u32(sc + PK_AT_VH);
   const uint32_t qh_tile = smem_u32(sc + PK_AT_QH);
   // Q tile: rows beyond nQ zero; row qi = (position r0 + qi / G, head kvh*G + qi % G), scaled by 1/sqrt(d)
   for (int i = threadIdx.x; i < 2 * PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(qh_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
@@ -220,13 +199,11 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
   for (int qi = warp; qi < nQ; qi += PK_WARPS) {
     const float *src = qkv + (size_t)(b * R + r0 + qi / G) * ldq + (size_t)(kvh * G + qi % G) * PK_D;
     __nv_bfloat16 *qh = reinterpret_cast<__nv_bfloat16 *>(sc + PK_AT_QH + qi * PK_QROW);
-    __nv_bfloat16 *ql = reinterpret_cast<__nv_bfloat16 *>(sc + PK_AT_QL + qi * PK_QROW);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float v = src[lane + 32 * j] * scale;
       const __nv_bfloat16 h = __float2bfloat16_rn(v);
       qh[lane + 32 * j] = h;
-      if (PRECISE) ql[lane + 32 * j] = __float2bfloat16_rn(v - __bfloat162float(h));
     }
   }
   const size_t head_off = ((size_t)b * nkv + kvh) * max_seq * PK_D;
@@ -237,80 +214,44 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
   for (int dt = 0; dt < 16; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
   uint4 qh[4][2];
   const int n_keys = j1 - j0;
-  if (!PRECISE) {
-    // bf16 cache: two tile buffers (the lo-part areas are free here), tile i+1 in flight while
-    // tile i is multiplied
-    const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(kc) + head_off;
-    const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(vc) + head_off;
-    auto fetch = [&](int tile0, int buf) {
-      const int n_t = min(PK_TK, n_keys - tile0);
-      const uint32_t k_t = smem_u32(sc + (buf ? PK_AT_KL : PK_AT_KH)), v_t = smem_u32(sc + (buf ? PK_AT_VL : PK_AT_VH));
-      for (int c = threadIdx.x; c < n_t * 32; c += PK_THREADS) {
-        const int row = c >> 5, part = c & 31;
-        const uint32_t dst = part < 16 ? k_t + row * PK_KROW + part * 16 : v_t + row * PK_VROW + (part - 16) * 16;
-        cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
-      }
-      const int n16 = min(PK_TK, (n_t + 15) & ~15);
-      for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS)      // P = 0 times stale bits must stay 0
-        sts128(v_t + (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16, make_uint4(0u, 0u, 0u, 0u));
-      asm volatile("cp.async.commit_group;" ::: "memory");
-    };
-    fetch(0, 0);
-    int buf = 0;
-    for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK, buf ^= 1) {
-      const int n_t = min(PK_TK, n_keys - tile0);
-      if (tile0 + PK_TK < n_keys) {
-        fetch(tile0 + PK_TK, buf ^ 1);
-        asm volatile("cp.async.wait_group 1;" ::: "memory");
-      } else {
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-      }
-      __syncthreads();                                    // tile (and, the first time, Q) visible to all
-      if (tile0 == 0) {
-#pragma unroll
-        for (int kbk = 0; kbk < 4; ++kbk) {
-          qh[kbk][0] = lds128(qh_tile + g * PK_QROW + kbk * 64 + t * 16);
-          qh[kbk][1] = lds128(qh_tile + (g + 8) * PK_QROW + kbk * 64 + t * 16);
-        }
-      }
-      attn_tile_compute_w<false>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH,
-                               buf ? PK_AT_VL : PK_AT_VH);
-      __syncthreads();                                    // done with this buffer before it is refilled
+  // bf16 cache: two tile buffers (the lo-part areas are free here), tile i+1 in flight while
+  // tile i is multiplied
+  const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(kc) + head_off;
+  const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(vc) + head_off;
+  auto fetch = [&](int tile0, int buf) {
+    const int n_t = min(PK_TK, n_keys - tile0);
+    const uint32_t k_t = smem_u32(sc + (buf ? PK_AT_KL : PK_AT_KH)), v_t = smem_u32(sc + (buf ? PK_AT_VL : PK_AT_VH));
+    for (int c = threadIdx.x; c < n_t * 32; c += PK_THREADS) {
+      const int row = c >> 5, part = c & 31;
+      const uint32_t dst = part < 16 ? k_t + row * PK_KROW + part * 16 : v_t + row * PK_VROW + (part - 16) * 16;
+      cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
     }
-  } else {
-    for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
-      const int n_t = min(PK_TK, n_keys - tile0);
-      __syncthreads();                                      // Q written / previous tile consumed
-      if (!PRECISE) {
-        const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(kc) + head_off;
-        const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(vc) + head_off;
-        for (int c = threadIdx.x; c < n_t * 32; c += PK_THREADS) {
-          const int row = c >> 5, part = c & 31;
-          const uint32_t dst = part < 16 ? kh_tile + row * PK_KROW + part * 16 : vh_tile + row * PK_VROW + (part - 16) * 16;
-          cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
-        }
-      } else {
-        attn_fetch_f32(reinterpret_cast<const float *>(kc) + head_off + (size_t)(j0 + tile0) * PK_D,
-                       reinterpret_cast<const float *>(vc) + head_off + (size_t)(j0 + tile0) * PK_D, n_t, sc);
-      }
-      const int n16 = min(PK_TK, (n_t + 15) & ~15);
-      for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS) {      // P = 0 times stale bits must stay 0
-        const uint32_t off = (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16;
-        sts128(vh_tile + off, make_uint4(0u, 0u, 0u, 0u));
-        if (PRECISE) sts128(vl_tile + off, make_uint4(0u, 0u, 0u, 0u));
-      }
-      cp_async_wait_all();
-      __syncthreads();
-      if (tile0 == 0) {
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          qh[kb][0] = lds128(qh_tile + g * PK_QROW + kb * 64 + t * 16);
-          qh[kb][1] = lds128(qh_tile + (g + 8) * PK_QROW + kb * 64 + t * 16);
-        }
-      }
-      // every key comes from the cache: key index i sits at position j0 + i
-      attn_tile_compute_w<PRECISE>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G);
+    const int n16 = min(PK_TK, (n_t + 15) & ~15);
+    for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS)      // P = 0 times stale bits must stay 0
+      sts128(v_t + (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16, make_uint4(0u, 0u, 0u, 0u));
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  fetch(0, 0);
+  int buf = 0;
+  for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK, buf ^= 1) {
+    const int n_t = min(PK_TK, n_keys - tile0);
+    if (tile0 + PK_TK < n_keys) {
+      fetch(tile0 + PK_TK, buf ^ 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
+    __syncthreads();                                    // tile (and, the first time, Q) visible to all
+    if (tile0 == 0) {
+#pragma unroll
+      for (int kbk = 0; kbk < 4; ++kbk) {
+        qh[kbk][0] = lds128(qh_tile + g * PK_QROW + kbk * 64 + t * 16);
+        qh[kbk][1] = lds128(qh_tile + (g + 8) * PK_QROW + kbk * 64 + t * 16);
+      }
+    }
+    attn_tile_compute_w(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH,
+                             buf ? PK_AT_VL : PK_AT_VH);
+    __syncthreads();                                    // done with this buffer before it is refilled
   }
   attn_combine_store_w(A, sc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
 }

@@ -323,10 +323,10 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
           c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
     } else {
       if (!tc_configured) {
-        CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM));
+        CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM));
         tc_configured = true;
       }
-      attn_tc_kernel<false><<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
+      attn_tc_kernel<<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
           c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
     }
   } else {
@@ -1015,9 +1015,9 @@ dmtd_status attention_launch_t(const float *q, const void *k, const void *v, int
           q, ld, static_cast<const float *>(k), static_cast<const float *>(v), max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o,
           part_ml, p.nsplit);
     } else {
-      e = cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM);
+      e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM);
       if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention: %s", cudaGetErrorString(e));
-      attn_tc_kernel<false><<<dim3(p.nsplit, nkv * n_rb, B), PK_THREADS, ATTN_TC_SMEM, stream>>>(
+      attn_tc_kernel<<<dim3(p.nsplit, nkv * n_rb, B), PK_THREADS, ATTN_TC_SMEM, stream>>>(
           q, ld, k, v, max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o, part_ml, p.nsplit);
     }
   } else {

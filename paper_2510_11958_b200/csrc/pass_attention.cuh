@@ -3,11 +3,10 @@
 // prologue).
 //
 // This file is the tensor-core form, used with a bf16 cache: Q, K, P and V enter the MMAs as
-// single bf16 values.  The PRECISE = true variants below (every operand a bf16 hi + lo pair,
-// three MMAs per product, fp32 accuracy with an fp32 cache) are kept for comparison, but nothing
-// instantiates them any more: mma.sync issues too slowly for three per product, and fp32 caches
-// run the FMA form (pass_attention_f32.cuh).  On the 36-layer model a bf16 cache alone moves the
-// logits by up to 0.05, an fp32 cache by 1e-4.
+// single bf16 values.  fp32 caches run the FMA form (pass_attention_f32.cuh): fp32 accuracy on
+// the tensor cores would take three mma.sync per product (bf16 hi + lo pairs), which issue too
+// slowly here.  On the 36-layer model a bf16 cache alone moves the logits by up to 0.05, an fp32
+// cache by 1e-4.
 #pragma once
 
 #include "pass_prologues.cuh"
@@ -25,7 +24,6 @@ namespace dmtd {
 #define PK_SUBSTAMP(i) do {} while (0)
 #endif
 
-constexpr int PK_FETCH = 10;                                  // float4 units of an fp32 tile a thread loads at once
 constexpr int PK_TK = 64;                                     // keys per shared-memory tile
 constexpr int PK_KROW = 320;                                  // bytes per K row: 256 + 64, conflict-free 16-byte operand loads
 constexpr int PK_VROW = 272;                                  // bytes per V row: 256 + 16, conflict-free ldmatrix
@@ -33,9 +31,9 @@ constexpr int PK_QROW = 272;
 constexpr int PK_OROW = PK_D + 8;                             // floats per partial-output row, padded against bank conflicts
 // layout of the attention scratch (the activation staging area and the row staging area behind it)
 constexpr int PK_AT_KH = 0;                                   // K tile, hi parts [PK_TK][PK_KROW]
-constexpr int PK_AT_KL = PK_AT_KH + PK_TK * PK_KROW;          // K tile, lo parts (fp32 cache only)
+constexpr int PK_AT_KL = PK_AT_KH + PK_TK * PK_KROW;          // second K tile (the standalone kernel's double buffer)
 constexpr int PK_AT_VH = PK_AT_KL + PK_TK * PK_KROW;          // V tile, hi parts [PK_TK][PK_VROW]
-constexpr int PK_AT_VL = PK_AT_VH + PK_TK * PK_VROW;
+constexpr int PK_AT_VL = PK_AT_VH + PK_TK * PK_VROW;          // second V tile
 constexpr int PK_AT_QH = PK_AT_VL + PK_TK * PK_VROW;          // Q tile [PK_QR][PK_QROW], hi then lo
 constexpr int PK_AT_QL = PK_AT_QH + PK_QR * PK_QROW;
 constexpr int PK_AT_NEW = PK_AT_QL + PK_QR * PK_QROW;         // K rows of the pass [4][128] floats, then V rows [4][128]
@@ -69,26 +67,15 @@ __device__ __forceinline__ void attn_plan_device(const PassParams &P, int pos0, 
   nsplit = max(1, (pos0 + CH - 1) / CH);
 }
 
-// 8 values -> 16 bytes of bf16 hi parts and, if asked, 16 bytes of lo parts (x = hi + lo).
-template <bool PRECISE>
-__device__ __forceinline__ void split8(const float (&f)[8], uint4 &hi, uint4 &lo) {
-  uint32_t h[4], l[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    h[j] = pack_bf16x2(f[2 * j], f[2 * j + 1]);
-    l[j] = 0u;
-    if (PRECISE)
-      l[j] = pack_bf16x2(f[2 * j] - __uint_as_float(h[j] << 16), f[2 * j + 1] - __uint_as_float(h[j] & 0xffff0000u));
-  }
-  hi = make_uint4(h[0], h[1], h[2], h[3]);
-  lo = make_uint4(l[0], l[1], l[2], l[3]);
+// 8 values -> 16 bytes of bf16.
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+  return make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
 }
 
 // Step a3 for one (sequence, kv head): one warp per head vector of the pass's rows (staged in
 // shared memory as q heads | k | v per row).  Query rows go to the Q tile (scaled by 1/sqrt(d));
 // K and V rows go to the new-row area as floats already rounded to the cache's type and, from
 // the block that owns slice 0, into the cache.
-template <bool PRECISE>
 __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLayer &Ly, unsigned char *sc, int b, int kvh,
                                               int R, int pos0, bool write_cache) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -127,26 +114,19 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
     }
     if (kind == 0) {
       __nv_bfloat16 *qh = reinterpret_cast<__nv_bfloat16 *>(sc + PK_AT_QH + task * PK_QROW);
-      __nv_bfloat16 *ql = reinterpret_cast<__nv_bfloat16 *>(sc + PK_AT_QL + task * PK_QROW);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const __nv_bfloat16 h = __float2bfloat16_rn(v[j]);
         qh[lane + 32 * j] = h;
-        if (PRECISE) ql[lane + 32 * j] = __float2bfloat16_rn(v[j] - __bfloat162float(h));
       }
     } else {
       float *row = reinterpret_cast<float *>(sc + PK_AT_NEW) + ((kind == 2 ? PK_MAX_ROWS : 0) + r) * PK_D;
       const size_t at = (((size_t)b * P.nkv + kvh) * P.max_seq + pos) * PK_D;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        if (PRECISE) {
-          row[lane + 32 * j] = v[j];
-          if (write_cache) reinterpret_cast<float *>(kind == 1 ? Ly.kc : Ly.vc)[at + lane + 32 * j] = v[j];
-        } else {
-          const __nv_bfloat16 h = __float2bfloat16_rn(v[j]);
-          row[lane + 32 * j] = __bfloat162float(h);
-          if (write_cache) reinterpret_cast<__nv_bfloat16 *>(kind == 1 ? Ly.kc : Ly.vc)[at + lane + 32 * j] = h;
-        }
+        const __nv_bfloat16 h = __float2bfloat16_rn(v[j]);
+        row[lane + 32 * j] = __bfloat162float(h);
+        if (write_cache) reinterpret_cast<__nv_bfloat16 *>(kind == 1 ? Ly.kc : Ly.vc)[at + lane + 32 * j] = h;
       }
     }
   }
@@ -166,15 +146,14 @@ struct AttnAcc {
 // k_off / v_off: where the tile's K and V (hi parts) sit in the scratch.  The Q fragments are
 // read from shared memory in a rolled loop: the code stays short (instruction fetch, not
 // arithmetic, bounds a stage that runs once per layer).
-template <bool PRECISE>
 __device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc, int n_t, int tile0, int n_cached, int j0,
                                                   int pos_new, int row_pos0, int G, int k_off = PK_AT_KH,
                                                   int v_off = PK_AT_VH) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int kg = warp & 3, dh = warp >> 2;
-  const uint32_t kh_tile = smem_u32(sc + k_off), kl_tile = smem_u32(sc + PK_AT_KL);
-  const uint32_t vh_tile = smem_u32(sc + v_off), vl_tile = smem_u32(sc + PK_AT_VL);
-  const uint32_t qh_tile = smem_u32(sc + PK_AT_QH), ql_tile = smem_u32(sc + PK_AT_QL);
+  const uint32_t kh_tile = smem_u32(sc + k_off);
+  const uint32_t vh_tile = smem_u32(sc + v_off);
+  const uint32_t qh_tile = smem_u32(sc + PK_AT_QH);
   float (&m_run)[2] = A.m_run;
   float (&l_part)[2] = A.l_part;
   float (&o)[8][4] = A.o;
@@ -186,21 +165,12 @@ __device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc,
   for (int kb = 0; kb < 4; ++kb) {
     const uint32_t q_off = g * PK_QROW + kb * 64 + t * 16;
     const uint4 q0 = lds128(qh_tile + q_off), q1 = lds128(qh_tile + q_off + 8 * PK_QROW);
-    uint4 p0 = make_uint4(0u, 0u, 0u, 0u), p1 = p0;
-    if (PRECISE) { p0 = lds128(ql_tile + q_off); p1 = lds128(ql_tile + q_off + 8 * PK_QROW); }
-#pragma unroll
+    #pragma unroll
     for (int nt = 0; nt < 2; ++nt) {
       const uint32_t off = (kg * 16 + nt * 8 + g) * PK_KROW + kb * 64 + t * 16;
       const uint4 Kh = lds128(kh_tile + off);
       mma_bf16_16816(c[nt], q0.x, q1.x, q0.y, q1.y, Kh.x, Kh.y);
       mma_bf16_16816(c[nt], q0.z, q1.z, q0.w, q1.w, Kh.z, Kh.w);
-      if (PRECISE) {
-        const uint4 Kl = lds128(kl_tile + off);
-        mma_bf16_16816(c[nt], q0.x, q1.x, q0.y, q1.y, Kl.x, Kl.y);
-        mma_bf16_16816(c[nt], q0.z, q1.z, q0.w, q1.w, Kl.z, Kl.w);
-        mma_bf16_16816(c[nt], p0.x, p1.x, p0.y, p1.y, Kh.x, Kh.y);
-        mma_bf16_16816(c[nt], p0.z, p1.z, p0.w, p1.w, Kh.z, Kh.w);
-      }
     }
   }
   // causal / range mask: lane holds rows g (e = 0, 1) and g + 8 (e = 2, 3), keys 2t, 2t + 1 of each n-tile
@@ -238,12 +208,11 @@ __device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc,
   l_part[0] = l_part[0] * corr[0] + psum[0];
   l_part[1] = l_part[1] * corr[1] + psum[1];
   // P as the A operand: hi parts and (fp32 cache) lo parts
-  uint32_t ah[4], al[4] = {0u, 0u, 0u, 0u};
+  uint32_t ah[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const float p0 = c[i >> 1][(i & 1) * 2], p1 = c[i >> 1][(i & 1) * 2 + 1];
     ah[i] = pack_bf16x2(p0, p1);
-    if (PRECISE) al[i] = pack_bf16x2(p0 - __uint_as_float(ah[i] << 16), p1 - __uint_as_float(ah[i] & 0xffff0000u));
   }
   const int mi = lane >> 3, rr = lane & 7;
   const uint32_t v_row = (kg * 16 + (mi & 1) * 8 + rr) * PK_VROW + (mi >> 1) * 16 + dh * 128;
@@ -255,13 +224,6 @@ __device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc,
     o[2 * d2 + 1][0] *= corr[0]; o[2 * d2 + 1][1] *= corr[0]; o[2 * d2 + 1][2] *= corr[1]; o[2 * d2 + 1][3] *= corr[1];
     mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
     mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
-    if (PRECISE) {
-      mma_bf16_16816(o[2 * d2], al[0], al[1], al[2], al[3], b0, b1);
-      mma_bf16_16816(o[2 * d2 + 1], al[0], al[1], al[2], al[3], b2, b3);
-      ldmatrix_x4_trans(vl_tile + v_row + d2 * 32, b0, b1, b2, b3);
-      mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
-      mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
-    }
   }
 }
 
@@ -328,43 +290,11 @@ __device__ __forceinline__ void attn_combine_store(AttnAcc &A, unsigned char *sc
   }
 }
 
-// Cached rows of an fp32 tile: through registers, PK_FETCH float4 per thread in flight (one trip
-// for a slice of up to 40 keys), each split into bf16 hi and lo parts.  A function of its own so
-// that its registers are not counted against the attention loop's.
-__device__ __noinline__ void attn_fetch_f32(const float *k_rows, const float *v_rows, int n_rows, unsigned char *sc) {
-  const int total = n_rows * 64;                          // float4 units: 32 of K and 32 of V per row
-  for (int base = 0; base < total; base += PK_FETCH * PK_THREADS) {
-    float4 v[PK_FETCH];
-#pragma unroll
-    for (int j = 0; j < PK_FETCH; ++j) {
-      const int c = base + j * PK_THREADS + threadIdx.x;
-      if (c < total) {
-        const int row = c >> 6, u = c & 63;
-        v[j] = __ldcg(reinterpret_cast<const float4 *>((u < 32 ? k_rows : v_rows) + (size_t)row * PK_D) + (u & 31));
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < PK_FETCH; ++j) {
-      const int c = base + j * PK_THREADS + threadIdx.x;
-      if (c < total) {
-        const int row = c >> 6, u = c & 63;
-        const uint32_t h0 = pack_bf16x2(v[j].x, v[j].y), h1 = pack_bf16x2(v[j].z, v[j].w);
-        const uint32_t l0 = pack_bf16x2(v[j].x - __uint_as_float(h0 << 16), v[j].y - __uint_as_float(h0 & 0xffff0000u));
-        const uint32_t l1 = pack_bf16x2(v[j].z - __uint_as_float(h1 << 16), v[j].w - __uint_as_float(h1 & 0xffff0000u));
-        const int off = u < 32 ? row * PK_KROW + u * 8 : row * PK_VROW + (u - 32) * 8;
-        *reinterpret_cast<uint2 *>(sc + (u < 32 ? PK_AT_KH : PK_AT_VH) + off) = make_uint2(h0, h1);
-        *reinterpret_cast<uint2 *>(sc + (u < 32 ? PK_AT_KL : PK_AT_VL) + off) = make_uint2(l0, l1);
-      }
-    }
-  }
-}
-
 // Steps a3 + a4 for the items (sequence, kv head, key slice) of this block.  The R*G query rows
 // of an item form one m16 tile; S = Q K^T and O = P V run as mma.m16n8k16 with K and V staged in
 // shared memory, each warp taking 16 keys of a 64-key tile with its own running max and sum.
 // The slice's unnormalised partial output goes to global memory with its max and sum; the
 // prologue of the O projection merges the slices.
-template <bool PRECISE>
 __device__ __noinline__ void attention_stage(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
   const PassShared S = pass_shared();
   const int G = P.nq / P.nkv, nQ = R * G;
@@ -374,16 +304,14 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
   if ((int)blockIdx.x >= items) return;
 
   unsigned char *const sc = S.bstage;
-  const uint32_t kh_tile = smem_u32(sc + PK_AT_KH), kl_tile = smem_u32(sc + PK_AT_KL);
-  const uint32_t vh_tile = smem_u32(sc + PK_AT_VH), vl_tile = smem_u32(sc + PK_AT_VL);
+  const uint32_t kh_tile = smem_u32(sc + PK_AT_KH);
+  const uint32_t vh_tile = smem_u32(sc + PK_AT_VH);
   const uint32_t qh_tile = smem_u32(sc + PK_AT_QH);
   // a 16-byte part (8 values) of a tile row: parts 0..15 are K, 16..31 are V
   auto put_part = [&](int row, int part, const float (&f)[8]) {
-    uint4 hi, lo;
-    split8<PRECISE>(f, hi, lo);
+    const uint4 hi = pack8(f);
     const uint32_t off = part < 16 ? row * PK_KROW + part * 16 : row * PK_VROW + (part - 16) * 16;
     sts128((part < 16 ? kh_tile : vh_tile) + off, hi);
-    if (PRECISE) sts128((part < 16 ? kl_tile : vl_tile) + off, lo);
   };
 
 #pragma unroll 1
@@ -397,20 +325,16 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     // cached rows of a tile
     auto fetch_cached = [&](int tile0) {
       const int n_c = min(PK_TK, n_cached - tile0);
-      if (!PRECISE) {
-        // bf16 cache: asynchronous copies, 16 bytes each
-        const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(Ly.kc) + head_off;
-        const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(Ly.vc) + head_off;
+      // bf16 cache: asynchronous copies, 16 bytes each
+      const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(Ly.kc) + head_off;
+      const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(Ly.vc) + head_off;
 #pragma unroll 1
-        for (int c = threadIdx.x; c < n_c * 32; c += PK_THREADS) {
-          const int row = c >> 5, part = c & 31;
-          const uint32_t dst = part < 16 ? kh_tile + row * PK_KROW + part * 16 : vh_tile + row * PK_VROW + (part - 16) * 16;
-          cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
-        }
-      } else {
-        attn_fetch_f32(reinterpret_cast<const float *>(Ly.kc) + head_off + (size_t)(j0 + tile0) * PK_D,
-                       reinterpret_cast<const float *>(Ly.vc) + head_off + (size_t)(j0 + tile0) * PK_D, n_c, sc);
+      for (int c = threadIdx.x; c < n_c * 32; c += PK_THREADS) {
+        const int row = c >> 5, part = c & 31;
+        const uint32_t dst = part < 16 ? kh_tile + row * PK_KROW + part * 16 : vh_tile + row * PK_VROW + (part - 16) * 16;
+        cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
       }
+    
     };
     PK_SUBSTAMP(0);
     pk_sync();                                            // the previous item is done with the scratch
@@ -435,7 +359,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     for (int i = threadIdx.x; i < 2 * PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(qh_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
     stage_wait(P, S);
     PK_SUBSTAMP(3);
-    attn_new_rows<PRECISE>(P, Ly, sc, b, kvh, R, pos0, split == 0);
+    attn_new_rows(P, Ly, sc, b, kvh, R, pos0, split == 0);
     PK_SUBSTAMP(4);
 
     AttnAcc A;
@@ -461,13 +385,12 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
       for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS) {    // P = 0 times stale bits must stay 0
         const uint32_t off = (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16;
         sts128(vh_tile + off, make_uint4(0u, 0u, 0u, 0u));
-        if (PRECISE) sts128(vl_tile + off, make_uint4(0u, 0u, 0u, 0u));
       }
       PK_SUBSTAMP(9);
       cp_async_wait_all();
       pk_sync();
       PK_SUBSTAMP(10);
-      attn_tile_compute<PRECISE>(A, sc, n_t, tile0, n_cached, j0, pos0, pos0, G);
+      attn_tile_compute(A, sc, n_t, tile0, n_cached, j0, pos0, pos0, G);
     }
     PK_SUBSTAMP(5);
     attn_combine_store(A, sc, nQ, G, b * R, kvh * G, P.nq, PK_NSPLIT_CAP, split, P.part_o, P.part_ml);
