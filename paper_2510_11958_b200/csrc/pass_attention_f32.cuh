@@ -253,21 +253,27 @@ __device__ __noinline__ void attention_stage_f32(const PassParams &P, const Pass
     const float *vc = reinterpret_cast<const float *>(Ly.vc) + (((size_t)b * P.nkv + kvh) * P.max_seq + j0) * PK_D;
     PK_SUBSTAMP(0);
     pk_sync();                                            // the previous item is done with the scratch
-    if (threadIdx.x == 0) {
-      // the pass's own q | k | v vectors of this kv head, the two norm weights and the rotary frequencies
-      const int ldq = (P.nq + 2 * P.nkv) * PK_D;
-      stage_begin(S, (uint32_t)(R * (G + 2) * PK_D * 4 + 2 * PK_D * 4 + (PK_D / 2) * 8));
-#pragma unroll 1
-      for (int r = 0; r < R; ++r) {
+    // the pass's own q | k | v vectors of this kv head (three copies per row), the two norm weights
+    // and the rotary frequencies: one copy per lane of the first warp
+    if (threadIdx.x == 0) stage_begin(S, (uint32_t)(R * (G + 2) * PK_D * 4 + 2 * PK_D * 4 + (PK_D / 2) * 8));
+    if (threadIdx.x < 32) {
+      __syncwarp();
+      const int c = threadIdx.x, ldq = (P.nq + 2 * P.nkv) * PK_D;
+      fence_proxy_async_global();
+      if (c < 3 * R) {
+        const int r = c / 3, what = c - 3 * r;              // 0: the G query heads, 1: k, 2: v
         const float *src = P.qkv + (size_t)(b * R + r) * ldq;
         float *dst = reinterpret_cast<float *>(sc + PK_F_ROWS) + r * PK_AT_ROW_FLOATS;
-        stage_copy(S, dst, src + kvh * G * PK_D, (uint32_t)(G * PK_D * 4));
-        stage_copy(S, dst + G * PK_D, src + (P.nq + kvh) * PK_D, PK_D * 4);
-        stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
+        if (what == 0) stage_copy(S, dst, src + kvh * G * PK_D, (uint32_t)(G * PK_D * 4));
+        else if (what == 1) stage_copy(S, dst + G * PK_D, src + (P.nq + kvh) * PK_D, PK_D * 4);
+        else stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
+      } else if (c == 3 * R) {
+        stage_copy(S, sc + PK_F_W, Ly.w_qn, PK_D * 4);
+      } else if (c == 3 * R + 1) {
+        stage_copy(S, sc + PK_F_W + PK_D * 4, Ly.w_kn, PK_D * 4);
+      } else if (c == 3 * R + 2) {
+        stage_copy(S, sc + PK_F_W + 2 * PK_D * 4, P.inv_freq, (PK_D / 2) * 8);
       }
-      stage_copy(S, sc + PK_F_W, Ly.w_qn, PK_D * 4);
-      stage_copy(S, sc + PK_F_W + PK_D * 4, Ly.w_kn, PK_D * 4);
-      stage_copy(S, sc + PK_F_W + 2 * PK_D * 4, P.inv_freq, (PK_D / 2) * 8);
     }
     PK_SUBSTAMP(1);
     // cached rows of a tile: asynchronous 16-byte copies, 32 of K and 32 of V per row

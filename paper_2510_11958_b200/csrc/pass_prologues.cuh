@@ -36,10 +36,14 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
                                            const float *w_norm, const PackedMat &W) {
   const PassShared S = pass_shared();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, H = P.H;
-  if (threadIdx.x == 0) {
-    stage_begin(S, (uint32_t)(M * H * 4));
-#pragma unroll 1
-    for (int m = 0; m < M; ++m) stage_copy(S, S.xs + m * H, x + (size_t)m * row_stride, (uint32_t)(H * 4));
+  // one copy per row, each issued by its own lane of the first warp
+  if (threadIdx.x == 0) stage_begin(S, (uint32_t)(M * H * 4));
+  if (warp == 0) {
+    __syncwarp();
+    if (lane < M) {
+      fence_proxy_async_global();
+      stage_copy(S, S.xs + lane * H, x + (size_t)lane * row_stride, (uint32_t)(H * 4));
+    }
   }
   const SlabSpan sp = slab_span(W);
   const int ks4 = sp.KS / 4, nu = sp.count * ks4;
@@ -88,13 +92,16 @@ __device__ __noinline__ void swiglu_prologue(const PassParams &P, int M, const P
   const PassShared S = pass_shared();
   const SlabSpan sp = slab_span(W);
   const int ks4 = sp.KS / 4, ldgu = 2 * P.I, total = sp.count * M * ks4;
-  if (threadIdx.x == 0) {
-    stage_begin(S, (uint32_t)(sp.count * M * 2 * sp.KS * 4));
+  // two copies (gate values, up values) per (slab, row) i = sl * M + m, spread over the lanes of the first warp
+  if (threadIdx.x == 0) stage_begin(S, (uint32_t)(sp.count * M * 2 * sp.KS * 4));
+  if (threadIdx.x < 32) {
+    __syncwarp();
+    fence_proxy_async_global();
 #pragma unroll 1
-    for (int i = 0; i < sp.count * M; ++i) {             // i = sl * M + m: gate values, then up values
-      const float *src = P.gu + (size_t)(i % M) * ldgu + (sp.first + i / M) * sp.KS;
-      stage_copy(S, S.xs + (size_t)i * 2 * sp.KS, src, (uint32_t)(sp.KS * 4));
-      stage_copy(S, S.xs + (size_t)i * 2 * sp.KS + sp.KS, src + P.I, (uint32_t)(sp.KS * 4));
+    for (int c = threadIdx.x; c < 2 * sp.count * M; c += 32) {
+      const int i = c >> 1, up = c & 1;
+      const float *src = P.gu + (size_t)(i % M) * ldgu + (sp.first + i / M) * sp.KS + up * P.I;
+      stage_copy(S, S.xs + (size_t)i * 2 * sp.KS + up * sp.KS, src, (uint32_t)(sp.KS * 4));
     }
   }
   stage_wait(P, S);
