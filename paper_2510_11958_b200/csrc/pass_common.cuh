@@ -23,6 +23,11 @@
 //    the blocks, so nothing tells it when a buffer may be cleared or reused: one run in ten had a
 //    pass with logits off by 1e-2.  Dropped.  (atomicAdd on unsigned long long compiled to the
 //    returning form and slowed the weight loop by 15 %; red.global.add.u64 in PTX did not.)
+//  * handing the block's chunks to its warps from one shared counter (so that the warps of a
+//    block finish a projection together instead of 1-2 us apart) was tried: the bookkeeping per
+//    4 KiB chunk (shared-memory atomic, table look-ups, two divisions, slot records) sits
+//    between a slot becoming free and its next request, and the stream ran at half speed.
+//    Fixed per-warp shares keep that path to a few dozen instructions.
 //  * mma.sync issues about once per 30 cycles per SM sub-partition here: enough for the weight
 //    loop (one atom per ~90 cycles), too slow for attention with bf16 hi/lo pairs, which is
 //    why the fp32-cache attention stage uses FMAs.
