@@ -711,7 +711,6 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   CTRY(dev_alloc(c, &c->dstate, 1));
 
   // workspace
-  c->ws_rows = std::max(256, max_batch * std::max(tau, 8));
   c->lda = std::max(H, std::max(QD, I));
   c->ldqkv = QD + 2 * KVD; c->ldgu = 2 * I; c->ldl = (s.vocab + 15) / 16 * 16;
   // Keys per slice of the split-KV attention: enough slices that a decode step of max_batch
@@ -722,6 +721,10 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
     c->CH = std::max(64, ((max_seq + want - 1) / want + 63) / 64 * 64);
   }
   c->nsplit_max = (max_seq + c->CH - 1) / c->CH;
+  // Rows of the workspace = rows of one prefill chunk: up to 1024 (fewer, larger launches, and the
+  // row blocks of one sequence find its K and V in L2), less where many key slices would make
+  // the slices' partial results large; never fewer than a decode pass needs.
+  c->ws_rows = std::max(std::max(256, max_batch * std::max(tau, 8)), std::min(1024, 16384 / std::max(1, c->nsplit_max)));
   CTRY(dev_alloc(c, &c->x_lo, (size_t)c->ws_rows * H));
   CTRY(dev_alloc(c, &c->x_up, (size_t)max_batch * H));
   CTRY(dev_alloc(c, &c->act, (size_t)c->ws_rows * c->lda));
