@@ -238,29 +238,35 @@ dmtd_status launch_gemv_nt(dmtd_ctx *c, const PackedMat &W, const float *act, in
   return DMTD_OK;
 }
 
-// out[m][n] += sum_k W[n][k] act[m][k] on the tcgen05 tensor cores, 128 activation rows at a time.
+// out[m][n] += sum_k W[n][k] act[m][k] on the tcgen05 tensor cores.  A block multiplies a 128-row
+// weight tile with up to 128 activation rows (a sweep); prefill chunks of more rows are several
+// sweeps in one launch (up to TG_MAX_SWEEPS), ordered so that the sweeps of one weight tile run
+// together and share it through L2.
 dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, int lda, int M, float *out, int ldo) {
-  for (int m0 = 0; m0 < M; m0 += TG_MAX_COLS / 2) {
+  const int SET = TG_MAX_COLS / 2;                       // rows per sweep
+  for (int m0 = 0; m0 < M; m0 += TG_MAX_SWEEPS * SET) {
     GemmTcParams P{};
     P.W = W; P.act_blocks = c->act_blocks;
-    P.rows = std::min(TG_MAX_COLS / 2, M - m0);
-    P.n_cols = (2 * P.rows + 15) / 16 * 16;
+    P.rows = std::min(TG_MAX_SWEEPS * SET, M - m0);
+    P.n_sweeps = (P.rows + SET - 1) / SET;
+    P.n_cols = P.n_sweeps > 1 ? TG_MAX_COLS : (2 * P.rows + 15) / 16 * 16;
     P.out = out + (size_t)m0 * ldo; P.ldo = ldo;
     P.error = &c->dstate->error; P.wait_limit = 2000000000ll;
     // Every block of a launch should be resident at once (a block streams at the rate its own
     // stages allow, so a second round of blocks doubles the time): blocks per SM follow from
     // shared memory and tensor memory; with more row tiles than that, two-stage blocks make room
     // for two per SM.  Row tiles are then split along k over as many blocks as still fit.
+    // (Several sweeps fill the SMs by themselves: no k split then.)
     int tmem_cols = 32;
     while (tmem_cols < P.n_cols) tmem_cols <<= 1;
     auto smem_of = [&](int st) { return st * (TG_WBLOCK + P.n_cols * 128) + 128; };
     auto per_sm_of = [&](int st) { return std::max(1, std::min((227 * 1024) / (smem_of(st) + 1024), 512 / tmem_cols)); };
     P.stages = TG_STAGES;
-    if (W.n_tiles > c->n_sms * per_sm_of(TG_STAGES) && W.n_tiles <= c->n_sms * per_sm_of(2)) P.stages = 2;
+    if (P.n_sweeps == 1 && W.n_tiles > c->n_sms * per_sm_of(TG_STAGES) && W.n_tiles <= c->n_sms * per_sm_of(2)) P.stages = 2;
     const int slots = c->n_sms * per_sm_of(P.stages);
-    P.ksplit = std::max(1, std::min(W.n_kb, slots / W.n_tiles));
+    P.ksplit = std::max(1, std::min(W.n_kb, slots / (W.n_tiles * P.n_sweeps)));
     long long units = (long long)W.n_kb * 8 * P.n_cols;
-    act_blocks_kernel<<<(int)std::min<long long>((units + 255) / 256, 4096), 256, 0, c->stream>>>(
+    act_blocks_kernel<<<dim3((int)std::min<long long>((units + 255) / 256, 4096), P.n_sweeps), 256, 0, c->stream>>>(
         act + (size_t)m0 * lda, lda, P.rows, W.K, P.n_cols, c->act_blocks);
     LAUNCH_OK(c, "act_blocks_kernel");
     int smem = smem_of(P.stages);
@@ -273,7 +279,7 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
     // launched with programmatic stream serialisation: its blocks may start (allocate tensor
     // memory, request their first weight blocks) while act_blocks_kernel is still running
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(W.n_tiles * P.ksplit); cfg.blockDim = dim3(TG_THREADS);
+    cfg.gridDim = dim3(W.n_tiles * P.ksplit * P.n_sweeps); cfg.blockDim = dim3(TG_THREADS);
     cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = c->stream;
     cudaLaunchAttribute attr{};
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -736,7 +742,7 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   CTRY(dev_alloc(c, &c->part_o, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * D));
   CTRY(dev_alloc(c, &c->part_ml, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * 2));
   CTRY(dev_alloc(c, &c->rope_tab, (size_t)c->ws_rows * (D / 2)));
-  if (c->umma_ok) CTRY(dev_alloc(c, &c->act_blocks, (size_t)(c->lda / TG_KB) * 8 * TG_MAX_COLS));
+  if (c->umma_ok) CTRY(dev_alloc(c, &c->act_blocks, (size_t)TG_MAX_SWEEPS * (c->lda / TG_KB) * 8 * TG_MAX_COLS));
   CTRY(setup_fused(c));
   CTRY(dmtd_reset(c));
   CCUDA(cudaStreamSynchronize(c->stream));   // repacking done: the caller may free its weights

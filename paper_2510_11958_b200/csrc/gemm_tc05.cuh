@@ -26,6 +26,7 @@ constexpr int TG_ROWS = 128;                 // weight rows per tile (MMA M)
 constexpr int TG_KB = 64;                    // k per pipeline stage: four MMAs of K = 16
 constexpr int TG_WBLOCK = TG_ROWS * TG_KB * 2;      // 16384 bytes
 constexpr int TG_MAX_COLS = 256;             // MMA N: two columns per activation row
+constexpr int TG_MAX_SWEEPS = 8;             // sweeps of 128 activation rows in one launch
 enum { TG_ERR_WAIT = 4 };
 
 // A weight matrix [N][K] as 16 KiB blocks [row tile][k block][k chunk 8][row group 16][row 8][8 values].
@@ -45,6 +46,10 @@ struct GemmTcParams {
   int ldo;
   int ksplit;                // blocks per row tile, each taking a share of the k blocks
   int stages;                // pipeline stages of a block, 2 .. TG_STAGES
+  int n_sweeps;              // sets of up to 128 activation rows in this launch (prefill chunks); set s has its
+                             // activation blocks s * n_kb blocks further and its output rows 128 s further.
+                             // Consecutive blocks of the grid are the sweeps of one (row tile, k share): they
+                             // run together, and all but the first find the weight blocks in L2.
   int *error;
   long long wait_limit;
 };
@@ -82,7 +87,11 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * S + 1);
   const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + S), done = smem_u32(bars + 2 * S);
 
-  const int tile = blockIdx.x / P.ksplit, ks = blockIdx.x % P.ksplit;
+  const int sweep = blockIdx.x % P.n_sweeps, unit = blockIdx.x / P.n_sweeps;
+  const int tile = unit / P.ksplit, ks = unit % P.ksplit;
+  const int rows = min(TG_MAX_COLS / 2, P.rows - sweep * (TG_MAX_COLS / 2));        // rows of this sweep
+  const uint4 *act_blocks = P.act_blocks + (size_t)sweep * P.W.n_kb * (P.n_cols * 8);
+  float *out = P.out + (size_t)sweep * (TG_MAX_COLS / 2) * P.ldo;
   const int kb0 = P.W.n_kb * ks / P.ksplit, kb1 = P.W.n_kb * (ks + 1) / P.ksplit, n_it = kb1 - kb0;
   int tmem_cols = 32;
   while (tmem_cols < P.n_cols) tmem_cols <<= 1;
@@ -113,7 +122,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int i = 0; i < n_first; ++i)
-      bulk_g2s(smem_u32(tg_smem + i * stage_bytes) + TG_WBLOCK, P.act_blocks + (size_t)(kb0 + i) * (act_block / 16),
+      bulk_g2s(smem_u32(tg_smem + i * stage_bytes) + TG_WBLOCK, act_blocks + (size_t)(kb0 + i) * (act_block / 16),
                (uint32_t)act_block, full0 + i * 8);
     for (int i = n_first; i < n_it; ++i) {
       const int st = i % S;
@@ -121,7 +130,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
       const uint32_t dst = smem_u32(tg_smem + st * stage_bytes);
       mbar_expect_tx(full0 + st * 8, (uint32_t)stage_bytes);
       bulk_g2s(dst, P.W.w + ((size_t)tile * P.W.n_kb + kb0 + i) * (TG_WBLOCK / 16), TG_WBLOCK, full0 + st * 8);
-      bulk_g2s(dst + TG_WBLOCK, P.act_blocks + (size_t)(kb0 + i) * (act_block / 16), (uint32_t)act_block, full0 + st * 8);
+      bulk_g2s(dst + TG_WBLOCK, act_blocks + (size_t)(kb0 + i) * (act_block / 16), (uint32_t)act_block, full0 + st * 8);
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer: four K = 16 MMAs per k block, then release the stage
@@ -155,7 +164,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
     const int n = tile * TG_ROWS + quarter * 32 + lane;
     if (tg_wait(done, 0, P)) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      for (int c0 = 0; c0 < P.n_cols; c0 += 16) {
+      for (int c0 = 0; c0 < P.n_cols && c0 < 2 * rows; c0 += 16) {
         uint32_t r[16];
         asm volatile(
             "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
@@ -166,7 +175,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int m = (c0 >> 1) + j;                  // columns 2m (hi) and 2m + 1 (lo) belong to activation row m
-          if (m < P.rows && n < P.W.N) atomicAdd(P.out + (size_t)m * P.ldo + n, __uint_as_float(r[2 * j]) + __uint_as_float(r[2 * j + 1]));
+          if (m < rows && n < P.W.N) atomicAdd(out + (size_t)m * P.ldo + n, __uint_as_float(r[2 * j]) + __uint_as_float(r[2 * j + 1]));
         }
       }
     }
@@ -181,8 +190,13 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
 // Activations [rows][lda] fp32 -> bf16 hi/lo columns in the canonical K-major block order:
 // block kb holds k = 64 kb .. 64 kb + 63 as [k chunk 8][column group n_cols/8][column 8][8 values];
 // column 2m is the hi part of row m, column 2m + 1 its lo part; columns beyond 2 * rows are zero.
-__global__ void act_blocks_kernel(const float *__restrict__ act, int lda, int rows, int K, int n_cols,
-                                  uint4 *__restrict__ blocks) {
+// blockIdx.y = set of up to 128 rows (a sweep of the GEMM): its rows start 128 y further, its
+// blocks n_kb blocks further.
+__global__ void act_blocks_kernel(const float *__restrict__ act_all, int lda, int rows_all, int K, int n_cols,
+                                  uint4 *__restrict__ blocks_all) {
+  const int rows = min(TG_MAX_COLS / 2, rows_all - (int)blockIdx.y * (TG_MAX_COLS / 2));
+  const float *act = act_all + (size_t)blockIdx.y * (TG_MAX_COLS / 2) * lda;
+  uint4 *blocks = blocks_all + (size_t)blockIdx.y * (K / TG_KB) * (n_cols * 8);
   // the GEMM that follows may be scheduled already: it waits for this grid before it reads the blocks
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int n_kb = K / TG_KB;
