@@ -242,7 +242,8 @@ dmtd_status launch_gemv_nt(dmtd_ctx *c, const PackedMat &W, const float *act, in
 // weight tile with up to 128 activation rows (a sweep); prefill chunks of more rows are several
 // sweeps in one launch (up to TG_MAX_SWEEPS), ordered so that the sweeps of one weight tile run
 // together and share it through L2.
-dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, int lda, int M, float *out, int ldo) {
+dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, int lda, int M, float *out, int ldo,
+                             int gate_up_I = 0) {
   const int SET = TG_MAX_COLS / 2;                       // rows per sweep
   for (int m0 = 0; m0 < M; m0 += TG_MAX_SWEEPS * SET) {
     GemmTcParams P{};
@@ -267,7 +268,7 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
     P.ksplit = std::max(1, std::min(W.n_kb, slots / (W.n_tiles * P.n_sweeps)));
     long long units = (long long)W.n_kb * 8 * P.n_cols;
     act_blocks_kernel<<<dim3((int)std::min<long long>((units + 255) / 256, 4096), P.n_sweeps), 256, 0, c->stream>>>(
-        act + (size_t)m0 * lda, lda, P.rows, W.K, P.n_cols, c->act_blocks);
+        act + (size_t)m0 * lda, lda, P.rows, W.K, P.n_cols, c->act_blocks, gate_up_I);
     LAUNCH_OK(c, "act_blocks_kernel");
     int smem = smem_of(P.stages);
     static int configured = 0;
@@ -401,9 +402,14 @@ dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos
       x, H, lw.w_post, H, s.rms_eps, c->act, c->lda, c->gu, c->ldgu, c->ldgu);
   LAUNCH_OK(c, "prep_norm_kernel");
   TRY(launch_gemv(c, lw.gu, lw.gu_u, c->act, c->lda, M, c->gu, c->ldgu));
-  prep_swiglu_kernel<<<dim3((I + 255) / 256, M), 256, 0, c->stream>>>(c->gu, c->ldgu, I, c->act, c->lda);
-  LAUNCH_OK(c, "prep_swiglu_kernel");
-  TRY(launch_gemv(c, lw.down, lw.down_u, c->act, c->lda, M, x, H));
+  if (lw.down_u.w && c->use_umma && M > 8) {
+    // the tcgen05 path gates while it writes its activation blocks
+    TRY(launch_gemm_tc05(c, lw.down_u, c->gu, c->ldgu, M, x, H, I));
+  } else {
+    prep_swiglu_kernel<<<dim3((I + 255) / 256, M), 256, 0, c->stream>>>(c->gu, c->ldgu, I, c->act, c->lda);
+    LAUNCH_OK(c, "prep_swiglu_kernel");
+    TRY(launch_gemv(c, lw.down, lw.down_u, c->act, c->lda, M, x, H));
+  }
   return DMTD_OK;
 }
 

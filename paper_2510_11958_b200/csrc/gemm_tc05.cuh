@@ -192,8 +192,10 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
 // column 2m is the hi part of row m, column 2m + 1 its lo part; columns beyond 2 * rows are zero.
 // blockIdx.y = set of up to 128 rows (a sweep of the GEMM): its rows start 128 y further, its
 // blocks n_kb blocks further.
+// With gate_up_I > 0 the source rows hold gate | up values (gate at k, up at gate_up_I + k) and the
+// activation is the SwiGLU gate silu(gate) * up (step a6, second half), computed on the way.
 __global__ void act_blocks_kernel(const float *__restrict__ act_all, int lda, int rows_all, int K, int n_cols,
-                                  uint4 *__restrict__ blocks_all) {
+                                  uint4 *__restrict__ blocks_all, int gate_up_I) {
   const int rows = min(TG_MAX_COLS / 2, rows_all - (int)blockIdx.y * (TG_MAX_COLS / 2));
   const float *act = act_all + (size_t)blockIdx.y * (TG_MAX_COLS / 2) * lda;
   uint4 *blocks = blocks_all + (size_t)blockIdx.y * (K / TG_KB) * (n_cols * 8);
@@ -208,7 +210,14 @@ __global__ void act_blocks_kernel(const float *__restrict__ act_all, int lda, in
     if (m < rows) {
       const float4 a = *reinterpret_cast<const float4 *>(act + (size_t)m * lda + k);
       const float4 b = *reinterpret_cast<const float4 *>(act + (size_t)m * lda + k + 4);
-      const float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+      float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+      if (gate_up_I > 0) {
+        const float4 ua = *reinterpret_cast<const float4 *>(act + (size_t)m * lda + gate_up_I + k);
+        const float4 ub = *reinterpret_cast<const float4 *>(act + (size_t)m * lda + gate_up_I + k + 4);
+        const float u[8] = {ua.x, ua.y, ua.z, ua.w, ub.x, ub.y, ub.z, ub.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) f[j] = f[j] / (1.f + expf(-f[j])) * u[j];
+      }
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const uint32_t h = pack_bf16x2(f[2 * j], f[2 * j + 1]);
