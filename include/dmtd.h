@@ -203,7 +203,7 @@ dmtd_status dmtd_set_tau(dmtd_ctx *ctx, int32_t tau);
  *   "tc_attention" 0/1  attention of the per-step kernels by the tiled split-KV kernels for
  *                       head_dim 128 (tensor cores with a bf16 cache, FMAs with an fp32 cache)
  *                       instead of the one-warp-per-key-group kernel (default 1)
- *   "tcgen05_gemm" 0/1  projections of more than 8 rows (prefill chunks included) on the tcgen05
+ *   "tcgen05_gemm" 0/1  projections of more than 4 rows (prefill chunks included) on the tcgen05
  *                       tensor cores; bf16 contexts whose hidden, query and intermediate sizes
  *                       are multiples of 64 hold the second weight copy it reads, which doubles
  *                       the weight memory of the context (default 1)

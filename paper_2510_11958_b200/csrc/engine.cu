@@ -47,7 +47,7 @@ struct dmtd_ctx {
   std::vector<LayerDev> layers;
   PackedMat embed{};
   UmmaMat embed_u{};
-  bool umma_ok = false, use_umma = true;    // tcgen05 GEMM for projections of more than 8 rows
+  bool umma_ok = false, use_umma = true;    // tcgen05 GEMM for projections of more than 4 rows
   uint4 *act_blocks = nullptr;
   float *w_final = nullptr;
   double *inv_freq = nullptr;
@@ -295,7 +295,7 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
 // out[m][n] += sum_k W[n][k] act[m][k]
 dmtd_status launch_gemv(dmtd_ctx *c, const PackedMat &W, const UmmaMat &U, const float *act, int lda, int M, float *out,
                         int ldo) {
-  if (U.w && c->use_umma && M > 8) return launch_gemm_tc05(c, U, act, lda, M, out, ldo);
+  if (U.w && c->use_umma && M > 4) return launch_gemm_tc05(c, U, act, lda, M, out, ldo);
   if (W.wf) {
     gemv_f32_kernel<<<2 * c->n_sms, 256, 0, c->stream>>>(W, act, lda, M, out, ldo);
     LAUNCH_OK(c, "gemv_f32_kernel");
@@ -402,7 +402,7 @@ dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos
       x, H, lw.w_post, H, s.rms_eps, c->act, c->lda, c->gu, c->ldgu, c->ldgu);
   LAUNCH_OK(c, "prep_norm_kernel");
   TRY(launch_gemv(c, lw.gu, lw.gu_u, c->act, c->lda, M, c->gu, c->ldgu));
-  if (lw.down_u.w && c->use_umma && M > 8) {
+  if (lw.down_u.w && c->use_umma && M > 4) {
     // the tcgen05 path gates while it writes its activation blocks
     TRY(launch_gemm_tc05(c, lw.down_u, c->gu, c->ldgu, M, x, H, I));
   } else {
@@ -662,7 +662,7 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   const int H = s.hidden, D = s.head_dim, QD = s.n_q_heads * D, KVD = s.n_kv_heads * D, I = s.intermediate;
 
   // weights; every bf16 context whose dimensions fit also gets the copy the tcgen05 GEMM reads:
-  // passes of more than 8 rows (batch x cycle length) and the prefill of every context use it
+  // passes of more than 4 rows (batch x cycle length) and the prefill of every context use it
   c->umma_ok = s.weight_dtype == DMTD_BF16 && H % TG_KB == 0 && QD % TG_KB == 0 && I % TG_KB == 0;
   c->layers.resize(s.n_layers);
   // k-slab width of the packed matrices: contexts small enough for the pass kernel (which stages

@@ -1,5 +1,5 @@
 // Skinny GEMM on the 5th-generation tensor cores (tcgen05, sm_100a) for projections with many
-// activation rows: out[m][n] += sum_k W[n][k] act[m][k] for 9..128 rows m.
+// activation rows: out[m][n] += sum_k W[n][k] act[m][k] for 5..128 rows m.
 //
 // Operands are swapped against the usual orientation: the 128 weight rows of a tile are the M
 // axis of the MMA, the activation rows its N axis (each row as two columns, the bf16 hi and lo

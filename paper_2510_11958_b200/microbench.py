@@ -100,7 +100,7 @@ def main():
                     "attention_gbs": kv_bytes / (t_attn * 1e-3) / 1e9,
                     "projections_ms_by_difference": t_layer - t_attn,
                     "projections_gbs_by_difference": w_layer / max(t_layer - t_attn, 1e-6) / 1e6,
-                    "projection_kernel": "gemv_bf16 (mma.sync)" if B <= 8 else "gemm_tc05 (tcgen05)",
+                    "projection_kernel": "gemv_bf16 (mma.sync)" if B <= 4 else "gemm_tc05 (tcgen05)",
                     "hbm_peak_gbs": peak, "layer_frac_of_peak": (w_layer + kv_bytes) / (t_layer * 1e-3) / 1e9 / peak,
                     "l2": "flushed between iterations"}
             print(json.dumps(line), flush=True)
