@@ -408,3 +408,84 @@ def test_step_layers_matches_pass():
         kb, vb = b.kv_cache(l, 0, 6)
         np.testing.assert_array_equal(ka, kb)
         np.testing.assert_array_equal(va, vb)
+
+
+# ----------------------------------------------------------------------------- corners named by review
+
+def test_chunked_prefill_equals_unchunked_forward():
+    """The prefill feeds prompts longer than 256 rows in causal chunks; a wrong chunk origin (rows
+    of the second chunk rotated or cached at the first chunk's positions) would pass every pin
+    with a short prompt.  The no-cache, no-chunk forward over the same 300 tokens must give the
+    same logits for the first generated token."""
+    shape = TINY
+    w = make_weights(shape, seed=4, norm_jitter=0.1)
+    P = 300
+    prompt = make_prompts(shape.vocab, 1, P, seed=9).numpy()
+    o = oracle.Oracle(shape, w, L_d=2, tau=3, max_seq=P + 4)
+    tok, logits = o.prefill(prompt)
+    vt, vl, vam = oracle.vanilla_generate(shape, w, prompt[0], 1)
+    np.testing.assert_allclose(logits[0], vl[0], rtol=0, atol=1e-11)
+    assert int(tok[0]) == int(vam[0])
+    # and the cache rows of the second chunk sit at their own positions: one more (short) pass
+    # through the decoding layers reads them
+    rc, t, lg = o.decode_cycle(1)
+    seq = np.concatenate([prompt[0], tok]).astype(np.int32)
+    ref = oracle.masked_parallel_forward(shape, w, 2, 3, seq, P)
+    np.testing.assert_allclose(lg[0, 0], ref[1], rtol=0, atol=1e-11)
+
+
+def test_argmax_picks_lowest_index_on_exact_tie():
+    """Two identical embedding rows give bit-identical logits at their two vocabulary entries
+    (identity layers: o_proj = down_proj = 0).  Make that pair the maximum: the lower index
+    must be emitted.  `>=` in place of `>` in the pick would emit the higher one."""
+    shape = TINY
+    w = make_weights(shape, seed=2)
+    for lw in w["layers"]:
+        lw["o_proj"].zero_()
+        lw["down_proj"].zero_()
+    lo, hi, last = 17, 801, 5
+    # logits = rmsnorm(E[last]) . E[v]: the row parallel to E[last] with a large norm wins
+    w["embed"][lo] = 3.0 * w["embed"][last]
+    w["embed"][hi] = w["embed"][lo]
+    prompt = np.array([[9, 3, last]], np.int32)
+    o = oracle.Oracle(shape, w, L_d=2, tau=3, max_seq=16)
+    tok, logits = o.prefill(prompt)
+    assert logits[0, lo] == logits[0, hi] == logits[0].max()
+    assert int(tok[0]) == lo
+    # the same through a decode pass
+    w2 = {"embed": w["embed"].clone(), "final_norm": w["final_norm"], "layers": w["layers"]}
+    o2 = oracle.Oracle(shape, w2, L_d=2, tau=3, max_seq=16)
+    o2.prefill(prompt, forced_first=np.array([last], np.int32))
+    rc, t, lg = o2.decode_cycle(1)
+    assert lg[0, 0, lo] == lg[0, 0, hi] == lg[0, 0].max()
+    assert int(t[0, 0]) == lo
+
+
+def test_set_tau_after_prefill_at_cycle_boundary():
+    """The cycle length may change between cycles (Section 3.7 evaluates inference cycle lengths
+    other than the training one).  A change in mid-cycle is refused; after a change at a boundary
+    the next full pass still refills every pending position of the old cycle, and the cycles that
+    follow have the new length: the pass trace says which positions enter which layers."""
+    shape = TINY
+    w = make_weights(shape, seed=0)
+    P = 6
+    prompt = make_prompts(shape.vocab, 1, P, seed=1).numpy()
+    o = oracle.Oracle(shape, w, L_d=2, tau=3, max_seq=40)
+    o.prefill(prompt)
+    assert o.set_tau(2) == -3                   # mid-cycle: refused
+    o.decode_cycle(3)                           # finishes cycle 1 (2 short passes)
+    assert o.state()["slot"] == 0
+    assert o.set_tau(2) == 0
+    st = o.state()
+    assert st["tau"] == 2 and st["n_known"] == P + 3
+    rc, t, lg = o.decode_cycle(2)
+    assert rc == 0 and t.shape[1] == 2
+    tr = o.trace()
+    # pass 3: full pass refills the two pending positions and the newest, then one short pass
+    assert (tr[3]["kind"], tr[3]["lo_begin"], tr[3]["lo_end"], tr[3]["up_begin"]) == (1, P, P + 3, P + 2)
+    assert (tr[4]["kind"], tr[4]["up_begin"]) == (2, P + 3)
+    rc, t2, lg2 = o.decode_cycle(2)
+    tr = o.trace()
+    assert (tr[5]["kind"], tr[5]["lo_begin"], tr[5]["lo_end"]) == (1, P + 3, P + 5)
+    st = o.state()
+    assert st["cycle"] == 3 and st["lo_len"] == P + 5 and st["slot"] == 0
