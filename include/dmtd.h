@@ -22,6 +22,14 @@
  *   - Sequences of a batch advance in lock-step and have equal prompt length; there is no
  *     end-of-sequence handling (generation stops after the requested number of tokens).
  *   - Greedy decoding: argmax of the logits, lowest index on ties.
+ *   - Device-side checks (a token id outside [0, vocab), which is clamped; a bounded wait of a
+ *     kernel that ran out) set a sticky error word in device memory; no kernel traps.  Every
+ *     call that synchronises the stream (dmtd_prefill_host, dmtd_decode_cycle_host,
+ *     dmtd_get_device_state) reads the word and returns INVALID_ARG (token id) or TIMEOUT
+ *     (wait).  From then on every call that would run kernels returns that status until
+ *     dmtd_reset; the asynchronous calls made between the fault and its discovery have
+ *     returned OK and advanced the host's copy of the schedule state, and what they produced
+ *     is invalid.
  */
 #ifndef DMTD_H
 #define DMTD_H
@@ -87,7 +95,8 @@ typedef struct {
  * and for V) and the workspace.  `cuda_stream` is a cudaStream_t (NULL = default stream).
  * Errors: SHAPE if L_d not in [1, L], tau < 1, n_q_heads % n_kv_heads != 0, head_dim not 64
  * or 128, n_q_heads/n_kv_heads > 16, hidden or intermediate not a multiple of 32 (bf16) or
- * 4 (fp32), lm_head not tied; CUDA if an allocation fails. */
+ * 4 (fp32); UNSUPPORTED if the LM head is not tied (tied_lm_head == 0 or lm_head != NULL);
+ * CUDA if an allocation fails. */
 dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
                         int32_t max_batch, int32_t max_seq, const dmtd_weights *weights,
                         void *cuda_stream, dmtd_ctx **out);
@@ -185,7 +194,8 @@ dmtd_status dmtd_decode_cycle_host(dmtd_ctx *ctx, int32_t max_new, int32_t *out_
                                    int32_t *n_out);
 
 /* The schedule state as the host tracks it / as the device counters hold it (the second
- * synchronises the stream).  The two always agree; tests compare both with the oracle. */
+ * synchronises the stream).  The two agree unless a device-side error was reported (see
+ * Conventions); tests compare both with the oracle. */
 dmtd_status dmtd_get_state(const dmtd_ctx *ctx, dmtd_state *out);
 dmtd_status dmtd_get_device_state(dmtd_ctx *ctx, dmtd_state *out);
 
@@ -213,6 +223,12 @@ dmtd_status dmtd_set_option(dmtd_ctx *ctx, const char *name, int64_t value);
 /* KV cache of one layer for inspection or for filling with test data: device pointers to
  * [max_batch][n_kv_heads][max_seq][head_dim] in kv_dtype. */
 dmtd_status dmtd_get_kv(dmtd_ctx *ctx, int32_t layer, void **k, void **v);
+
+/* Diagnostics: write the context's device error word from the host, as a device-side check
+ * would (1 = token id out of range, 2 = weight-copy wait, 3 = grid-barrier wait, 4 =
+ * tensor-core pipeline wait; 0 clears it).  Lets the error path of the synchronising calls be
+ * exercised without making a GPU wait run out.  Synchronises the stream. */
+dmtd_status dmtd_debug_set_error_word(dmtd_ctx *ctx, int32_t word);
 
 /* Number of this library's kernels launched on the stream since create (graph replays count
  * their kernel nodes). */

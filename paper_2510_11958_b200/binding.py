@@ -89,6 +89,7 @@ def load_library():
         "dmtd_set_option": [vp, C.c_char_p, i64],
         "dmtd_get_kv": [vp, i32, C.POINTER(vp), C.POINTER(vp)],
         "dmtd_get_launch_count": [vp, C.POINTER(i64)],
+        "dmtd_debug_set_error_word": [vp, i32],
         "dmtd_attention_decode": [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp, C.c_size_t, vp, vp],
         "dmtd_attention_decode_static": [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp],
     }
@@ -240,6 +241,9 @@ class Dmtd:
         k, v = C.c_void_p(), C.c_void_p()
         self._check(self.dll.dmtd_get_kv(self._ctx, layer, C.byref(k), C.byref(v)))
         return k.value, v.value
+
+    def debug_set_error_word(self, word):
+        self._check(self.dll.dmtd_debug_set_error_word(self._ctx, int(word)))
 
     def launch_count(self):
         n = C.c_int64(0)

@@ -26,6 +26,10 @@ namespace {
 
 thread_local std::string g_create_error;
 
+// Clock ticks a device-side wait (grid barrier, bulk-copy or tensor-core barrier) may spin before
+// it gives up and reports through the context's error word: about a second of SM clock.
+constexpr long long kDeviceWaitLimitTicks = 2000000000ll;
+
 struct LayerDev {
   PackedMat qkv, o, gu, down;
   UmmaMat qkv_u{}, o_u{}, gu_u{}, down_u{};     // second copy for the tcgen05 GEMM (contexts with many rows)
@@ -57,6 +61,8 @@ struct dmtd_ctx {
   size_t kv_layer_elems = 0;
   int *tokens = nullptr;                    // [max_batch][max_seq]
   DevState *dstate = nullptr;
+  int *h_error = nullptr;                   // pinned host copy of the device error word, refreshed by calls that synchronise
+  dmtd_status device_failure = DMTD_OK;     // sticky until dmtd_reset: a device-side check or wait reported an error
   dmtd_state h{};                           // host mirror
   bool prefilled = false;
   int B = 0;
@@ -228,11 +234,6 @@ int gemv_smem_bytes(const PackedMat &W, int NT) {
 template <int NT>
 dmtd_status launch_gemv_nt(dmtd_ctx *c, const PackedMat &W, const float *act, int lda, int M, float *out, int ldo) {
   int smem = gemv_smem_bytes(W, NT);
-  static int configured = 0;
-  if (configured < smem) {
-    CUDA_TRY(c, cudaFuncSetAttribute(gemv_bf16_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
-    configured = 100 * 1024;
-  }
   gemv_bf16_kernel<NT><<<2 * c->n_sms, GEMV_THREADS, smem, c->stream>>>(W, act, lda, M, out, ldo);
   LAUNCH_OK(c, "gemv_bf16_kernel");
   return DMTD_OK;
@@ -252,7 +253,7 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
     P.n_sweeps = (P.rows + SET - 1) / SET;
     P.n_cols = P.n_sweeps > 1 ? TG_MAX_COLS : (2 * P.rows + 15) / 16 * 16;
     P.out = out + (size_t)m0 * ldo; P.ldo = ldo;
-    P.error = &c->dstate->error; P.wait_limit = 2000000000ll;
+    P.error = &c->dstate->error; P.wait_limit = kDeviceWaitLimitTicks;
     // Every block of a launch should be resident at once (a block streams at the rate its own
     // stages allow, so a second round of blocks doubles the time): blocks per SM follow from
     // shared memory and tensor memory; with more row tiles than that, two-stage blocks make room
@@ -271,12 +272,6 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
         act + (size_t)m0 * lda, lda, P.rows, W.K, P.n_cols, c->act_blocks, gate_up_I);
     LAUNCH_OK(c, "act_blocks_kernel");
     int smem = smem_of(P.stages);
-    static int configured = 0;
-    if (configured < smem) {
-      CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       TG_STAGES * (TG_WBLOCK + TG_MAX_COLS * 128) + 128));
-      configured = TG_STAGES * (TG_WBLOCK + TG_MAX_COLS * 128) + 128;
-    }
     // launched with programmatic stream serialisation: its blocks may start (allocate tensor
     // memory, request their first weight blocks) while act_blocks_kernel is still running
     cudaLaunchConfig_t cfg{};
@@ -320,29 +315,15 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
   int RB = std::max(1, ATTN_QR / G), n_rb = (R + RB - 1) / RB;
   if (D == PK_D && c->use_tc_attention) {
     // head_dim 128: the tensor-core kernel with a bf16 cache, the FMA kernel with an fp32 cache
-    static bool tc_configured = false;
     if constexpr (std::is_same<KVT, float>::value) {
-      if (!tc_configured) {
-        CUDA_TRY(c, cudaFuncSetAttribute(attn_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_F32_SMEM));
-        tc_configured = true;
-      }
       attn_f32_kernel<<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_F32_SMEM, c->stream>>>(
           c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
     } else {
-      if (!tc_configured) {
-        CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM));
-        tc_configured = true;
-      }
       attn_tc_kernel<<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
           c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
     }
   } else {
   size_t smem = (size_t)ATTN_WARPS * ATTN_QR * D * sizeof(float);
-  static bool configured = false;
-  if (!configured) {
-    CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<D, KVT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
-    configured = true;
-  }
   attn_partial_kernel<D, KVT><<<dim3(nsplit, s.n_kv_heads * n_rb, B), ATTN_WARPS * 32, smem, c->stream>>>(
       c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml,
       nsplit);
@@ -432,6 +413,24 @@ dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, floa
   return DMTD_OK;
 }
 
+// Kernels that need more than 48 KiB of dynamic shared memory must be told so once per device
+// (the attribute belongs to the device's copy of the kernel, not to the process): done at create,
+// with the context's device current.
+dmtd_status configure_kernels(dmtd_ctx *c) {
+  const auto dyn = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  CUDA_TRY(c, cudaFuncSetAttribute(gemv_bf16_kernel<1>, dyn, 100 * 1024));
+  CUDA_TRY(c, cudaFuncSetAttribute(gemv_bf16_kernel<2>, dyn, 100 * 1024));
+  CUDA_TRY(c, cudaFuncSetAttribute(gemv_bf16_kernel<4>, dyn, 100 * 1024));
+  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc05_kernel, dyn, TG_STAGES * (TG_WBLOCK + TG_MAX_COLS * 128) + 128));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_f32_kernel, dyn, ATTN_F32_SMEM));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel, dyn, ATTN_TC_SMEM));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<64, float>, dyn, 64 * 1024));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<64, __nv_bfloat16>, dyn, 64 * 1024));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<128, float>, dyn, 64 * 1024));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<128, __nv_bfloat16>, dyn, 64 * 1024));
+  return DMTD_OK;
+}
+
 // ---------------------------------------------------------------------------- fused pass
 
 // Can the block-per-SM pass kernel stream this matrix?  Its k-slab must fit the staging area
@@ -516,7 +515,7 @@ dmtd_status enqueue_pass_fused(dmtd_ctx *c, int kind, int R_lower, bool write_to
   P.timing = c->pass_timing;
   P.part_o = c->f_part_o; P.part_ml = c->f_part_ml; P.amax_val = c->amax_val; P.amax_idx = c->amax_idx;
   P.out_argmax = out_argmax; P.barrier = c->grid_bar; P.error = &c->dstate->error;
-  P.wait_limit = 2000000000ll;              // about a second of SM clock
+  P.wait_limit = kDeviceWaitLimitTicks;
   CUDA_TRY(c, cudaMemsetAsync(c->grid_bar, 0, sizeof(unsigned int), c->stream));
   void *args[] = {&P};
   CUDA_TRY(c, cudaLaunchCooperativeKernel((const void *)dmtd_pass_kernel, dim3(c->n_sms), dim3(PK_THREADS), args,
@@ -562,6 +561,30 @@ void host_advance(dmtd_ctx *c, int kind) {
   h.slot = (h.slot + 1) % h.tau;
   h.n_emitted += 1;
 }
+
+// Calls that return results to the host synchronise the stream anyway: they bring the device's
+// error word along (4 bytes into pinned memory, queued before the synchronise) and turn it into a
+// status.  The word is sticky on the device and the failure is sticky here until dmtd_reset.
+dmtd_status queue_error_read(dmtd_ctx *c) {
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_error, &c->dstate->error, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  return DMTD_OK;
+}
+dmtd_status device_error_status(dmtd_ctx *c, int word) {
+  if (word == 0) return DMTD_OK;
+  if (word == PK_ERR_TOKEN) {
+    c->device_failure = DMTD_ERR_INVALID_ARG;
+    return fail(c, DMTD_ERR_INVALID_ARG, "a token id outside [0, vocab) reached the embedding gather; "
+                "the results since then are invalid, call dmtd_reset");
+  }
+  c->device_failure = DMTD_ERR_TIMEOUT;
+  return fail(c, DMTD_ERR_TIMEOUT, "a device-side wait gave up (%s); the results since then are invalid, call dmtd_reset",
+              word == PK_ERR_COPY_WAIT ? "weight copy" : word == PK_ERR_BARRIER_WAIT ? "grid barrier" : "tensor-core pipeline");
+}
+#define CHECK_NOT_FAILED(c)                                                                          \
+  do {                                                                                               \
+    if ((c)->device_failure != DMTD_OK)                                                              \
+      return fail((c), (c)->device_failure, "the context reported a device-side error earlier; call dmtd_reset"); \
+  } while (0)
 
 void drop_graphs(dmtd_ctx *c) {
   for (int k = 0; k < 3; ++k)
@@ -721,6 +744,8 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   }
   CTRY(dev_alloc(c, &c->tokens, (size_t)max_batch * max_seq));
   CTRY(dev_alloc(c, &c->dstate, 1));
+  CCUDA(cudaHostAlloc(reinterpret_cast<void **>(&c->h_error), sizeof(int), cudaHostAllocDefault));
+  *c->h_error = 0;
 
   // workspace
   c->lda = std::max(H, std::max(QD, I));
@@ -749,6 +774,7 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   CTRY(dev_alloc(c, &c->part_ml, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * 2));
   CTRY(dev_alloc(c, &c->rope_tab, (size_t)c->ws_rows * (D / 2)));
   if (c->umma_ok) CTRY(dev_alloc(c, &c->act_blocks, (size_t)TG_MAX_SWEEPS * (c->lda / TG_KB) * 8 * TG_MAX_COLS));
+  CTRY(configure_kernels(c));
   CTRY(setup_fused(c));
   CTRY(dmtd_reset(c));
   CCUDA(cudaStreamSynchronize(c->stream));   // repacking done: the caller may free its weights
@@ -764,6 +790,7 @@ void dmtd_destroy(dmtd_ctx *c) {
   drop_graphs(c);
   if (c->capture_stream) cudaStreamDestroy(c->capture_stream);
   for (void *p : c->allocs) cudaFree(p);
+  if (c->h_error) cudaFreeHost(c->h_error);
   delete c;
 }
 
@@ -776,6 +803,8 @@ dmtd_status dmtd_reset(dmtd_ctx *c) {
   c->h = dmtd_state{};
   c->h.tau = c->tau; c->h.L_d = c->L_d;
   c->prefilled = false; c->B = 0;
+  c->device_failure = DMTD_OK;
+  if (c->h_error) *c->h_error = 0;
   return DMTD_OK;
 }
 
@@ -783,6 +812,7 @@ dmtd_status dmtd_prefill(dmtd_ctx *c, const int32_t *prompt, int32_t B, int32_t 
                          int32_t *out_token, float *out_logits) {
   if (!c) return DMTD_ERR_INVALID_ARG;
   if (!prompt || B < 1 || P < 1) return fail(c, DMTD_ERR_INVALID_ARG, "prefill: null prompt or non-positive size");
+  CHECK_NOT_FAILED(c);
   if (c->prefilled) return fail(c, DMTD_ERR_STATE, "prefill: context already holds a sequence; call dmtd_reset first");
   if (B > c->max_batch || P + 1 > c->max_seq) return fail(c, DMTD_ERR_CAPACITY, "prefill: B=%d P=%d exceed max_batch=%d max_seq=%d", B, P, c->max_batch, c->max_seq);
   const int L = c->s.n_layers, lo = L - c->L_d;
@@ -826,13 +856,15 @@ dmtd_status dmtd_decode_cycle(dmtd_ctx *c, int32_t max_new, int32_t *out_tokens,
   if (!c) return DMTD_ERR_INVALID_ARG;
   if (!n_out || max_new < 0) return fail(c, DMTD_ERR_INVALID_ARG, "decode_cycle: n_out is null or max_new < 0");
   *n_out = 0;
+  CHECK_NOT_FAILED(c);
   if (!c->prefilled) return fail(c, DMTD_ERR_STATE, "decode_cycle: no prefill yet");
   const int first = c->h.n_known;
   int n = 0;
   dmtd_status rc = DMTD_OK;
   while (n < max_new) {
     if (c->h.n_known + 1 > c->max_seq) { rc = fail(c, DMTD_ERR_CAPACITY, "decode_cycle: position %d does not fit max_seq=%d", c->h.n_known, c->max_seq); break; }
-    TRY(run_greedy_pass(c));
+    rc = run_greedy_pass(c);
+    if (rc != DMTD_OK) break;                // the passes that were enqueued still count
     ++n;
     if (c->h.slot == 0) break;     // the cycle is complete
   }
@@ -847,6 +879,7 @@ dmtd_status dmtd_decode_cycle(dmtd_ctx *c, int32_t max_new, int32_t *out_tokens,
 dmtd_status dmtd_decode_forced(dmtd_ctx *c, const int32_t *forced, int32_t n, float *out_logits, int32_t *out_argmax) {
   if (!c) return DMTD_ERR_INVALID_ARG;
   if (!forced || n < 0) return fail(c, DMTD_ERR_INVALID_ARG, "decode_forced: null forced tokens or n < 0");
+  CHECK_NOT_FAILED(c);
   if (!c->prefilled) return fail(c, DMTD_ERR_STATE, "decode_forced: no prefill yet");
   if (c->h.n_known + n > c->max_seq) return fail(c, DMTD_ERR_CAPACITY, "decode_forced: %d more positions do not fit max_seq=%d", n, c->max_seq);
   if (n == 0) return DMTD_OK;
@@ -868,7 +901,8 @@ dmtd_status dmtd_step_layers(dmtd_ctx *c, int32_t l0, int32_t l1, float *hidden,
   if (!c) return DMTD_ERR_INVALID_ARG;
   if (!hidden || l0 < 0 || l1 > c->s.n_layers || l0 > l1 || B < 1 || R < 1 || pos0 < 0)
     return fail(c, DMTD_ERR_INVALID_ARG, "step_layers: bad layer range, sizes or null hidden");
-  if (B > c->max_batch || pos0 + R > c->max_seq || B * R > c->ws_rows)
+  CHECK_NOT_FAILED(c);
+  if (B > c->max_batch || R > c->max_seq || pos0 > c->max_seq - R || (long long)B * R > c->ws_rows)
     return fail(c, DMTD_ERR_CAPACITY, "step_layers: B=%d R=%d pos0=%d exceed max_batch=%d max_seq=%d rows=%d", B, R, pos0, c->max_batch, c->max_seq, c->ws_rows);
   set_int_kernel<<<1, 1, 0, c->stream>>>(&c->dstate->scratch, pos0);
   LAUNCH_OK(c, "set_int_kernel");
@@ -890,8 +924,9 @@ dmtd_status dmtd_prefill_host(dmtd_ctx *c, const int32_t *prompt_host, int32_t B
   TRY(dmtd_prefill(c, stage, B, P, nullptr, nullptr, nullptr));
   if (out_token_host)
     CUDA_TRY(c, cudaMemcpy2DAsync(out_token_host, 4, c->tokens + P, (size_t)c->max_seq * 4, 4, B, cudaMemcpyDeviceToHost, c->stream));
+  TRY(queue_error_read(c));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
-  return DMTD_OK;
+  return device_error_status(c, *c->h_error);
 }
 
 dmtd_status dmtd_decode_cycle_host(dmtd_ctx *c, int32_t max_new, int32_t *out_tokens_host, int32_t *n_out) {
@@ -903,8 +938,10 @@ dmtd_status dmtd_decode_cycle_host(dmtd_ctx *c, int32_t max_new, int32_t *out_to
   if (out_tokens_host && *n_out > 0)
     CUDA_TRY(c, cudaMemcpy2DAsync(out_tokens_host, (size_t)c->tau * 4, c->tokens + first, (size_t)c->max_seq * 4,
                                   (size_t)*n_out * 4, c->B, cudaMemcpyDeviceToHost, c->stream));
+  TRY(queue_error_read(c));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
-  return rc;
+  dmtd_status dev = device_error_status(c, *c->h_error);
+  return dev != DMTD_OK ? dev : rc;
 }
 
 dmtd_status dmtd_get_state(const dmtd_ctx *c, dmtd_state *out) {
@@ -918,8 +955,7 @@ dmtd_status dmtd_get_device_state(dmtd_ctx *c, dmtd_state *out) {
   DevState d{};
   CUDA_TRY(c, cudaMemcpyAsync(&d, c->dstate, sizeof d, cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
-  if (d.error == PK_ERR_TOKEN) return fail(c, DMTD_ERR_INVALID_ARG, "a token id outside [0, vocab) reached the embedding gather");
-  if (d.error) return fail(c, DMTD_ERR_TIMEOUT, "a device-side wait of the pass kernel gave up (%s)", d.error == PK_ERR_COPY_WAIT ? "weight copy" : "grid barrier");
+  TRY(device_error_status(c, d.error));
   out->n_known = d.n_known; out->lo_len = d.lo_len; out->up_len = d.up_len; out->cycle = d.cycle;
   out->slot = d.slot; out->n_emitted = d.n_emitted; out->tau = d.tau; out->L_d = c->L_d;
   return DMTD_OK;
@@ -952,6 +988,13 @@ dmtd_status dmtd_get_kv(dmtd_ctx *c, int32_t layer, void **k, void **v) {
   size_t kvb = c->s.kv_dtype == DMTD_BF16 ? 2 : 4;
   if (k) *k = static_cast<unsigned char *>(c->kc) + (size_t)layer * c->kv_layer_elems * kvb;
   if (v) *v = static_cast<unsigned char *>(c->vc) + (size_t)layer * c->kv_layer_elems * kvb;
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_debug_set_error_word(dmtd_ctx *c, int32_t word) {
+  if (!c || word < 0) return DMTD_ERR_INVALID_ARG;
+  CUDA_TRY(c, cudaMemcpyAsync(&c->dstate->error, &word, sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   return DMTD_OK;
 }
 
@@ -1009,7 +1052,7 @@ dmtd_status attention_check(const float *q, const void *k, const void *v, int kv
   if (D != 64 && D != 128) return fail(nullptr, DMTD_ERR_SHAPE, "attention: head_dim must be 64 or 128");
   if (nq < 1 || nkv < 1 || nq % nkv || nq / nkv > ATTN_QR)
     return fail(nullptr, DMTD_ERR_SHAPE, "attention: n_q_heads must be a multiple of n_kv_heads, at most 16 per kv head");
-  if (pos0 + R > max_seq) return fail(nullptr, DMTD_ERR_CAPACITY, "attention: pos0 + R = %d exceeds max_seq = %d", pos0 + R, max_seq);
+  if (R > max_seq || pos0 > max_seq - R) return fail(nullptr, DMTD_ERR_CAPACITY, "attention: pos0 = %d with R = %d rows exceeds max_seq = %d", pos0, R, max_seq);
   return DMTD_OK;
 }
 

@@ -85,6 +85,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
   const int S = P.stages;
   uint64_t *bars = reinterpret_cast<uint64_t *>(tg_smem + S * stage_bytes);    // full[S], empty[S], done
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * S + 1);
+  volatile int *gave_up = reinterpret_cast<volatile int *>(tmem_slot + 1);   // a wait of this block ran out: no epilogue
   const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + S), done = smem_u32(bars + 2 * S);
 
   const int sweep = blockIdx.x % P.n_sweeps, unit = blockIdx.x / P.n_sweeps;
@@ -98,6 +99,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2 * S + 1; ++s) mbar_init(smem_u32(bars + s), 1);
+    *gave_up = 0;
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -140,7 +142,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
     for (int i = 0; i < n_it && ok; ++i) {
       const int st = i % S;
       ok = tg_wait(full0 + st * 8, (i / S) & 1, P);
-      if (!ok) break;
+      if (!ok) { *gave_up = 1; __threadfence_block(); break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t a_base = smem_u32(tg_smem + st * stage_bytes), b_base = a_base + TG_WBLOCK;
 #pragma unroll
@@ -162,7 +164,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
     // ---- epilogue: thread = weight row (lane of tensor memory), registers = columns
     const int quarter = warp & 3;
     const int n = tile * TG_ROWS + quarter * 32 + lane;
-    if (tg_wait(done, 0, P)) {
+    // the accumulators are complete only if no wait of this block ran out
+    if (tg_wait(done, 0, P) && !*gave_up) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       for (int c0 = 0; c0 < P.n_cols && c0 < 2 * rows; c0 += 16) {
         uint32_t r[16];

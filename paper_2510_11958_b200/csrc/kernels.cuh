@@ -54,7 +54,7 @@ __global__ void embed_kernel(PackedMat E, const int *__restrict__ tokens, int ma
   int m = blockIdx.x, b = m / R, r = m % R;
   int tok = tokens[(size_t)b * max_seq + *pos0 + r];
   if (tok < 0 || tok >= E.N) {
-    if (threadIdx.x == 0) st->error = 1;
+    if (threadIdx.x == 0) atomicMax(&st->error, 1);
     tok = min(max(tok, 0), E.N - 1);
   }
   float *xr = x + (size_t)m * ldx;

@@ -325,10 +325,11 @@ def test_fused_pass_kernel_free_running(dmtd):
         assert (got[b, :upto] == toks[b, :upto]).all()
 
 
-@pytest.mark.parametrize("B,tau,P,n_new", [(12, 3, 23, 8), (40, 1, 9, 3), (32, 4, 9, 9)])      # 36, 40 and 128 rows per pass
+@pytest.mark.parametrize("B,tau,P,n_new", [(12, 3, 23, 8), (40, 1, 9, 3), (32, 3, 9, 9), (32, 4, 9, 9)])      # 36, 40, 96 and 128 rows per pass
 def test_tcgen05_projections_many_rows(dmtd, B, tau, P, n_new):
-    """Passes of more than 8 rows run their projections on the tcgen05 GEMM (prefill chunks of up
-    to 256 rows included): against the oracle, and against the mma.sync GEMV on the same inputs."""
+    """Passes of more than 4 rows run their projections on the tcgen05 GEMM (prefill chunks
+    included): against the oracle, and against the mma.sync GEMV on the same inputs.  96 rows is the
+    lower-layer row count of batch 32 at tau = 3 (192 accumulator columns in 256 of tensor memory)."""
     shape = SHAPES["mid"].with_(intermediate=1856)          # every K a multiple of the 64-wide k block
     w = make_weights(shape, seed=0, norm_jitter=0.1)
     prompts = make_prompts(shape.vocab, B, P, seed=1).numpy()
@@ -377,3 +378,85 @@ def test_single_layer_cell_random_hidden_and_kv(dmtd, oracle_lib, B, S):
     scale = np.abs(ref).max()
     # bf16 cache on the tensor cores: Q, P and the appended K, V rounded to bf16 (2^-9 relative)
     assert np.abs(got.double().cpu().numpy() - ref).max() <= 4e-3 * max(1.0, scale)
+
+
+def test_device_error_word_reaches_the_synchronising_calls(dmtd):
+    """Host-made failures only (no GPU wait is made to run out): a token id outside the vocabulary
+    (clamped on the device, reported as INVALID_ARG), and the error word written from the host as a
+    device-side wait that gave up would write it (reported as TIMEOUT).  The failure is sticky until
+    dmtd_reset, after which the context works as before."""
+    from paper_2510_11958_b200.binding import STATUS
+    shape = SHAPES["tiny"]
+    w = make_weights(shape, seed=0)
+    eng = _engine(dmtd, shape, to_cuda(w), 2, 3, 1, 32)
+    good = make_prompts(shape.vocab, 1, 6, seed=1)
+    bad = good.clone()
+    bad[0, 2] = shape.vocab + 7
+    with pytest.raises(dmtd.DmtdError) as e:
+        eng.prefill_host(bad)
+    assert e.value.status == STATUS["INVALID_ARG"]
+    out_host = torch.zeros(1, 3, dtype=torch.int32)
+    with pytest.raises(dmtd.DmtdError) as e:
+        eng.decode_cycle_host(3, out_host)
+    assert e.value.status == STATUS["INVALID_ARG"]
+    eng.reset()
+    first = eng.prefill_host(good)
+    assert eng.decode_cycle_host(3, out_host) == 2
+    want = out_host.clone()
+    # a wait that gave up, as the host would see it
+    for word, status in ((3, "TIMEOUT"), (2, "TIMEOUT"), (4, "TIMEOUT"), (1, "INVALID_ARG")):
+        eng.debug_set_error_word(word)
+        with pytest.raises(dmtd.DmtdError) as e:
+            eng.decode_cycle_host(3, out_host)
+        assert e.value.status == STATUS[status]
+        with pytest.raises(dmtd.DmtdError) as e:
+            eng.decode_cycle(3)
+        assert e.value.status == STATUS[status]
+        with pytest.raises(dmtd.DmtdError) as e:
+            eng.device_state()
+        assert e.value.status == STATUS[status]
+        eng.reset()
+        assert (eng.prefill_host(good) == first).all()
+        assert eng.decode_cycle_host(3, out_host) == 2
+        assert (out_host == want).all()
+        assert eng.device_state() == eng.state()
+
+
+def test_set_tau_at_a_cycle_boundary_in_mid_generation(dmtd):
+    """Section 3.7 runs a model trained with one cycle length at others: the cycle length changes
+    between cycles of one generation (3 -> 2 -> 4), teacher-forced, against the oracle doing the
+    same; both refuse a change in mid-cycle."""
+    import oracle
+    from paper_2510_11958_b200.binding import STATUS
+    shape = SHAPES["mid"]
+    w = make_weights(shape, seed=0, norm_jitter=0.1)
+    B, P = 2, 11
+    prompts = make_prompts(shape.vocab, B, P, seed=1).numpy()
+    forced = make_prompts(shape.vocab, B, 16, seed=2).numpy()
+    plan = [(3, 3), (2, 4), (4, 8)]                  # (cycle length, forced tokens run with it), whole cycles each
+    for fused in (1, 0):
+        o = oracle.Oracle(shape, w, L_d=2, tau=3, max_batch=B, max_seq=P + 20)
+        eng = _engine(dmtd, shape, to_cuda(w), 2, 3, B, P + 20, kv_dtype="f32")
+        eng.set_option("fused_pass", fused)
+        p = torch.from_numpy(prompts).cuda()
+        f = torch.from_numpy(forced).cuda()
+        _, lg = eng.prefill(p, forced_first=f[:, 0].contiguous(), want_logits=True)
+        _, rl = o.prefill(prompts, forced_first=forced[:, 0])
+        assert np.abs(lg.double().cpu().numpy() - rl).max() <= LOGIT_ATOL
+        with pytest.raises(dmtd.DmtdError) as e:
+            eng.set_tau(2)                           # slot 1: mid-cycle
+        assert e.value.status == STATUS["STATE"]
+        assert o.set_tau(2) != 0
+        at = 1
+        for i, (tau, n) in enumerate(plan):
+            if i > 0:
+                eng.set_tau(tau)
+                assert o.set_tau(tau) == 0
+            n_run = n - 1 if i == 0 else n            # the prefill was pass 1 of the first cycle
+            got, gam = eng.decode_forced(f[:, at:at + n_run].contiguous())
+            ref, ram = o.decode_forced(np.ascontiguousarray(forced[:, at:at + n_run]))
+            at += n_run
+            err, _ = check_logits(got.double().cpu().numpy(), ref, gam.cpu().numpy(), ram)
+            assert err < 1e-3
+            assert eng.state()["slot"] == 0
+            assert eng.device_state() == o.state()

@@ -67,3 +67,15 @@ def test_replica_aggregation_two_ranks(tmp_path):
                        capture_output=True, text=True, timeout=240, env=env)
     assert r.returncode == 0, r.stdout + r.stderr
     assert "OK 15.0 300.0" in r.stdout
+
+
+def test_bench_gpus_flag_starts_its_own_replicas():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks itself; the dry run
+    exercises the rendezvous, the barriers and the max/sum aggregation on gloo, without a GPU."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run-replicas"],
+                       capture_output=True, text=True, timeout=240, env=env)
+    assert r.returncode == 0, r.stdout + r.stderr
+    import json
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert lines == [{"dry_run": True, "n_gpus": 2, "ms_max": 11.0, "units": 200.0}]
