@@ -41,6 +41,8 @@ def main():
     ap.add_argument("--ghz", type=float, default=None, help="SM clock for tick -> us (default: measured in the launch itself)")
     ap.add_argument("--kv", default=None, choices=["bf16", "f32"], help="KV cache type (default: the workload's)")
     ap.add_argument("--prompt-len", type=int, default=None, help="prompt length (default: the workload's)")
+    ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
+                    help="a dmtd_set_option setting for the run, e.g. prefetch_chunks=0 (repeatable)")
     ap.add_argument("--build-only", action="store_true")
     args = ap.parse_args()
     build_timing_library()
@@ -60,6 +62,9 @@ def main():
     eng = bd.Dmtd(shape, w, L_d=wl.L_d, tau=wl.tau, max_batch=wl.batch, max_seq=wl.prompt_len + 64,
                   kv_dtype=args.kv or wl.kv_dtype)
     del w
+    for kv in args.option:
+        name, value = kv.split("=")
+        eng.set_option(name, int(value))
     eng.prefill(make_prompts(shape.vocab, wl.batch, wl.prompt_len, seed=wl.prompt_seed).cuda())
     for _ in range(4):
         eng.decode_cycle(wl.tau)                     # ends at a cycle boundary: the next pass is a full one
@@ -84,9 +89,10 @@ def main():
         d = np.diff(s[:n]) / (args.ghz * 1e3)
         per = d[: n_layers * 15].reshape(n_layers, 15)
         print(f"{label}: {(s[n - 1] - s[0]) / (args.ghz * 1e3):.1f} us from first to last stamp")
+        rest = per[1:] if n_layers > 1 else per          # the first layer of a pass starts with a cold ring
         print("  us per layer (mean over layers 1..): " +
-              " ".join(f"{nm}={per[1:, i].mean():.1f}" for i, nm in enumerate(NAMES) if nm != "-") +
-              f" | sum {per[1:].mean(0).sum():.1f}")
+              " ".join(f"{nm}={rest[:, i].mean():.1f}" for i, nm in enumerate(NAMES) if nm != "-") +
+              f" | sum {rest.mean(0).sum():.1f}")
         print("  head: prologue %.1f, projection %.1f, barrier %.1f" % tuple(d[n_layers * 15: n_layers * 15 + 3]))
         if blk == 0:
             a = s[SLOTS - 20:SLOTS - 12]

