@@ -31,6 +31,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
            "--use_fast_math" if False else "-DDMTD_NO_FAST_MATH", "-Xcompiler", "-fPIC", "-shared",
            "-I", os.path.join(ROOT, "include")]
+    cmd += os.environ.get("DMTD_NVCC_FLAGS", "").split()      # e.g. -DDMTD_PASS_SLOTS=2 for an experiment
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(HERE, "csrc", f) for f in SOURCES] + ["-o", tmp]

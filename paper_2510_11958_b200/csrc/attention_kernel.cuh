@@ -260,7 +260,8 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
 // fp32 accuracy, and they issue too slowly): the tile arithmetic of the pass kernel's fp32
 // attention stage, one 64-key tile in shared memory per block and two blocks per SM, so that one
 // block's copies run under the other's arithmetic.
-constexpr int ATTN_F32_SMEM = PK_F_NEW;           // K and V tile, Q, partial scores, running max / sum / rescale factor
+using StepF32Map = AttnF32Map<64>;
+constexpr int ATTN_F32_SMEM = StepF32Map::NEW;           // K and V tile, Q, partial scores, running max / sum / rescale factor
 
 __global__ void __launch_bounds__(PK_THREADS, 2)
 attn_f32_kernel(const float *__restrict__ qkv, int ldq, const float *__restrict__ kc, const float *__restrict__ vc, int max_seq,
@@ -285,11 +286,11 @@ attn_f32_kernel(const float *__restrict__ qkv, int ldq, const float *__restrict_
   const float scale = rsqrtf((float)PK_D);
   for (int qi = warp; qi < nQ; qi += PK_WARPS) {
     const float *src = qkv + (size_t)(b * R + r0 + qi / G) * ldq + (size_t)(kvh * G + qi % G) * PK_D;
-    float *dst = reinterpret_cast<float *>(sc + PK_F_Q) + qi * PK_D;
+    float *dst = reinterpret_cast<float *>(sc + StepF32Map::Q) + qi * PK_D;
 #pragma unroll
     for (int j = 0; j < 4; ++j) dst[lane + 32 * j] = src[lane + 32 * j] * scale;
   }
-  float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR;
+  float *const m_run = reinterpret_cast<float *>(sc + StepF32Map::STAT), *const l_run = m_run + PK_QR;
   if ((int)threadIdx.x < PK_QR) { m_run[threadIdx.x] = -INFINITY; l_run[threadIdx.x] = 0.f; }
   const float *kb = kc + (((size_t)b * nkv + kvh) * max_seq + j0) * PK_D;
   const float *vb = vc + (((size_t)b * nkv + kvh) * max_seq + j0) * PK_D;
@@ -309,26 +310,26 @@ attn_f32_kernel(const float *__restrict__ qkv, int ldq, const float *__restrict_
     }
     asm volatile("cp.async.commit_group;" ::: "memory");      // an empty group past the last tile keeps the counts uniform
   };
-  fetch(kb, 0, PK_F_K, PK_F_KROW);
-  fetch(vb, 0, PK_F_V, PK_D * 4);
+  fetch(kb, 0, StepF32Map::K, PK_F_KROW);
+  fetch(vb, 0, StepF32Map::V, PK_D * 4);
 #pragma unroll 1
   for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
     const int n_t = min(PK_TK, n_keys - tile0);
     asm volatile("cp.async.wait_group 1;" ::: "memory");      // K of this tile (V may still be on its way)
     __syncthreads();                                      // ... from every thread; the first time also Q and the statistics
-    attn_f32_scores(sc, nQ, n_t);
+    attn_f32_scores<StepF32Map>(sc, nQ, n_t);
     __syncthreads();                                      // K consumed
-    fetch(kb, tile0 + PK_TK, PK_F_K, PK_F_KROW);
+    fetch(kb, tile0 + PK_TK, StepF32Map::K, PK_F_KROW);
     // every key comes from the cache: key index i sits at position j0 + i
-    attn_f32_softmax(sc, nQ, G, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0);
+    attn_f32_softmax<StepF32Map>(sc, nQ, G, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0);
     asm volatile("cp.async.wait_group 1;" ::: "memory");      // V of this tile (the next K may still be on its way)
     __syncthreads();                                      // probabilities and V from every thread
-    attn_f32_pv(sc, acc, nQ, n_t);
+    attn_f32_pv<StepF32Map>(sc, acc, nQ, n_t);
     __syncthreads();                                      // V and the probabilities consumed
-    fetch(vb, tile0 + PK_TK, PK_F_V, PK_D * 4);
+    fetch(vb, tile0 + PK_TK, StepF32Map::V, PK_D * 4);
   }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
-  attn_f32_combine(sc, acc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
+  attn_f32_combine<StepF32Map>(sc, acc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
 }
 
 }  // namespace dmtd

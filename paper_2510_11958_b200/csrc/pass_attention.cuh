@@ -44,7 +44,19 @@ constexpr int PK_AT_ROWS = PK_AT_RED + 2 * PK_WARPS * PK_QR * 4;   // the pass's
 constexpr int PK_AT_ROW_FLOATS = (PK_MAX_GROUP + 2) * PK_D;
 constexpr int PK_AT_END = PK_AT_ROWS + PK_MAX_ROWS * PK_AT_ROW_FLOATS * 4;
 static_assert(PK_AT_TILES_END <= PK_AT_RED && PK_WARPS * PK_QR * PK_OROW * 4 <= PK_AT_RED, "attention scratch overlaps");
-static_assert(PK_AT_END <= PK_BSTAGE_BYTES + PK_XS_BYTES, "attention scratch does not fit");
+// The pass kernel keeps one tile of each kind, so its map of the same pieces is more compact (its
+// scratch is what the weight rings leave of the SM's shared memory):
+constexpr int PK_PA_KH = 0;                                   // K tile [PK_TK][PK_KROW]
+constexpr int PK_PA_VH = PK_PA_KH + PK_TK * PK_KROW;          // V tile [PK_TK][PK_VROW]
+constexpr int PK_PA_QH = PK_PA_VH + PK_TK * PK_VROW;          // Q tile [PK_QR][PK_QROW], and a second one kept zero
+constexpr int PK_PA_NEW = PK_PA_QH + 2 * PK_QR * PK_QROW;     // K rows of the pass [4][128] floats, then V rows [4][128]
+constexpr int PK_PA_TILES_END = PK_PA_NEW + 2 * PK_MAX_ROWS * PK_D * 4;
+constexpr int PK_PA_OS = 0;                                   // after the tiles are consumed: [warps][16][PK_OROW] floats
+constexpr int PK_PA_RED = PK_WARPS * PK_QR * PK_OROW * 4;     // running max [warps][16], then sum / merge factor [warps][16]
+constexpr int PK_PA_ROWS = PK_PA_RED + 2 * PK_WARPS * PK_QR * 4;   // the pass's q | k | v vectors of one kv head, fp32, per row
+constexpr int PK_PA_END = PK_PA_ROWS + PK_MAX_ROWS * PK_AT_ROW_FLOATS * 4;
+static_assert(PK_PA_TILES_END <= PK_PA_RED, "attention scratch overlaps");
+static_assert(PK_PA_END <= PK_SCRATCH_BYTES, "attention scratch does not fit");
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -80,7 +92,7 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
                                               int R, int pos0, bool write_cache) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = P.nq / P.nkv, nQ = R * G;
-  const float *rows = reinterpret_cast<const float *>(sc + PK_AT_ROWS);
+  const float *rows = reinterpret_cast<const float *>(sc + PK_PA_ROWS);
   const float scale = rsqrtf((float)PK_D);
 #pragma unroll 1
   for (int task = warp; task < nQ + 2 * R; task += PK_WARPS) {
@@ -113,14 +125,14 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
       }
     }
     if (kind == 0) {
-      __nv_bfloat16 *qh = reinterpret_cast<__nv_bfloat16 *>(sc + PK_AT_QH + task * PK_QROW);
+      __nv_bfloat16 *qh = reinterpret_cast<__nv_bfloat16 *>(sc + PK_PA_QH + task * PK_QROW);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const __nv_bfloat16 h = __float2bfloat16_rn(v[j]);
         qh[lane + 32 * j] = h;
       }
     } else {
-      float *row = reinterpret_cast<float *>(sc + PK_AT_NEW) + ((kind == 2 ? PK_MAX_ROWS : 0) + r) * PK_D;
+      float *row = reinterpret_cast<float *>(sc + PK_PA_NEW) + ((kind == 2 ? PK_MAX_ROWS : 0) + r) * PK_D;
       const size_t at = (((size_t)b * P.nkv + kvh) * P.max_seq + pos) * PK_D;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -147,13 +159,13 @@ struct AttnAcc {
 // read from shared memory in a rolled loop: the code stays short (instruction fetch, not
 // arithmetic, bounds a stage that runs once per layer).
 __device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc, int n_t, int tile0, int n_cached, int j0,
-                                                  int pos_new, int row_pos0, int G, int k_off = PK_AT_KH,
-                                                  int v_off = PK_AT_VH) {
+                                                  int pos_new, int row_pos0, int G, int k_off = PK_PA_KH,
+                                                  int v_off = PK_PA_VH) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int kg = warp & 3, dh = warp >> 2;
   const uint32_t kh_tile = smem_u32(sc + k_off);
   const uint32_t vh_tile = smem_u32(sc + v_off);
-  const uint32_t qh_tile = smem_u32(sc + PK_AT_QH);
+  const uint32_t qh_tile = smem_u32(sc + PK_PA_QH);
   float (&m_run)[2] = A.m_run;
   float (&l_part)[2] = A.l_part;
   float (&o)[8][4] = A.o;
@@ -235,8 +247,8 @@ __device__ __forceinline__ void attn_combine_store(AttnAcc &A, unsigned char *sc
                                                    int slot_stride, int split, float *part_o, float *part_ml) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int kg = warp & 3, dh = warp >> 2;
-  float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
-  float *const red_m = reinterpret_cast<float *>(sc + PK_AT_RED);
+  float *const o_s = reinterpret_cast<float *>(sc + PK_PA_OS);
+  float *const red_m = reinterpret_cast<float *>(sc + PK_PA_RED);
   float *const red_l = red_m + PK_WARPS * PK_QR;
   float (&m_run)[2] = A.m_run;
   float (&l_part)[2] = A.l_part;
@@ -304,9 +316,9 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
   if ((int)blockIdx.x >= items) return;
 
   unsigned char *const sc = S.bstage;
-  const uint32_t kh_tile = smem_u32(sc + PK_AT_KH);
-  const uint32_t vh_tile = smem_u32(sc + PK_AT_VH);
-  const uint32_t qh_tile = smem_u32(sc + PK_AT_QH);
+  const uint32_t kh_tile = smem_u32(sc + PK_PA_KH);
+  const uint32_t vh_tile = smem_u32(sc + PK_PA_VH);
+  const uint32_t qh_tile = smem_u32(sc + PK_PA_QH);
   // a 16-byte part (8 values) of a tile row: parts 0..15 are K, 16..31 are V
   auto put_part = [&](int row, int part, const float (&f)[8]) {
     const uint4 hi = pack8(f);
@@ -345,7 +357,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
 #pragma unroll 1
       for (int r = 0; r < R; ++r) {
         const float *src = P.qkv + (size_t)(b * R + r) * ldq;
-        float *dst = reinterpret_cast<float *>(sc + PK_AT_ROWS) + r * PK_AT_ROW_FLOATS;
+        float *dst = reinterpret_cast<float *>(sc + PK_PA_ROWS) + r * PK_AT_ROW_FLOATS;
         stage_copy(S, dst, src + kvh * G * PK_D, (uint32_t)(G * PK_D * 4));
         stage_copy(S, dst + G * PK_D, src + (P.nq + kvh) * PK_D, PK_D * 4);
         stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
@@ -376,7 +388,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
 #pragma unroll 1
       for (int c = threadIdx.x + max(0, n_cached - tile0) * 32; c < n_t * 32; c += PK_THREADS) {
         const int row = c >> 5, part = c & 31, r = tile0 + row - n_cached;
-        const float *src = reinterpret_cast<const float *>(sc + PK_AT_NEW) + ((part < 16 ? 0 : PK_MAX_ROWS) + r) * PK_D + (part & 15) * 8;
+        const float *src = reinterpret_cast<const float *>(sc + PK_PA_NEW) + ((part < 16 ? 0 : PK_MAX_ROWS) + r) * PK_D + (part & 15) * 8;
         const float f[8] = {src[0], src[1], src[2], src[3], src[4], src[5], src[6], src[7]};
         put_part(row, part, f);
       }

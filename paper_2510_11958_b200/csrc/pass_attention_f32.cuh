@@ -14,17 +14,28 @@ namespace dmtd {
 
 constexpr int PK_F_KROW = 528;                                   // bytes per K row: 512 + 16, conflict-free 16-byte reads by 8 lanes on 8 rows
 constexpr int PK_F_PARTS = 4;                                    // a score is the sum of 4 partial dot products over 32 dimensions each
-constexpr int PK_F_K = 0;                                        // K tile [PK_TK][PK_F_KROW]
-constexpr int PK_F_V = PK_F_K + PK_TK * PK_F_KROW;               // V tile [PK_TK][128] floats
-constexpr int PK_F_Q = PK_F_V + PK_TK * PK_D * 4;                // Q [PK_QR][128] floats, scaled by 1/sqrt(d)
-constexpr int PK_F_S = PK_F_Q + PK_QR * PK_D * 4;                // partial scores [part][PK_TK][PK_QR]; part 0's area then holds the probabilities
-constexpr int PK_F_STAT = PK_F_S + PK_F_PARTS * PK_TK * PK_QR * 4;   // running max, running sum, rescale factor [3][PK_QR]
-constexpr int PK_F_NEW = PK_F_STAT + 3 * PK_QR * 4;              // K rows of the pass [4][128], then V rows [4][128]
-constexpr int PK_F_W = PK_F_NEW + 2 * PK_MAX_ROWS * PK_D * 4;    // q-norm weights, k-norm weights (floats), rotary frequencies (doubles)
-constexpr int PK_F_ROWS = PK_F_W + 2 * PK_D * 4 + (PK_D / 2) * 8;    // the pass's q | k | v vectors of one kv head, fp32, per row
-constexpr int PK_F_END = PK_F_ROWS + PK_MAX_ROWS * PK_AT_ROW_FLOATS * 4;
-static_assert(PK_F_END <= PK_BSTAGE_BYTES + PK_XS_BYTES, "fp32 attention scratch does not fit");
-static_assert(PK_WARPS * PK_QR * PK_OROW * 4 <= PK_F_S, "partial-output overlay (over K, V and Q, all consumed by then) reaches the scores");
+
+// Map of the fp32 attention scratch for tiles of TK keys (at most 64: the score step maps a key to
+// a lane of one of two warps).  The per-step kernel uses 64-key tiles; the pass kernel, whose
+// scratch is what the weight rings leave of the SM's shared memory, 48-key tiles.
+template <int TK>
+struct AttnF32Map {
+  static_assert(TK % 8 == 0 && TK <= 64, "tile size");
+  static constexpr int TKEYS = TK;
+  static constexpr int K = 0;                                    // K tile [TK][PK_F_KROW]
+  static constexpr int V = K + TK * PK_F_KROW;                   // V tile [TK][128] floats
+  static constexpr int Q = V + TK * PK_D * 4;                    // Q [PK_QR][128] floats, scaled by 1/sqrt(d)
+  static constexpr int S = Q + PK_QR * PK_D * 4;                 // partial scores [part][TK][PK_QR]; part 0's area then holds the probabilities
+  static constexpr int STAT = S + PK_F_PARTS * TK * PK_QR * 4;   // running max, running sum, rescale factor [3][PK_QR]
+  static constexpr int NEW = STAT + 3 * PK_QR * 4;               // K rows of the pass [4][128], then V rows [4][128]
+  static constexpr int W = NEW + 2 * PK_MAX_ROWS * PK_D * 4;     // q-norm weights, k-norm weights (floats), rotary frequencies (doubles)
+  static constexpr int ROWS = W + 2 * PK_D * 4 + (PK_D / 2) * 8; // the pass's q | k | v vectors of one kv head, fp32, per row
+  static constexpr int END = ROWS + PK_MAX_ROWS * PK_AT_ROW_FLOATS * 4;
+  // the partial-output overlay of the combine step lies over K, V, Q and the scores (all consumed by then)
+  static_assert(PK_WARPS * PK_QR * PK_OROW * 4 <= STAT, "partial-output overlay reaches the running statistics");
+};
+using PassF32Map = AttnF32Map<48>;
+static_assert(PassF32Map::END <= PK_SCRATCH_BYTES, "fp32 attention scratch does not fit");
 
 // QK-norm (Section 3.1's Qwen3 block) and the half-split rotary embedding of one head vector,
 // one value per lane and quarter: v[j] is element lane + 32 j.
@@ -49,13 +60,14 @@ __device__ __forceinline__ void head_norm_rope(const float *w, const double *inv
 }
 
 // Step a3 for one (sequence, kv head): one warp per head vector of the pass's rows.
+template <class L>
 __device__ __forceinline__ void attn_new_rows_f32(const PassParams &P, const PassLayer &Ly, unsigned char *sc, int b, int kvh,
                                                   int R, int pos0, bool write_cache) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = P.nq / P.nkv, nQ = R * G;
-  const float *rows = reinterpret_cast<const float *>(sc + PK_F_ROWS);
-  const float *w_q = reinterpret_cast<const float *>(sc + PK_F_W), *w_k = w_q + PK_D;
-  const double *inv_freq = reinterpret_cast<const double *>(sc + PK_F_W + 2 * PK_D * 4);
+  const float *rows = reinterpret_cast<const float *>(sc + L::ROWS);
+  const float *w_q = reinterpret_cast<const float *>(sc + L::W), *w_k = w_q + PK_D;
+  const double *inv_freq = reinterpret_cast<const double *>(sc + L::W + 2 * PK_D * 4);
   const float scale = rsqrtf((float)PK_D);
 #pragma unroll 1
   for (int task = warp; task < nQ + 2 * R; task += PK_WARPS) {
@@ -69,8 +81,8 @@ __device__ __forceinline__ void attn_new_rows_f32(const PassParams &P, const Pas
     for (int j = 0; j < 4; ++j) v[j] = src[lane + 32 * j];
     if (kind != 2) head_norm_rope(kind == 0 ? w_q : w_k, inv_freq, P.eps, kind == 0 ? scale : 1.f, pos0 + r, lane, v);
     float *dst;
-    if (kind == 0) dst = reinterpret_cast<float *>(sc + PK_F_Q) + task * PK_D;
-    else dst = reinterpret_cast<float *>(sc + PK_F_NEW) + ((kind == 2 ? PK_MAX_ROWS : 0) + r) * PK_D;
+    if (kind == 0) dst = reinterpret_cast<float *>(sc + L::Q) + task * PK_D;
+    else dst = reinterpret_cast<float *>(sc + L::NEW) + ((kind == 2 ? PK_MAX_ROWS : 0) + r) * PK_D;
 #pragma unroll
     for (int j = 0; j < 4; ++j) dst[lane + 32 * j] = v[j];
     if (kind != 0 && write_cache) {
@@ -88,9 +100,10 @@ __device__ __forceinline__ float4 lds_f4(const unsigned char *p) { return *reint
 // (reads K and Q), the softmax step (scores to probabilities, running max and sum), O += P V
 // (reads V).  Key index i of the slice sits at position (i < n_cached ? j0 + i : pos_new + i -
 // n_cached); query row q may see positions up to row_pos0 + q / G.
+template <class L>
 __device__ __forceinline__ void attn_f32_scores(unsigned char *sc, int nQ, int n_t) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  float *const sm_s = reinterpret_cast<float *>(sc + PK_F_S);
+  float *const sm_s = reinterpret_cast<float *>(sc + L::S);
   {
     // partial scores: warp = (part, half of the tile's keys), lane = key.  Part p is dimensions
     // 32 p .. 32 p + 31; the lanes of a warp read the same Q values (one broadcast each) and
@@ -100,12 +113,12 @@ __device__ __forceinline__ void attn_f32_scores(unsigned char *sc, int nQ, int n
     if (key < n_t) {
       float4 kr[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) kr[j] = lds_f4(sc + PK_F_K + key * PK_F_KROW + (part * 8 + j) * 16);
+      for (int j = 0; j < 8; ++j) kr[j] = lds_f4(sc + L::K + key * PK_F_KROW + (part * 8 + j) * 16);
       // four query rows at a time: four independent chains of FMAs (rows beyond nQ hold whatever
       // the scratch held; nobody reads their sums)
 #pragma unroll 1
       for (int q0 = 0; q0 < nQ; q0 += 4) {
-        const unsigned char *qp = sc + PK_F_Q + q0 * PK_D * 4 + part * 128;
+        const unsigned char *qp = sc + L::Q + q0 * PK_D * 4 + part * 128;
         float s[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -115,17 +128,18 @@ __device__ __forceinline__ void attn_f32_scores(unsigned char *sc, int nQ, int n
             s[e] += kr[j].x * qv.x + kr[j].y * qv.y + kr[j].z * qv.z + kr[j].w * qv.w;
           }
         }
-        *reinterpret_cast<float4 *>(sm_s + (part * PK_TK + key) * PK_QR + q0) = make_float4(s[0], s[1], s[2], s[3]);
+        *reinterpret_cast<float4 *>(sm_s + (part * L::TKEYS + key) * PK_QR + q0) = make_float4(s[0], s[1], s[2], s[3]);
       }
     }
   }
 }
 
+template <class L>
 __device__ __forceinline__ void attn_f32_softmax(unsigned char *sc, int nQ, int G, int n_t, int tile0, int n_cached, int j0,
                                                  int pos_new, int row_pos0) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  float *const sm_s = reinterpret_cast<float *>(sc + PK_F_S);
-  float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR, *const corr = l_run + PK_QR;
+  float *const sm_s = reinterpret_cast<float *>(sc + L::S);
+  float *const m_run = reinterpret_cast<float *>(sc + L::STAT), *const l_run = m_run + PK_QR, *const corr = l_run + PK_QR;
       // per query row: the tile's max joins the running max; scores become probabilities
 #pragma unroll 2
       for (int q = warp; q < nQ; q += PK_WARPS) {
@@ -138,7 +152,7 @@ __device__ __forceinline__ void attn_f32_softmax(unsigned char *sc, int nQ, int 
           if (key < n_t && key_pos <= row_pos0 + q / G) {
             v[h] = 0.f;
 #pragma unroll
-            for (int p = 0; p < PK_F_PARTS; ++p) v[h] += sm_s[(p * PK_TK + key) * PK_QR + q];
+            for (int p = 0; p < PK_F_PARTS; ++p) v[h] += sm_s[(p * L::TKEYS + key) * PK_QR + q];
           }
         }
         const float v0 = v[0], v1 = v[1];
@@ -147,7 +161,7 @@ __device__ __forceinline__ void attn_f32_softmax(unsigned char *sc, int nQ, int 
         const float p0 = v0 > -INFINITY ? __expf(v0 - m_new) : 0.f;
         const float p1 = v1 > -INFINITY ? __expf(v1 - m_new) : 0.f;
         sm_s[lane * PK_QR + q] = p0;
-        sm_s[(lane + 32) * PK_QR + q] = p1;
+        if (lane + 32 < L::TKEYS) sm_s[(lane + 32) * PK_QR + q] = p1;
         const float ps = warp_sum(p0 + p1);
         if (lane == 0) {
           const float f = m_old > -INFINITY ? __expf(m_old - m_new) : 0.f;
@@ -158,9 +172,10 @@ __device__ __forceinline__ void attn_f32_softmax(unsigned char *sc, int nQ, int 
       }
 }
 
+template <class L>
 __device__ __forceinline__ void attn_f32_pv(unsigned char *sc, float (&acc)[PK_QR][4], int nQ, int n_t) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const float *const corr = reinterpret_cast<const float *>(sc + PK_F_STAT) + 2 * PK_QR;
+  const float *const corr = reinterpret_cast<const float *>(sc + L::STAT) + 2 * PK_QR;
       // O += P V: warp = key group (keys warp, warp + 8, ..), lane = 4 output dimensions
 #pragma unroll
       for (int q = 0; q < PK_QR; ++q) {
@@ -171,11 +186,11 @@ __device__ __forceinline__ void attn_f32_pv(unsigned char *sc, float (&acc)[PK_Q
       }
 #pragma unroll 2
       for (int key = warp; key < n_t; key += PK_WARPS) {
-        const float4 vv = lds_f4(sc + PK_F_V + (key * PK_D + lane * 4) * 4);
+        const float4 vv = lds_f4(sc + L::V + (key * PK_D + lane * 4) * 4);
 #pragma unroll
         for (int q4 = 0; q4 < PK_QR / 4; ++q4) {
           if (q4 * 4 < nQ) {
-            const float4 pv = lds_f4(sc + PK_F_S + (key * PK_QR + q4 * 4) * 4);
+            const float4 pv = lds_f4(sc + L::S + (key * PK_QR + q4 * 4) * 4);
             const float pq[4] = {pv.x, pv.y, pv.z, pv.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -189,22 +204,24 @@ __device__ __forceinline__ void attn_f32_pv(unsigned char *sc, float (&acc)[PK_Q
 
 // The three steps on a tile that is complete in shared memory; the caller syncs before the tile's
 // space is written again.
+template <class L>
 __device__ __forceinline__ void attn_f32_tile(unsigned char *sc, float (&acc)[PK_QR][4], int nQ, int G, int n_t, int tile0,
                                               int n_cached, int j0, int pos_new, int row_pos0) {
-  attn_f32_scores(sc, nQ, n_t);
+  attn_f32_scores<L>(sc, nQ, n_t);
   pk_sync();
-  attn_f32_softmax(sc, nQ, G, n_t, tile0, n_cached, j0, pos_new, row_pos0);
+  attn_f32_softmax<L>(sc, nQ, G, n_t, tile0, n_cached, j0, pos_new, row_pos0);
   pk_sync();
-  attn_f32_pv(sc, acc, nQ, n_t);
+  attn_f32_pv<L>(sc, acc, nQ, n_t);
 }
 
 // The slice's partial result: the key groups' outputs summed, with the running max and sum, at
 // slot (row0 + q / G, head0 + q % G, split), where a (row, head) owns `slot_stride` slots.
+template <class L>
 __device__ __forceinline__ void attn_f32_combine(unsigned char *sc, float (&acc)[PK_QR][4], int nQ, int G, int row0, int head0,
                                                  int nq, int slot_stride, int split, float *part_o, float *part_ml) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const float *const m_run = reinterpret_cast<const float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR;
-    float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
+  const float *const m_run = reinterpret_cast<const float *>(sc + L::STAT), *const l_run = m_run + PK_QR;
+    float *const o_s = reinterpret_cast<float *>(sc + PK_PA_OS);
     pk_sync();                                            // tiles consumed: their space becomes o_s
 #pragma unroll
     for (int q = 0; q < PK_QR; ++q)
@@ -240,7 +257,7 @@ __device__ __noinline__ void attention_stage_f32(const PassParams &P, const Pass
   const int items = P.B * P.nkv * nsplit;
   if ((int)blockIdx.x >= items) return;
   unsigned char *const sc = S.bstage;
-  float *const m_run = reinterpret_cast<float *>(sc + PK_F_STAT), *const l_run = m_run + PK_QR;
+  float *const m_run = reinterpret_cast<float *>(sc + PassF32Map::STAT), *const l_run = m_run + PK_QR;
 
 #pragma unroll 1
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
@@ -263,26 +280,26 @@ __device__ __noinline__ void attention_stage_f32(const PassParams &P, const Pass
       if (c < 3 * R) {
         const int r = c / 3, what = c - 3 * r;              // 0: the G query heads, 1: k, 2: v
         const float *src = P.qkv + (size_t)(b * R + r) * ldq;
-        float *dst = reinterpret_cast<float *>(sc + PK_F_ROWS) + r * PK_AT_ROW_FLOATS;
+        float *dst = reinterpret_cast<float *>(sc + PassF32Map::ROWS) + r * PK_AT_ROW_FLOATS;
         if (what == 0) stage_copy(S, dst, src + kvh * G * PK_D, (uint32_t)(G * PK_D * 4));
         else if (what == 1) stage_copy(S, dst + G * PK_D, src + (P.nq + kvh) * PK_D, PK_D * 4);
         else stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
       } else if (c == 3 * R) {
-        stage_copy(S, sc + PK_F_W, Ly.w_qn, PK_D * 4);
+        stage_copy(S, sc + PassF32Map::W, Ly.w_qn, PK_D * 4);
       } else if (c == 3 * R + 1) {
-        stage_copy(S, sc + PK_F_W + PK_D * 4, Ly.w_kn, PK_D * 4);
+        stage_copy(S, sc + PassF32Map::W + PK_D * 4, Ly.w_kn, PK_D * 4);
       } else if (c == 3 * R + 2) {
-        stage_copy(S, sc + PK_F_W + 2 * PK_D * 4, P.inv_freq, (PK_D / 2) * 8);
+        stage_copy(S, sc + PassF32Map::W + 2 * PK_D * 4, P.inv_freq, (PK_D / 2) * 8);
       }
     }
     PK_SUBSTAMP(1);
     // cached rows of a tile: asynchronous 16-byte copies, 32 of K and 32 of V per row
     auto fetch_cached = [&](int tile0) {
-      const int n_c = min(PK_TK, n_cached - tile0);
+      const int n_c = min(PassF32Map::TKEYS, n_cached - tile0);
 #pragma unroll 1
       for (int c = threadIdx.x; c < n_c * 64; c += PK_THREADS) {
         const int row = c >> 6, u = c & 63;
-        const uint32_t dst = smem_u32(sc) + (u < 32 ? PK_F_K + row * PK_F_KROW + u * 16 : PK_F_V + row * PK_D * 4 + (u - 32) * 16);
+        const uint32_t dst = smem_u32(sc) + (u < 32 ? PassF32Map::K + row * PK_F_KROW + u * 16 : PassF32Map::V + row * PK_D * 4 + (u - 32) * 16);
         cp_async16(dst, (u < 32 ? kc : vc) + (size_t)(tile0 + row) * PK_D + (u & 31) * 4);
       }
     };
@@ -291,15 +308,15 @@ __device__ __noinline__ void attention_stage_f32(const PassParams &P, const Pass
     if ((int)threadIdx.x < PK_QR) { m_run[threadIdx.x] = -INFINITY; l_run[threadIdx.x] = 0.f; }
     stage_wait(P, S);
     PK_SUBSTAMP(3);
-    attn_new_rows_f32(P, Ly, sc, b, kvh, R, pos0, split == 0);
+    attn_new_rows_f32<PassF32Map>(P, Ly, sc, b, kvh, R, pos0, split == 0);
     PK_SUBSTAMP(4);
 
     float acc[PK_QR][4];
 #pragma unroll
     for (int q = 0; q < PK_QR; ++q) acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f;
 #pragma unroll 1
-    for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK) {
-      const int n_t = min(PK_TK, n_keys - tile0);
+    for (int tile0 = 0; tile0 < n_keys; tile0 += PassF32Map::TKEYS) {
+      const int n_t = min(PassF32Map::TKEYS, n_keys - tile0);
       pk_sync();                                          // new rows written / previous tile consumed
       PK_SUBSTAMP(8);
       if (tile0 > 0) fetch_cached(tile0);
@@ -307,17 +324,17 @@ __device__ __noinline__ void attention_stage_f32(const PassParams &P, const Pass
 #pragma unroll 1
       for (int c = threadIdx.x + max(0, n_cached - tile0) * 64; c < n_t * 64; c += PK_THREADS) {
         const int row = c >> 6, u = c & 63, r = tile0 + row - n_cached;
-        const float4 val = lds_f4(sc + PK_F_NEW + (((u < 32 ? 0 : PK_MAX_ROWS) + r) * PK_D + (u & 31) * 4) * 4);
-        *reinterpret_cast<float4 *>(sc + (u < 32 ? PK_F_K + row * PK_F_KROW + u * 16 : PK_F_V + row * PK_D * 4 + (u - 32) * 16)) = val;
+        const float4 val = lds_f4(sc + PassF32Map::NEW + (((u < 32 ? 0 : PK_MAX_ROWS) + r) * PK_D + (u & 31) * 4) * 4);
+        *reinterpret_cast<float4 *>(sc + (u < 32 ? PassF32Map::K + row * PK_F_KROW + u * 16 : PassF32Map::V + row * PK_D * 4 + (u - 32) * 16)) = val;
       }
       PK_SUBSTAMP(9);
       cp_async_wait_all();
       pk_sync();
       PK_SUBSTAMP(10);
-      attn_f32_tile(sc, acc, nQ, G, n_t, tile0, n_cached, j0, pos0, pos0);
+      attn_f32_tile<PassF32Map>(sc, acc, nQ, G, n_t, tile0, n_cached, j0, pos0, pos0);
     }
     PK_SUBSTAMP(5);
-    attn_f32_combine(sc, acc, nQ, G, b * R, kvh * G, P.nq, PK_NSPLIT_CAP, split, P.part_o, P.part_ml);
+    attn_f32_combine<PassF32Map>(sc, acc, nQ, G, b * R, kvh * G, P.nq, PK_NSPLIT_CAP, split, P.part_o, P.part_ml);
     PK_SUBSTAMP(6);
   }
   pk_sync();

@@ -37,28 +37,40 @@
 
 namespace dmtd {
 
-constexpr int PK_WARPS = 8;
-constexpr int PK_THREADS = PK_WARPS * 32;
-constexpr int PK_CHUNK_ATOMS = 4;                          // atoms (1 KiB each) per bulk copy
-constexpr int PK_CHUNK_BYTES = PK_CHUNK_ATOMS * 1024;
+// Ring geometry (overridable at build time for sweeps).  Measured on the Qwen3-4B shape, batch 1,
+// us per layer of a full pass: chunks of 4 / 5 / 6 / 7 / 8 atoms in 2 slots 66.9 / 64.9 / 63.6 /
+// 63.5 / 64.8; 3 slots of 5 atoms 64.6, 4 slots of 4 atoms 64.7.  Two things pull one way: the copy
+// engine of an SM spends ~100 cycles per bulk copy whatever its size (a plain stream of 4 KiB copies
+// tops out at 60 GB/s per SM, of 8 KiB copies at 100 GB/s; the SM's share of HBM is 44 GB/s), and
+// what the rings hold is what HBM delivers while the stage threads sit in a barrier.  The other
+// way: every other load of the SM waits behind the copies in flight.
+#ifndef DMTD_PASS_CHUNK
+#define DMTD_PASS_CHUNK 7
+#endif
 #ifndef DMTD_PASS_SLOTS
 #define DMTD_PASS_SLOTS 2
 #endif
+constexpr int PK_WARPS = 8;
+constexpr int PK_THREADS = PK_WARPS * 32;
+constexpr int PK_CHUNK_ATOMS = DMTD_PASS_CHUNK;            // atoms (1 KiB each) per bulk copy
+constexpr int PK_CHUNK_BYTES = PK_CHUNK_ATOMS * 1024;
+
 constexpr int PK_SLOTS = DMTD_PASS_SLOTS;                  // ring slots per warp
 constexpr int PK_MAX_ROWS = 4;                             // activation rows (B*R) per stage
-constexpr int PK_MAX_KS = 1280;                            // largest k-slab of a packed matrix
+constexpr int PK_MAX_KS = 256;                             // largest k-slab of a packed matrix the kernel streams
 constexpr int PK_MAX_LAYERS = 40;
 constexpr int PK_NSPLIT_CAP = 16;                          // key slices per (sequence, kv head)
 constexpr int PK_D = 128;                                  // head_dim
 constexpr int PK_QR = 16;                                  // query rows per attention item
-constexpr int PK_MAX_GROUP = 8;                            // query heads per kv head
-constexpr int PK_XS_FLOATS = 20480;                        // activation staging area, floats
+constexpr int PK_MAX_GROUP = 4;                            // query heads per kv head
 
 // shared memory map (bytes)
-constexpr int PK_RING_BYTES = PK_WARPS * PK_SLOTS * PK_CHUNK_BYTES;           // 65536
-constexpr int PK_BROW_MAX = PK_MAX_KS * 2 + 64;                               // 2624
-constexpr int PK_BSTAGE_BYTES = 2 * 8 * PK_BROW_MAX;                          // 41984: two slabs of 8 columns
-constexpr int PK_XS_BYTES = PK_XS_FLOATS * 4;                                 // 81920
+constexpr int PK_RING_BYTES = PK_WARPS * PK_SLOTS * PK_CHUNK_BYTES;           // 114688
+constexpr int PK_BROW_MAX = PK_MAX_KS * 2 + 64;                               // 576
+constexpr int PK_BSTAGE_BYTES = 2 * 8 * PK_BROW_MAX;                          // 9216: two slabs of 8 columns
+constexpr int PK_SCRATCH_BYTES = 88576;                                       // bstage + xs; the attention stages lay their own map over both
+constexpr int PK_XS_BYTES = PK_SCRATCH_BYTES - PK_BSTAGE_BYTES;
+constexpr int PK_XS_FLOATS = PK_XS_BYTES / 4;                                 // 19840: staged activation rows
 constexpr int PK_OFF_RING = 0;
 constexpr int PK_OFF_BSTAGE = PK_OFF_RING + PK_RING_BYTES;
 constexpr int PK_OFF_XS = PK_OFF_BSTAGE + PK_BSTAGE_BYTES;                    // directly behind bstage
@@ -100,10 +112,7 @@ struct PassParams {
 };
 
 constexpr int PK_SMEM_BYTES = PK_OFF_LAYERS + PK_MAX_LAYERS * (int)sizeof(PassLayer);
-// 196 KiB is a shared-memory configuration of the SM; one byte more selects the 228 KiB one and
-// leaves 28 KiB of L1, which the register spills of the prologues then thrash (measured: the merge
-// prologue went from 2.6 to 9.8 us)
-static_assert(PK_SMEM_BYTES <= 196 * 1024, "shared memory map too large");
+static_assert(PK_SMEM_BYTES <= 227 * 1024, "shared memory map too large");
 
 // ---------------------------------------------------------------------------- PTX wrappers
 
@@ -119,6 +128,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// the same question without waiting: try_wait may suspend the thread for a while before it answers no
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
       : "memory");

@@ -29,7 +29,7 @@ def build_timing_library():
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
            "-DDMTD_PASS_TIMING", "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"),
-           os.path.join(HERE, "csrc", "engine.cu"), "-o", LIB]
+           os.path.join(HERE, "csrc", "engine.cu"), "-o", LIB] + os.environ.get("DMTD_NVCC_FLAGS", "").split()
     subprocess.run(cmd, check=True)
     return LIB
 
