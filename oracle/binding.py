@@ -156,7 +156,7 @@ def _pack(shape, weights):
 class Oracle:
     """One oracle context (Section 2.2's schedule on the CPU)."""
 
-    def __init__(self, shape, weights, L_d, tau, max_batch=1, max_seq=256, literal_sum=False):
+    def __init__(self, shape, weights, L_d, tau, max_batch=1, max_seq=256, literal_sum=False, L_e=0):
         self.lib = lib()
         self.shape = shape
         self._s, self._w, self._keep = _pack(shape, weights)
@@ -169,6 +169,10 @@ class Oracle:
         self.B = 0
         if literal_sum:
             self.lib.dll.oracle_set_literal_sum(self._ctx, 1)
+        if L_e:
+            rc = self.lib.dll.oracle_set_encoding_layers(self._ctx, L_e)
+            if rc:
+                raise ValueError(f"oracle_set_encoding_layers failed: {rc}")
 
     def close(self):
         if self._ctx:
@@ -300,15 +304,15 @@ def vanilla_generate(shape, weights, prompt, n_new, forced=None):
     return toks, logits, am
 
 
-def masked_parallel_forward(shape, weights, L_d, tau, tokens, P, literal_sum=False):
+def masked_parallel_forward(shape, weights, L_d, tau, tokens, P, literal_sum=False, L_e=0):
     """Eq. 1-5 in one pass over `tokens`; logits at positions P-1 .. n-1."""
     l = lib()
     s, w, keep = _pack(shape, weights)
     tokens = np.ascontiguousarray(tokens, np.int32).reshape(-1)
     n = tokens.size
     out = np.empty((n - (P - 1), shape.vocab), np.float64)
-    rc = l.dll.oracle_masked_parallel_forward(
-        C.byref(s), C.byref(w), L_d, tau, tokens.ctypes.data_as(C.c_void_p), n, P,
+    rc = l.dll.oracle_masked_parallel_forward_exdy(
+        C.byref(s), C.byref(w), L_e, L_d, tau, tokens.ctypes.data_as(C.c_void_p), n, P,
         1 if literal_sum else 0, out.ctypes.data_as(C.c_void_p))
     if rc:
         raise RuntimeError(f"oracle_masked_parallel_forward: {rc}")

@@ -218,6 +218,8 @@ struct oracle_ctx {
   oracle_weights w;
   oracle_layer_weights *layers;
   int32_t L_d, tau, max_batch, max_seq, B, literal_sum;
+  int32_t L_e;            /* encoding layers reused by the short passes (the ExDy variant); 0 = none */
+  double *h_enc;          /* [max_batch][max_seq][hidden]: output of the encoding layers at every decode position */
   double *kc, *vc;        /* [n_layers][max_batch][max_seq][nkv*d] */
   int32_t *tokens;        /* [max_batch][max_seq] */
   oracle_state st;
@@ -252,9 +254,10 @@ int oracle_create(const oracle_shape *shape, int32_t L_d, int32_t tau, int32_t m
   c->kc = (double *)calloc(n, sizeof(double));
   c->vc = (double *)calloc(n, sizeof(double));
   c->tokens = (int32_t *)calloc((size_t)max_batch * max_seq, sizeof(int32_t));
+  c->h_enc = (double *)calloc((size_t)max_batch * max_seq * shape->hidden, sizeof(double));
   c->calls = (int64_t *)calloc((size_t)shape->n_layers, sizeof(int64_t));
   c->rows = (int64_t *)calloc((size_t)shape->n_layers, sizeof(int64_t));
-  if (!c->kc || !c->vc || !c->tokens) { oracle_destroy(c); return -4; }
+  if (!c->kc || !c->vc || !c->tokens || !c->h_enc) { oracle_destroy(c); return -4; }
   oracle_reset(c);
   *out = c;
   return 0;
@@ -262,7 +265,7 @@ int oracle_create(const oracle_shape *shape, int32_t L_d, int32_t tau, int32_t m
 
 void oracle_destroy(oracle_ctx *c) {
   if (!c) return;
-  free(c->layers); free(c->kc); free(c->vc); free(c->tokens); free(c->trace);
+  free(c->layers); free(c->kc); free(c->vc); free(c->tokens); free(c->trace); free(c->h_enc);
   free(c->calls); free(c->rows); free(c);
 }
 
@@ -280,6 +283,14 @@ int oracle_set_tau(oracle_ctx *c, int32_t tau) {
   if (!c || tau < 1) return -1;
   if (c->prefilled && c->st.slot != 0) return -3;    /* only at a cycle boundary */
   c->tau = tau; c->st.tau = tau;
+  return 0;
+}
+
+int oracle_set_encoding_layers(oracle_ctx *c, int32_t L_e) {
+  if (!c || L_e < 0) return -1;
+  if (c->prefilled) return -3;                          /* a property of the whole generation */
+  if (L_e + c->L_d > c->s.n_layers) return -2;
+  c->L_e = L_e;
   return 0;
 }
 
@@ -350,16 +361,16 @@ int oracle_prefill(oracle_ctx *c, const int32_t *prompt, int32_t B, int32_t P,
       int R = P - p0 < chunk ? P - p0 : chunk;
       const int32_t *tok = c->tokens + (size_t)b * c->max_seq + p0;
       embed_rows(&c->s, &c->w, tok, R, x);
+      /* base of Eq. 4's sum: the embedding, or (ExDy) the output of the encoding layers */
+      double *base = (double *)malloc((size_t)R * H * sizeof(double));
       for (int l = 0; l < L; ++l) {
-        if (l == lo && c->literal_sum) {
-          double *e = (double *)malloc((size_t)R * H * sizeof(double));
-          embed_rows(&c->s, &c->w, tok, R, e);
-          for (size_t i = 0; i < (size_t)R * H; ++i) x[i] += e[i];
-          free(e);
-        }
+        if (l == c->L_e) memcpy(base, x, (size_t)R * H * sizeof(double));
+        if (l == lo && c->literal_sum)
+          for (size_t i = 0; i < (size_t)R * H; ++i) x[i] += base[i];
         layer_forward(&c->s, &c->layers[l], x, R, p0, oracle_k_cache(c, l, b),
                       oracle_v_cache(c, l, b));
       }
+      free(base);
       if (p0 + R == P) memcpy(last + (size_t)b * H, x + (size_t)(R - 1) * H, (size_t)H * sizeof(double));
     }
   }
@@ -374,35 +385,41 @@ int oracle_prefill(oracle_ctx *c, const int32_t *prompt, int32_t B, int32_t P,
   return 0;
 }
 
-/* One forward pass of the decode stage, full or upper-only according to the slot. */
+/* One forward pass of the decode stage, full or short according to the slot.
+ *
+ * Every pass first takes the newest token's embedding through the L_e encoding layers (none in
+ * the paper's default E0Dy setting) and keeps the result, h_enc, for that position: it is the
+ * input of the decoding layers in a short pass (Section 2.1: h_enc takes the place of h_emb when
+ * the encoding layers are reused too) and the input of the thinking layers when the position is
+ * refilled.  lo_len is the number of positions with KV in the thinking layers [L_e, L - L_d). */
 static int run_pass(oracle_ctx *c, const int32_t *forced, int forced_stride, int32_t *out_token,
                     int out_stride, double *out_logits) {
   if (c->st.n_known + 1 > c->max_seq) return -4;
-  int B = c->B, H = c->s.hidden, L = c->s.n_layers, lo = L - c->L_d;
+  int B = c->B, H = c->s.hidden, L = c->s.n_layers, lo = L - c->L_d, Le = c->L_e;
   int newest = c->st.n_known - 1;          /* position of the token whose id we learnt last */
-  double *xu = (double *)malloc((size_t)B * H * sizeof(double));   /* upper-stack input */
+  double *xu = (double *)malloc((size_t)B * H * sizeof(double));   /* decoding-stack input */
+  for (int b = 0; b < B; ++b)
+    embed_rows(&c->s, &c->w, c->tokens + (size_t)b * c->max_seq + newest, 1, xu + (size_t)b * H);
+  run_layers(c, 0, Le, xu, B, 1, newest);
+  for (int b = 0; b < B; ++b)
+    memcpy(c->h_enc + ((size_t)b * c->max_seq + newest) * H, xu + (size_t)b * H, (size_t)H * sizeof(double));
   if (c->st.slot != 0) {
-    /* upper-only pass: the newest token's embedding goes straight into the decoding layers */
-    for (int b = 0; b < B; ++b)
-      embed_rows(&c->s, &c->w, c->tokens + (size_t)b * c->max_seq + newest, 1, xu + (size_t)b * H);
+    /* short pass: h_enc of the newest token goes straight into the decoding layers */
     record_pass(c, 2, 0, 0, newest, newest + 1);
   } else {
-    /* full pass: every position the lower layers have not seen yet (the tau-1 tokens of the
+    /* full pass: every position the thinking layers have not seen yet (the tau-1 tokens of the
      * previous cycle plus the newest) goes through them together - this refills their KV -
      * and only the newest row continues upward */
     int p0 = c->st.lo_len, R = c->st.n_known - p0;
     double *x = (double *)malloc((size_t)B * R * H * sizeof(double));
     for (int b = 0; b < B; ++b)
-      embed_rows(&c->s, &c->w, c->tokens + (size_t)b * c->max_seq + p0, R, x + (size_t)b * R * H);
-    run_layers(c, 0, lo, x, B, R, p0);
+      memcpy(x + (size_t)b * R * H, c->h_enc + ((size_t)b * c->max_seq + p0) * H, (size_t)R * H * sizeof(double));
+    run_layers(c, Le, lo, x, B, R, p0);
     for (int b = 0; b < B; ++b) {
-      memcpy(xu + (size_t)b * H, x + ((size_t)b * R + (R - 1)) * H, (size_t)H * sizeof(double));
-      if (c->literal_sum) {
-        double *e = (double *)malloc((size_t)H * sizeof(double));
-        embed_rows(&c->s, &c->w, c->tokens + (size_t)b * c->max_seq + newest, 1, e);
-        for (int i = 0; i < H; ++i) xu[(size_t)b * H + i] += e[i];
-        free(e);
-      }
+      double *dst = xu + (size_t)b * H;
+      const double *think = x + ((size_t)b * R + (R - 1)) * H;
+      const double *base = c->h_enc + ((size_t)b * c->max_seq + newest) * H;
+      for (int i = 0; i < H; ++i) dst[i] = c->literal_sum ? base[i] + think[i] : think[i];
     }
     free(x);
     c->st.cycle += 1;
@@ -521,27 +538,35 @@ int oracle_anchor_mask(int32_t p, int32_t P, int32_t tau) {
   return (p < P) || ((p - (P - 1)) % tau == 0);
 }
 
-int oracle_masked_parallel_forward(const oracle_shape *shape, const oracle_weights *w,
-                                   int32_t L_d, int32_t tau, const int32_t *tokens, int32_t n,
-                                   int32_t P, int32_t literal_sum, double *out_logits) {
+int oracle_masked_parallel_forward_exdy(const oracle_shape *shape, const oracle_weights *w,
+                                        int32_t L_e, int32_t L_d, int32_t tau,
+                                        const int32_t *tokens, int32_t n, int32_t P,
+                                        int32_t literal_sum, double *out_logits) {
   if (!shape_ok(shape) || !w || !tokens || !out_logits) return -1;
-  if (L_d < 1 || L_d > shape->n_layers || tau < 1 || P < 1 || n < P) return -1;
+  if (L_d < 1 || L_e < 0 || L_e + L_d > shape->n_layers || tau < 1 || P < 1 || n < P) return -1;
   int H = shape->hidden, L = shape->n_layers, lo = L - L_d;
-  double *emb = (double *)malloc((size_t)n * H * sizeof(double));
+  double *enc = (double *)malloc((size_t)n * H * sizeof(double));
   double *think = (double *)malloc((size_t)n * H * sizeof(double));
-  embed_rows(shape, w, tokens, n, emb);
-  memcpy(think, emb, (size_t)n * H * sizeof(double));
-  forward_no_reuse(shape, w, 0, lo, think, n);                   /* Eq. 1-2 */
+  embed_rows(shape, w, tokens, n, enc);                          /* h_emb */
+  forward_no_reuse(shape, w, 0, L_e, enc, n);                    /* Eq. 1: h_enc (= h_emb when L_e = 0) */
+  memcpy(think, enc, (size_t)n * H * sizeof(double));
+  forward_no_reuse(shape, w, L_e, lo, think, n);                 /* Eq. 2: h_think */
   for (int p = 0; p < n; ++p) {
     int m = oracle_anchor_mask(p, P, tau);                        /* Eq. 3 */
     for (int i = 0; i < H; ++i) {
       size_t j = (size_t)p * H + i;
-      if (!m) think[j] = emb[j];
-      else if (literal_sum) think[j] = emb[j] + think[j];
+      if (!m) think[j] = enc[j];                                  /* Eq. 4 with h_enc in h_emb's place */
+      else if (literal_sum) think[j] = enc[j] + think[j];
     }
   }
   forward_no_reuse(shape, w, lo, L, think, n);                   /* Eq. 5: decoding layers */
   lm_head(shape, w, think + (size_t)(P - 1) * H, n - (P - 1), out_logits);
-  free(emb); free(think);
+  free(enc); free(think);
   return 0;
+}
+
+int oracle_masked_parallel_forward(const oracle_shape *shape, const oracle_weights *w,
+                                   int32_t L_d, int32_t tau, const int32_t *tokens, int32_t n,
+                                   int32_t P, int32_t literal_sum, double *out_logits) {
+  return oracle_masked_parallel_forward_exdy(shape, w, 0, L_d, tau, tokens, n, P, literal_sum, out_logits);
 }

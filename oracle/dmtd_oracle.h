@@ -99,6 +99,11 @@ int oracle_set_tau(oracle_ctx *c, int32_t tau);
 /* full_pass_add_emb = 1 switches the upper-layer input at full-pass positions to
  * embedding + lower-stack output (the literal sum of Eq. 4); default 0 (select).        */
 int oracle_set_literal_sum(oracle_ctx *c, int32_t on);
+/* The ExDy variant (Section 2.1, the paragraph after Eq. 4; Section 3.3): the short passes reuse
+ * the first L_e encoding layers as well as the last L_d decoding layers, and the decoding layers
+ * read the encoding layers' output where the default reads the embedding.  Before prefill only;
+ * L_e + L_d <= n_layers.  Default 0 (the paper's E0Dy setting).                            */
+int oracle_set_encoding_layers(oracle_ctx *c, int32_t L_e);
 
 /* Pass 1 of cycle 1: all P prompt rows through all layers.  out_token[B] = argmax of the
  * last row's logits (lowest index wins ties); out_logits [B][vocab] may be NULL.  If
@@ -143,6 +148,14 @@ int oracle_anchor_mask(int32_t p, int32_t P, int32_t tau);   /* the mask m_p of 
 int oracle_masked_parallel_forward(const oracle_shape *shape, const oracle_weights *w,
                                    int32_t L_d, int32_t tau, const int32_t *tokens, int32_t n,
                                    int32_t P, int32_t literal_sum, double *out_logits);
+
+/* The same with L_e encoding layers reused (ExDy): h_enc = EncodingLayers(h_emb) is computed for
+ * every position, h_think = ThinkingLayers(h_enc), and the decoding layers read h_think at mask
+ * positions (h_enc + h_think with literal_sum) and h_enc elsewhere.                         */
+int oracle_masked_parallel_forward_exdy(const oracle_shape *shape, const oracle_weights *w,
+                                        int32_t L_e, int32_t L_d, int32_t tau,
+                                        const int32_t *tokens, int32_t n, int32_t P,
+                                        int32_t literal_sum, double *out_logits);
 
 #ifdef __cplusplus
 }

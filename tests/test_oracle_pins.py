@@ -489,3 +489,95 @@ def test_set_tau_after_prefill_at_cycle_boundary():
     assert (tr[5]["kind"], tr[5]["lo_begin"], tr[5]["lo_end"]) == (1, P + 3, P + 5)
     st = o.state()
     assert st["cycle"] == 3 and st["lo_len"] == P + 5 and st["slot"] == 0
+
+
+# ----------------------------------------------------------------------------- ExDy (encoding layers reused too)
+
+def _run_exdy(shape, w, L_e, L_d, tau, prompt, forced, literal=False):
+    o = oracle.Oracle(shape, w, L_d=L_d, tau=tau, max_seq=prompt.shape[1] + forced.shape[1] + 1,
+                      literal_sum=literal, L_e=L_e)
+    tok, lg = o.prefill(prompt, forced_first=forced[:, 0])
+    l, am = o.decode_forced(forced[:, 1:])
+    return np.concatenate([lg[None], l], 0), o
+
+
+@pytest.mark.parametrize("L_e,L_d,tau,P", [(1, 1, 3, 5), (1, 2, 2, 4), (2, 1, 4, 7), (1, 1, 1, 3)])
+@pytest.mark.parametrize("literal", [False, True])
+def test_exdy_scheduled_equals_masked_parallel_forward(L_e, L_d, tau, P, literal):
+    """Section 2.1 (after Eq. 4): with the encoding layers reused, h_enc takes h_emb's place in
+    Eq. 4.  The cached, scheduled decode (encoding + decoding layers on every short pass, the
+    thinking layers refilled from the saved h_enc rows) must equal the one-shot masked forward
+    written from Eq. 1-5.  A refill fed with embeddings instead of h_enc, a short pass that skips
+    the encoding layers, or encoding-layer KV missing at some position each break the equality."""
+    shape = TINY
+    w = make_weights(shape, seed=6, norm_jitter=0.1)
+    n_new = 3 * tau + 2
+    prompt = make_prompts(shape.vocab, 1, P, seed=3).numpy()
+    forced = make_prompts(shape.vocab, 1, n_new, seed=4).numpy()
+    logits, o = _run_exdy(shape, w, L_e, L_d, tau, prompt, forced, literal)
+    seq = np.concatenate([prompt[0], forced[0]]).astype(np.int32)
+    ref = oracle.masked_parallel_forward(shape, w, L_d, tau, seq[:P + n_new - 1], P, literal_sum=literal, L_e=L_e)
+    np.testing.assert_allclose(logits[:, 0], ref, rtol=0, atol=1e-11)
+
+
+def test_exdy_with_no_thinking_layers_is_vanilla_decoding():
+    """L_e + L_d = L: nothing is left to skip, every pass runs every layer on one row."""
+    shape = TINY
+    w = make_weights(shape, seed=0)
+    prompt = make_prompts(shape.vocab, 1, 9, seed=1).numpy()
+    n_new = 10
+    o = oracle.Oracle(shape, w, L_d=3, tau=3, max_seq=32, L_e=1)
+    tok, lg = o.prefill(prompt)
+    toks, logits = [tok], [lg]
+    while len(toks) < n_new:
+        rc, t, l = o.decode_cycle(n_new - len(toks))
+        toks += [t[:, i] for i in range(t.shape[1])]
+        logits += [l[i] for i in range(l.shape[0])]
+    vt, vl, _ = oracle.vanilla_generate(shape, w, prompt[0], n_new)
+    assert (np.stack(toks, 1)[0] == vt[9:]).all()
+    np.testing.assert_allclose(np.stack(logits, 0)[:, 0], vl, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("L_e,L_d,tau", [(1, 1, 3), (1, 2, 2), (2, 1, 4)])
+def test_exdy_layer_counters(oracle_lib, L_e, L_d, tau):
+    """Layers traversed per cycle: the encoding and decoding layers on every pass, the thinking
+    layers once: L + (tau - 1)(L_e + L_d), i.e. Eq. 7 with L_e + L_d reused layers."""
+    shape = TINY
+    L = shape.n_layers
+    w = make_weights(shape, seed=0)
+    prompt = make_prompts(shape.vocab, 1, 4, seed=1).numpy()
+    o = oracle.Oracle(shape, w, L_d=L_d, tau=tau, max_seq=64, L_e=L_e)
+    o.prefill(prompt, want_logits=False)
+    if tau > 1:
+        o.decode_cycle(tau, want_logits=False)
+    c0, r0 = o.layer_counters()
+    n_cycles = 3
+    for _ in range(n_cycles):
+        o.decode_cycle(tau, want_logits=False)
+    c1, r1 = o.layer_counters()
+    calls, rows = c1 - c0, r1 - r0
+    for l in range(L):
+        reused = l < L_e or l >= L - L_d
+        assert calls[l] == n_cycles * (tau if reused else 1)
+        assert rows[l] == n_cycles * tau                      # every token visits every layer once
+    plt = calls.sum() / (n_cycles * tau * L)
+    assert abs(plt - oracle_lib.plt(L, L_e + L_d, tau)) < 1e-15
+
+
+def test_exdy_differs_from_decoding_layers_only():
+    """Reusing an encoding layer changes the function (it is not a re-labelling of E0Dy)."""
+    shape = TINY
+    w = make_weights(shape, seed=0)
+    prompt = make_prompts(shape.vocab, 1, 5, seed=1).numpy()
+    forced = make_prompts(shape.vocab, 1, 7, seed=2).numpy()
+    a, _ = _run_exdy(shape, w, 1, 1, 3, prompt, forced)
+    b, _ = _run_exdy(shape, w, 0, 1, 3, prompt, forced)
+    assert np.abs(a[0] - b[0]).max() == 0.0                   # the prefill is the same full-depth pass
+    assert np.abs(a[1:3] - b[1:3]).max() > 1e-3               # the short passes are not
+
+
+def test_exdy_rejects_bad_split():
+    shape = TINY
+    w = make_weights(shape, seed=0)
+    with pytest.raises(ValueError):
+        oracle.Oracle(shape, w, L_d=3, tau=3, L_e=2)           # 2 + 3 > 4 layers
