@@ -143,6 +143,20 @@ dmtd_status dmtd_decode_forced(dmtd_ctx *ctx, const int32_t *forced, int32_t n,
 dmtd_status dmtd_step_layers(dmtd_ctx *ctx, int32_t l0, int32_t l1, float *hidden, int32_t B,
                              int32_t R, int32_t pos0);
 
+/* Eq. 1-5 as one scoring pass over given token sequences (Section 2.1: the cyclical-masking
+ * forward the decode schedule is the cached, incremental form of): every position through the
+ * lower layers, the decoding layers reading the lower-stack output at mask positions (inside
+ * the prompt and at the anchors P-1 + k tau, Section 2.2) and the embedding - or, with
+ * encoding layers reused, their output - elsewhere; logits of positions P-1 .. n-1.
+ *   tokens      device int32 [B][n]: prompt (P tokens) and continuation
+ *   out_logits  device float [B][n - (P-1)][vocab]
+ * Uses the context's cycle length, decoding-layer count and options (literal_sum,
+ * encoding_layers).  Overwrites the KV cache from position 0 and leaves the context without a
+ * sequence.  Errors: STATE if the context holds a sequence; CAPACITY if B > max_batch or
+ * n > max_seq. */
+dmtd_status dmtd_masked_forward(dmtd_ctx *ctx, const int32_t *tokens, int32_t B, int32_t n,
+                                int32_t P, float *out_logits);
+
 /* Step a4 on its own: split-KV attention of R new rows per sequence against a KV cache (the
  * attention of Section 2.2's passes needs the cached K and V of every earlier token), with the
  * online-softmax merge of the key slices.  No context is needed.
@@ -210,6 +224,12 @@ dmtd_status dmtd_set_tau(dmtd_ctx *ctx, int32_t tau);
  *   "fused_pass"   0/1  run each decode pass as one persistent kernel where the model and batch
  *                       allow it (bf16 weights, bf16 or fp32 KV, head_dim 128, at most 4 rows per pass);
  *                       0 = always the per-step kernels (default 1)
+ *   "encoding_layers" x  the ExDy variant (Section 2.1, the paragraph after Eq. 4; Section 3.3): the
+ *                       short passes run the first x encoding layers as well as the last L_d
+ *                       decoding layers, the decoding layers read the encoding layers' output
+ *                       where the default reads the embedding, and a full pass refills only the
+ *                       thinking layers [x, L - L_d).  0 <= x <= L - L_d; only before the prefill;
+ *                       such contexts run the per-step kernels (default 0, the paper's E0Dy)
  *   "tc_attention" 0/1  attention of the per-step kernels by the tiled split-KV kernels for
  *                       head_dim 128 (tensor cores with a bf16 cache, FMAs with an fp32 cache)
  *                       instead of the one-warp-per-key-group kernel (default 1)
@@ -217,7 +237,7 @@ dmtd_status dmtd_set_tau(dmtd_ctx *ctx, int32_t tau);
  *                       tensor cores; bf16 contexts whose hidden, query and intermediate sizes
  *                       are multiples of 64 hold the second weight copy it reads, which doubles
  *                       the weight memory of the context (default 1)
- * Errors: INVALID_ARG for an unknown name or value. */
+ * Errors: INVALID_ARG for an unknown name or value; SHAPE / STATE for encoding_layers as above. */
 dmtd_status dmtd_set_option(dmtd_ctx *ctx, const char *name, int64_t value);
 
 /* KV cache of one layer for inspection or for filling with test data: device pointers to

@@ -81,6 +81,7 @@ def load_library():
         "dmtd_decode_cycle": [vp, i32, vp, C.POINTER(i32)],
         "dmtd_decode_forced": [vp, vp, i32, vp, vp],
         "dmtd_step_layers": [vp, i32, i32, vp, i32, i32, i32],
+        "dmtd_masked_forward": [vp, vp, i32, i32, i32, vp],
         "dmtd_prefill_host": [vp, vp, i32, i32, vp],
         "dmtd_decode_cycle_host": [vp, i32, vp, C.POINTER(i32)],
         "dmtd_get_state": [vp, C.POINTER(_State)],
@@ -204,6 +205,14 @@ class Dmtd:
         B, R, _ = hidden.shape
         self._check(self.dll.dmtd_step_layers(self._ctx, l0, l1, _ptr(hidden), B, R, pos0))
         return hidden
+
+    def masked_forward(self, tokens, P):
+        """tokens: cuda int32 [B, n].  Returns logits [B, n - (P-1), V] of positions P-1 .. n-1."""
+        assert tokens.is_cuda and tokens.dtype == torch.int32 and tokens.is_contiguous()
+        B, n = tokens.shape
+        out = torch.empty(B, n - (P - 1), self.shape.vocab, dtype=torch.float32, device=tokens.device)
+        self._check(self.dll.dmtd_masked_forward(self._ctx, _ptr(tokens), B, n, P, _ptr(out)))
+        return out
 
     def prefill_host(self, prompt_host):
         """prompt_host: CPU int32 [B, P] (pinned for speed).  Returns the first tokens as a CPU tensor."""

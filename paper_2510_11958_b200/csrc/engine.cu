@@ -41,6 +41,7 @@ struct LayerDev {
 struct dmtd_ctx {
   dmtd_model_shape s{};
   int L_d = 0, tau = 0, max_batch = 0, max_seq = 0;
+  int L_e = 0;                              // encoding layers the short passes reuse as well (ExDy); 0 = none
   int device = 0, n_sms = 0;
   cudaStream_t stream = nullptr;
   cudaStream_t capture_stream = nullptr;    // graphs are recorded here (the caller's stream may be the legacy one)
@@ -72,6 +73,9 @@ struct dmtd_ctx {
   float *x_lo = nullptr, *x_up = nullptr, *act = nullptr, *qkv = nullptr, *gu = nullptr,
         *logits = nullptr, *part_o = nullptr, *part_ml = nullptr;
   float2 *rope_tab = nullptr;
+  float *h_pend = nullptr;                  // [max_batch][pend_cap][hidden]: h_enc of positions the thinking layers have not seen
+  float *h_base = nullptr;                  // [ws_rows][hidden]: h_emb / h_enc of a chunk of rows (literal sum, masked forward)
+  int pend_cap = 0;
 
   // options
   bool use_graph = true, literal_sum = false, use_fused = true, use_tc_attention = true;
@@ -395,7 +399,7 @@ dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos
 }
 
 // Step a9/a10: final norm, tied LM head, greedy pick, token feedback.
-dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, float *out_logits) {
+dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, float *out_logits, size_t out_pitch_floats = 0) {
   const dmtd_model_shape &s = c->s;
   prep_norm_kernel<<<dim3(B, (c->ldl + PREP_ZERO_COLS - 1) / PREP_ZERO_COLS), 256, 0, c->stream>>>(
       c->x_up, s.hidden, c->w_final, s.hidden, s.rms_eps, c->act, c->lda,
@@ -403,8 +407,8 @@ dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, floa
   LAUNCH_OK(c, "prep_norm_kernel");
   TRY(launch_gemv(c, c->embed, c->embed_u, c->act, c->lda, B, c->logits, c->ldl));
   if (out_logits)
-    CUDA_TRY(c, cudaMemcpy2DAsync(out_logits, (size_t)s.vocab * 4, c->logits, (size_t)c->ldl * 4, (size_t)s.vocab * 4, B,
-                                  cudaMemcpyDeviceToDevice, c->stream));
+    CUDA_TRY(c, cudaMemcpy2DAsync(out_logits, (out_pitch_floats ? out_pitch_floats : (size_t)s.vocab) * 4, c->logits,
+                                  (size_t)c->ldl * 4, (size_t)s.vocab * 4, B, cudaMemcpyDeviceToDevice, c->stream));
   argmax_slices_kernel<<<dim3(B, ARGMAX_SLICES), 256, 0, c->stream>>>(c->logits, c->ldl, s.vocab, c->pick_val, c->pick_idx);
   LAUNCH_OK(c, "argmax_slices_kernel");
   argmax_pick_kernel<<<B, 32, 0, c->stream>>>(c->pick_val, c->pick_idx, ARGMAX_SLICES, c->tokens, c->max_seq, c->dstate,
@@ -492,7 +496,7 @@ dmtd_status setup_fused(dmtd_ctx *c) {
 }
 
 bool fused_pass_ok(const dmtd_ctx *c, int kind, int R_lower) {
-  if (!c->fused_ok || !c->use_fused || c->literal_sum) return false;
+  if (!c->fused_ok || !c->use_fused || c->literal_sum || c->L_e > 0) return false;
   const int lo = c->s.n_layers - c->L_d;
   const int R = (kind == 1 && lo > 0) ? R_lower : 1;
   return c->B * R <= PK_MAX_ROWS && R * (c->s.n_q_heads / c->s.n_kv_heads) <= PK_QR &&
@@ -535,7 +539,33 @@ dmtd_status enqueue_pass(dmtd_ctx *c, int kind, int R_lower, bool write_token, i
   const int newest = c->h.n_known - 1;
   if (!c->capturing && fused_pass_ok(c, kind, R_lower))
     return enqueue_pass_fused(c, kind, R_lower, write_token, out_argmax, out_logits);
-  if (kind == 1 && lo > 0) {
+  if (c->L_e > 0) {
+    // ExDy: the newest token's embedding goes through the encoding layers in every pass; their
+    // output h_enc is kept until the thinking layers have seen the position
+    const int Le = c->L_e;
+    TRY(launch_embed(c, &c->dstate->newest, B, 1, c->x_up, false));
+    TRY(launch_rope_table(c, &c->dstate->newest, 1));
+    for (int l = 0; l < Le; ++l) TRY(run_layer(c, l, c->x_up, B, 1, &c->dstate->newest, newest + 1));
+    if (kind == 1) {
+      // full pass: the pending rows' h_enc and the newest row's through the thinking layers
+      gather_pending_kernel<<<B * R_lower, 256, 0, c->stream>>>(c->h_pend, c->pend_cap, c->x_up, R_lower, H, c->x_lo);
+      LAUNCH_OK(c, "gather_pending_kernel");
+      TRY(launch_rope_table(c, &c->dstate->lo_len, R_lower));
+      for (int l = Le; l < lo; ++l) TRY(run_layer(c, l, c->x_lo, B, R_lower, &c->dstate->lo_len, c->h.n_known));
+      if (c->literal_sum) {
+        select_last_kernel<<<B, 256, 0, c->stream>>>(c->x_lo, R_lower, H, c->h_base);
+        LAUNCH_OK(c, "select_last_kernel");
+        copy_rows_kernel<<<64, 256, 0, c->stream>>>(c->h_base, c->x_up, (size_t)B * H / 4, 1);
+        LAUNCH_OK(c, "copy_rows_kernel");
+      } else {
+        select_last_kernel<<<B, 256, 0, c->stream>>>(c->x_lo, R_lower, H, c->x_up);
+        LAUNCH_OK(c, "select_last_kernel");
+      }
+    } else if (kind == 2) {
+      save_pending_kernel<<<B, 256, 0, c->stream>>>(c->x_up, c->h_pend, c->pend_cap, H, c->dstate);
+      LAUNCH_OK(c, "save_pending_kernel");
+    }
+  } else if (kind == 1 && lo > 0) {
     TRY(launch_embed(c, &c->dstate->lo_len, B, R_lower, c->x_lo, false));
     TRY(launch_rope_table(c, &c->dstate->lo_len, R_lower));
     for (int l = 0; l < lo; ++l) TRY(run_layer(c, l, c->x_lo, B, R_lower, &c->dstate->lo_len, c->h.n_known));
@@ -773,6 +803,9 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   CTRY(dev_alloc(c, &c->part_o, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * D));
   CTRY(dev_alloc(c, &c->part_ml, (size_t)c->ws_rows * s.n_q_heads * c->nsplit_max * 2));
   CTRY(dev_alloc(c, &c->rope_tab, (size_t)c->ws_rows * (D / 2)));
+  c->pend_cap = std::max(1, c->ws_rows / max_batch);
+  CTRY(dev_alloc(c, &c->h_pend, (size_t)max_batch * c->pend_cap * H));
+  CTRY(dev_alloc(c, &c->h_base, (size_t)c->ws_rows * H));
   if (c->umma_ok) CTRY(dev_alloc(c, &c->act_blocks, (size_t)TG_MAX_SWEEPS * (c->lda / TG_KB) * 8 * TG_MAX_COLS));
   CTRY(configure_kernels(c));
   CTRY(setup_fused(c));
@@ -830,7 +863,19 @@ dmtd_status dmtd_prefill(dmtd_ctx *c, const int32_t *prompt, int32_t B, int32_t 
     TRY(launch_embed(c, &c->dstate->scratch, B, R, c->x_lo, false));
     TRY(launch_rope_table(c, &c->dstate->scratch, R));
     for (int l = 0; l < L; ++l) {
-      if (l == lo && c->literal_sum && lo > 0) TRY(launch_embed(c, &c->dstate->scratch, B, R, c->x_lo, true));
+      if (c->literal_sum && c->L_e > 0) {
+        // Eq. 4's sum with h_enc in h_emb's place: keep the encoding layers' output, add it at the boundary
+        if (l == c->L_e) {
+          copy_rows_kernel<<<256, 256, 0, c->stream>>>(c->x_lo, c->h_base, (size_t)B * R * c->s.hidden / 4, 0);
+          LAUNCH_OK(c, "copy_rows_kernel");
+        }
+        if (l == lo) {
+          copy_rows_kernel<<<256, 256, 0, c->stream>>>(c->h_base, c->x_lo, (size_t)B * R * c->s.hidden / 4, 1);
+          LAUNCH_OK(c, "copy_rows_kernel");
+        }
+      } else if (l == lo && c->literal_sum && lo > 0) {
+        TRY(launch_embed(c, &c->dstate->scratch, B, R, c->x_lo, true));
+      }
       TRY(run_layer(c, l, c->x_lo, B, R, &c->dstate->scratch, p0 + R));
     }
     last_R = R;
@@ -911,6 +956,45 @@ dmtd_status dmtd_step_layers(dmtd_ctx *c, int32_t l0, int32_t l1, float *hidden,
   return DMTD_OK;
 }
 
+dmtd_status dmtd_masked_forward(dmtd_ctx *c, const int32_t *tokens, int32_t B, int32_t n, int32_t P, float *out_logits) {
+  if (!c) return DMTD_ERR_INVALID_ARG;
+  if (!tokens || !out_logits || B < 1 || P < 1 || n < P) return fail(c, DMTD_ERR_INVALID_ARG, "masked_forward: null pointer, or not 1 <= P <= n");
+  CHECK_NOT_FAILED(c);
+  if (c->prefilled) return fail(c, DMTD_ERR_STATE, "masked_forward: the context holds a sequence; call dmtd_reset first");
+  if (B > c->max_batch || n > c->max_seq) return fail(c, DMTD_ERR_CAPACITY, "masked_forward: B=%d n=%d exceed max_batch=%d max_seq=%d", B, n, c->max_batch, c->max_seq);
+  const int L = c->s.n_layers, lo = L - c->L_d, Le = c->L_e, H = c->s.hidden;
+  c->B = B;
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->tokens, (size_t)c->max_seq * 4, tokens, (size_t)n * 4, (size_t)n * 4, B,
+                                cudaMemcpyDeviceToDevice, c->stream));
+  // Eq. 1-5 chunk by chunk: a chunk of rows goes through every layer before the next one starts
+  // (each layer is causal and the earlier chunks' K and V are in the cache by then).
+  const int Rc_max = std::max(1, c->ws_rows / B);
+  const size_t n_out = (size_t)(n - (P - 1));
+  for (int p0 = 0; p0 < n; p0 += Rc_max) {
+    const int R = std::min(Rc_max, n - p0);
+    const size_t n4 = (size_t)B * R * H / 4;
+    set_int_kernel<<<1, 1, 0, c->stream>>>(&c->dstate->scratch, p0);
+    LAUNCH_OK(c, "set_int_kernel");
+    TRY(launch_embed(c, &c->dstate->scratch, B, R, c->x_lo, false));                 // h_emb
+    TRY(launch_rope_table(c, &c->dstate->scratch, R));
+    for (int l = 0; l < Le; ++l) TRY(run_layer(c, l, c->x_lo, B, R, &c->dstate->scratch, p0 + R));   // Eq. 1: h_enc
+    copy_rows_kernel<<<256, 256, 0, c->stream>>>(c->x_lo, c->h_base, n4, 0);
+    LAUNCH_OK(c, "copy_rows_kernel");
+    for (int l = Le; l < lo; ++l) TRY(run_layer(c, l, c->x_lo, B, R, &c->dstate->scratch, p0 + R));  // Eq. 2: h_think
+    masked_select_kernel<<<B * R, 256, 0, c->stream>>>(c->x_lo, c->h_base, R, H, p0, P, c->tau, c->literal_sum ? 1 : 0);   // Eq. 3-4
+    LAUNCH_OK(c, "masked_select_kernel");
+    for (int l = lo; l < L; ++l) TRY(run_layer(c, l, c->x_lo, B, R, &c->dstate->scratch, p0 + R));   // Eq. 5: decoding layers
+    for (int r = std::max(0, P - 1 - p0); r < R; ++r) {                                                // ... and the LM head
+      select_row_kernel<<<B, 256, 0, c->stream>>>(c->x_lo, R, r, H, c->x_up);
+      LAUNCH_OK(c, "select_row_kernel");
+      TRY(run_head(c, B, false, nullptr, out_logits + (size_t)(p0 + r - (P - 1)) * c->s.vocab, n_out * c->s.vocab));
+    }
+  }
+  // the cache now holds this forward's K and V; the schedule state is untouched (still "no sequence")
+  c->B = 0;
+  return DMTD_OK;
+}
+
 dmtd_status dmtd_prefill_host(dmtd_ctx *c, const int32_t *prompt_host, int32_t B, int32_t P, int32_t *out_token_host) {
   if (!c) return DMTD_ERR_INVALID_ARG;
   if (!prompt_host || B < 1 || P < 1) return fail(c, DMTD_ERR_INVALID_ARG, "prefill_host: null prompt or non-positive size");
@@ -974,6 +1058,12 @@ dmtd_status dmtd_set_tau(dmtd_ctx *c, int32_t tau) {
 
 dmtd_status dmtd_set_option(dmtd_ctx *c, const char *name, int64_t value) {
   if (!c || !name) return DMTD_ERR_INVALID_ARG;
+  if (!strcmp(name, "encoding_layers")) {
+    if (c->prefilled) return fail(c, DMTD_ERR_STATE, "encoding_layers can only change before the prefill (call dmtd_reset first)");
+    if (value < 0 || value + c->L_d > c->s.n_layers)
+      return fail(c, DMTD_ERR_SHAPE, "encoding_layers must be in [0, n_layers - L_d]");
+    c->L_e = (int)value; drop_graphs(c); return DMTD_OK;
+  }
   if (value != 0 && value != 1) return fail(c, DMTD_ERR_INVALID_ARG, "option %s takes 0 or 1", name);
   if (!strcmp(name, "cuda_graph")) { c->use_graph = value != 0; return DMTD_OK; }
   if (!strcmp(name, "literal_sum")) { c->literal_sum = value != 0; drop_graphs(c); return DMTD_OK; }

@@ -525,6 +525,63 @@ __global__ void select_last_kernel(const float *__restrict__ x_lo, int R, int H,
 }
 
 // ------------------------------------------------------------------------------------
+// The ExDy variant (Section 2.1, the paragraph after Eq. 4): the short passes also run the first
+// L_e encoding layers, and the output of those layers, h_enc, stands where the default has the
+// embedding.  h_enc of a position that has not been through the thinking layers yet is kept
+// (pending row = position - lo_len) and fed to them at the next full pass.
+// ------------------------------------------------------------------------------------
+// pend[b][newest - lo_len][:] = x_up[b][:]
+__global__ void save_pending_kernel(const float *__restrict__ x_up, float *__restrict__ pend, int pend_cap, int H,
+                                    const DevState *st) {
+  const int b = blockIdx.x, r = st->newest - st->lo_len;
+  if (r < 0 || r >= pend_cap) return;
+  float *dst = pend + ((size_t)b * pend_cap + r) * H;
+  for (int k = threadIdx.x; k < H; k += blockDim.x) dst[k] = x_up[(size_t)b * H + k];
+}
+
+// x_lo[b][r][:] = pend[b][r][:] for r < R - 1, x_up[b][:] for the newest row r = R - 1
+__global__ void gather_pending_kernel(const float *__restrict__ pend, int pend_cap, const float *__restrict__ x_up, int R, int H,
+                                      float *__restrict__ x_lo) {
+  const int b = blockIdx.x / R, r = blockIdx.x % R;
+  const float *src = r < R - 1 ? pend + ((size_t)b * pend_cap + r) * H : x_up + (size_t)b * H;
+  float *dst = x_lo + (size_t)blockIdx.x * H;
+  for (int k = threadIdx.x; k < H; k += blockDim.x) dst[k] = src[k];
+}
+
+// dst[i] = src[i] / dst[i] += src[i], n floats (n a multiple of 4)
+__global__ void copy_rows_kernel(const float *__restrict__ src, float *__restrict__ dst, size_t n4, int accumulate) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    float4 v = reinterpret_cast<const float4 *>(src)[i];
+    if (accumulate) {
+      const float4 d = reinterpret_cast<const float4 *>(dst)[i];
+      v.x += d.x; v.y += d.y; v.z += d.z; v.w += d.w;
+    }
+    reinterpret_cast<float4 *>(dst)[i] = v;
+  }
+}
+
+// Eq. 3-4 over a chunk of rows of the masked parallel forward: row (b, r) sits at position
+// p0 + r; at a mask position (inside the prompt, or (p - (P-1)) mod tau == 0: the anchors of
+// Section 2.2) the decoding layers read h_think (x), or base + h_think with the literal sum of
+// Eq. 4; elsewhere they read base (h_emb, or h_enc when encoding layers are reused).
+__global__ void masked_select_kernel(float *__restrict__ x, const float *__restrict__ base, int R, int H, int p0, int P,
+                                     int tau, int literal_sum) {
+  const int r = blockIdx.x % R, p = p0 + r;
+  const bool m = p < P || (p - (P - 1)) % tau == 0;
+  float *xr = x + (size_t)blockIdx.x * H;
+  const float *br = base + (size_t)blockIdx.x * H;
+  if (m && !literal_sum) return;
+  for (int k = threadIdx.x; k < H; k += blockDim.x) xr[k] = m ? br[k] + xr[k] : br[k];
+}
+
+// x_up[b][:] = x[b][r][:]
+__global__ void select_row_kernel(const float *__restrict__ x, int R, int r, int H, float *__restrict__ x_up) {
+  const int b = blockIdx.x;
+  const float *src = x + ((size_t)b * R + r) * H;
+  for (int k = threadIdx.x; k < H; k += blockDim.x) x_up[(size_t)b * H + k] = src[k];
+}
+
+// ------------------------------------------------------------------------------------
 // a9 (second half): greedy pick, lowest index on ties; a10: feed the token back.
 // Two levels: ARGMAX_SLICES blocks per sequence each find the best of their slice of the
 // vocabulary, then one block per sequence picks among them.  The token goes to position
