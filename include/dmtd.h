@@ -217,6 +217,17 @@ dmtd_status dmtd_get_device_state(dmtd_ctx *ctx, dmtd_state *out);
  * training one, Section 3.7).  Only at a cycle boundary (slot == 0) or before prefill. */
 dmtd_status dmtd_set_tau(dmtd_ctx *ctx, int32_t tau);
 
+/* How the next token is picked from the logits.  temperature == 0 (the default): greedy, as in
+ * the paper's experiments.  temperature > 0: a draw from softmax(logits / temperature) by the
+ * Gumbel-max rule, argmax_i (logit_i / temperature - log(-log(u_i))), inside the same
+ * vocabulary-parallel pick as the greedy rule (the paper has no sampling rule; this is what a
+ * serving stack needs next to Section 3.7's runtime cycle lengths).  u_i in (0, 1) is made from
+ * the top 24 bits of word i mod 4 of Philox4x32-10 with counter (i / 4, position of the token,
+ * sequence index, 0) and key `seed`: a run is reproducible and independent of batch layout.
+ * May be changed between any two calls.  Errors: INVALID_ARG for a negative or non-finite
+ * temperature. */
+dmtd_status dmtd_set_sampling(dmtd_ctx *ctx, float temperature, uint64_t seed);
+
 /* Options, by name:
  *   "cuda_graph"   0/1  replay captured CUDA graphs for whole passes (default 1)
  *   "literal_sum"  0/1  upper-layer input of a full pass = embedding + lower-stack output, the

@@ -109,6 +109,19 @@ class OracleLib:
     def plt(self, L, L_d, tau):
         return self.dll.oracle_plt(L, L_d, tau)
 
+    def philox(self, ctr, key):
+        c = (C.c_uint32 * 4)(*ctr)
+        k = (C.c_uint32 * 2)(*key)
+        out = (C.c_uint32 * 4)()
+        self.dll.oracle_philox4x32(c, k, out)
+        return [int(v) for v in out]
+
+    def sample_token(self, z, temperature, seed, position, sequence):
+        z = np.ascontiguousarray(z, np.float64)
+        self.dll.oracle_sample_token.argtypes = [_dp, C.c_int, C.c_double, C.c_uint64, C.c_int32, C.c_int32]
+        self.dll.oracle_sample_token.restype = C.c_int32
+        return int(self.dll.oracle_sample_token(z, z.size, float(temperature), int(seed), int(position), int(sequence)))
+
 
 _lib = None
 
@@ -190,6 +203,10 @@ class Oracle:
 
     def set_tau(self, tau):
         return self.lib.dll.oracle_set_tau(self._ctx, tau)
+
+    def set_sampling(self, temperature, seed):
+        self.lib.dll.oracle_set_sampling.argtypes = [C.c_void_p, C.c_double, C.c_uint64]
+        return self.lib.dll.oracle_set_sampling(self._ctx, float(temperature), int(seed))
 
     def prefill(self, prompt, forced_first=None, want_logits=True):
         prompt = np.ascontiguousarray(prompt, np.int32)

@@ -202,6 +202,42 @@ static int32_t argmax_lowest(const double *z, int n) {
   return best;
 }
 
+/* Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3",
+ * SC'11): a counter-based generator - the four output words are a fixed function of a 128-bit
+ * counter and a 64-bit key, so the CUDA path can draw the same numbers with no shared state. */
+void oracle_philox4x32(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+    uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+    uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* Sampling from softmax(z / T) by the Gumbel-max rule: argmax_i (z_i / T + g_i) with independent
+ * standard Gumbel noise g_i = -log(-log(u_i)).  u_i in (0, 1) comes from the top 24 bits of word i mod 4 of
+ * Philox(counter = (i / 4, position, sequence, 0), key = seed): the draw depends only on the
+ * seed, the position the token will take, the sequence index and the vocabulary index.  The
+ * lowest index wins a tie, as in the greedy rule (T <= 0 means greedy). */
+int32_t oracle_sample_token(const double *z, int n, double temperature, uint64_t seed, int32_t position,
+                            int32_t sequence) {
+  if (!(temperature > 0.0)) return argmax_lowest(z, n);
+  uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  int32_t best = 0;
+  double best_v = -INFINITY;
+  for (int i = 0; i < n; ++i) {
+    uint32_t ctr[4] = {(uint32_t)(i >> 2), (uint32_t)position, (uint32_t)sequence, 0u}, r[4];
+    oracle_philox4x32(ctr, key, r);
+    double u = ((double)(r[i & 3] >> 8) + 0.5) * (1.0 / 16777216.0);      /* the word's top 24 bits: exact in fp32 too */
+    double v = z[i] / temperature - log(-log(u));
+    if (v > best_v) { best_v = v; best = i; }
+  }
+  return best;
+}
+
 static int shape_ok(const oracle_shape *s) {
   if (!s) return 0;
   if (s->n_layers < 1 || s->hidden < 1 || s->n_q_heads < 1 || s->n_kv_heads < 1) return 0;
@@ -218,6 +254,8 @@ struct oracle_ctx {
   oracle_weights w;
   oracle_layer_weights *layers;
   int32_t L_d, tau, max_batch, max_seq, B, literal_sum;
+  double temperature;     /* > 0: sample by the Gumbel-max rule; 0: greedy */
+  uint64_t sample_seed;
   int32_t L_e;            /* encoding layers reused by the short passes (the ExDy variant); 0 = none */
   double *h_enc;          /* [max_batch][max_seq][hidden]: output of the encoding layers at every decode position */
   double *kc, *vc;        /* [n_layers][max_batch][max_seq][nkv*d] */
@@ -294,6 +332,13 @@ int oracle_set_encoding_layers(oracle_ctx *c, int32_t L_e) {
   return 0;
 }
 
+int oracle_set_sampling(oracle_ctx *c, double temperature, uint64_t seed) {
+  if (!c || !(temperature >= 0.0)) return -1;
+  c->temperature = temperature;
+  c->sample_seed = seed;
+  return 0;
+}
+
 int oracle_set_literal_sum(oracle_ctx *c, int32_t on) {
   if (!c) return -1;
   c->literal_sum = on ? 1 : 0;
@@ -327,7 +372,7 @@ static void emit(oracle_ctx *c, const double *x_last /*[B][hidden]*/, const int3
   double *z = (double *)malloc((size_t)B * V * sizeof(double));
   lm_head(&c->s, &c->w, x_last, B, z);
   for (int b = 0; b < B; ++b) {
-    int32_t pick = argmax_lowest(z + (size_t)b * V, V);
+    int32_t pick = oracle_sample_token(z + (size_t)b * V, V, c->temperature, c->sample_seed, c->st.n_known, b);
     if (out_token) out_token[(size_t)b * out_stride] = pick;
     c->tokens[(size_t)b * c->max_seq + c->st.n_known] =
         forced ? forced[(size_t)b * forced_stride] : pick;

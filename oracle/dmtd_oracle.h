@@ -87,6 +87,12 @@ void oracle_attention(const double *q, const double *k, const double *v, int R, 
 void oracle_linear(const void *W, int dtype, int n_out, int n_in, const double *x, int rows,
                    double *y);
 double oracle_silu(double t);
+/* Philox4x32-10, the counter-based generator of Salmon et al. (SC'11). */
+void oracle_philox4x32(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]);
+/* One draw from softmax(z / temperature) by the Gumbel-max rule with Philox noise keyed by
+ * (seed; vocabulary index, position, sequence); temperature <= 0: greedy argmax.         */
+int32_t oracle_sample_token(const double *z, int n, double temperature, uint64_t seed,
+                            int32_t position, int32_t sequence);
 /* Eq. 7. */
 double oracle_plt(int L, int L_d, int tau);
 
@@ -99,6 +105,9 @@ int oracle_set_tau(oracle_ctx *c, int32_t tau);
 /* full_pass_add_emb = 1 switches the upper-layer input at full-pass positions to
  * embedding + lower-stack output (the literal sum of Eq. 4); default 0 (select).        */
 int oracle_set_literal_sum(oracle_ctx *c, int32_t on);
+/* temperature > 0: every emitted token is drawn from softmax(logits / temperature) (the paper
+ * decodes greedily; sampling is this build's extension, see oracle_sample_token); 0: greedy. */
+int oracle_set_sampling(oracle_ctx *c, double temperature, uint64_t seed);
 /* The ExDy variant (Section 2.1, the paragraph after Eq. 4; Section 3.3): the short passes reuse
  * the first L_e encoding layers as well as the last L_d decoding layers, and the decoding layers
  * read the encoding layers' output where the default reads the embedding.  Before prefill only;

@@ -242,6 +242,11 @@ class Dmtd:
     def set_tau(self, tau):
         self._check(self.dll.dmtd_set_tau(self._ctx, tau))
 
+    def set_sampling(self, temperature, seed):
+        self.dll.dmtd_set_sampling.argtypes = [C.c_void_p, C.c_float, C.c_uint64]
+        self.dll.dmtd_set_sampling.restype = C.c_int
+        self._check(self.dll.dmtd_set_sampling(self._ctx, float(temperature), int(seed)))
+
     def set_option(self, name, value):
         self._check(self.dll.dmtd_set_option(self._ctx, name.encode(), int(value)))
 

@@ -75,6 +75,37 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// Sampling beside the greedy rule: the token is argmax_i (z_i / T + g_i) with standard Gumbel
+// noise g_i = -log(-log(u_i)), a draw from softmax(z / T) that keeps the vocabulary-parallel
+// two-level pick of the greedy path.  u_i comes from Philox4x32-10 (Salmon et al., SC'11), a
+// counter-based generator: counter (i / 4, position, sequence, 0), key = seed, word i mod 4, its
+// top 24 bits + 1/2 over 2^24.  on == 0: greedy.
+struct SampleParams {
+  float inv_temperature;
+  unsigned key0, key1;
+  int on;
+};
+
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, unsigned k0, unsigned k1) {
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const unsigned hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const unsigned hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return c;
+}
+
+// The value the pick compares for vocabulary entry i: the logit itself, or logit / T + noise.
+__device__ __forceinline__ float pick_value(float z, int i, int position, int sequence, const SampleParams &sp) {
+  if (!sp.on) return z;
+  const uint4 r = philox4x32_10(make_uint4((unsigned)i >> 2, (unsigned)position, (unsigned)sequence, 0u), sp.key0, sp.key1);
+  const unsigned w = (i & 3) == 0 ? r.x : (i & 3) == 1 ? r.y : (i & 3) == 2 ? r.z : r.w;
+  const float u = ((float)(w >> 8) + 0.5f) * (1.0f / 16777216.0f);
+  return z * sp.inv_temperature - logf(-logf(u));
+}
+
 __device__ __forceinline__ uint4 ldg_stream(const uint4 *p) {
   uint4 v;
   asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"

@@ -79,6 +79,8 @@ struct dmtd_ctx {
 
   // options
   bool use_graph = true, literal_sum = false, use_fused = true, use_tc_attention = true;
+  float temperature = 0.f;                  // > 0: tokens are drawn from softmax(logits / temperature); 0: greedy
+  uint64_t sample_seed = 0;
 
   // fused pass kernel: one persistent launch per pass
   bool fused_ok = false;
@@ -398,6 +400,14 @@ dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos
   return DMTD_OK;
 }
 
+SampleParams sample_params(const dmtd_ctx *c) {
+  SampleParams sp{};
+  sp.on = c->temperature > 0.f ? 1 : 0;
+  sp.inv_temperature = sp.on ? 1.f / c->temperature : 1.f;
+  sp.key0 = (unsigned)c->sample_seed; sp.key1 = (unsigned)(c->sample_seed >> 32);
+  return sp;
+}
+
 // Step a9/a10: final norm, tied LM head, greedy pick, token feedback.
 dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, float *out_logits, size_t out_pitch_floats = 0) {
   const dmtd_model_shape &s = c->s;
@@ -409,7 +419,8 @@ dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, floa
   if (out_logits)
     CUDA_TRY(c, cudaMemcpy2DAsync(out_logits, (out_pitch_floats ? out_pitch_floats : (size_t)s.vocab) * 4, c->logits,
                                   (size_t)c->ldl * 4, (size_t)s.vocab * 4, B, cudaMemcpyDeviceToDevice, c->stream));
-  argmax_slices_kernel<<<dim3(B, ARGMAX_SLICES), 256, 0, c->stream>>>(c->logits, c->ldl, s.vocab, c->pick_val, c->pick_idx);
+  argmax_slices_kernel<<<dim3(B, ARGMAX_SLICES), 256, 0, c->stream>>>(c->logits, c->ldl, s.vocab, c->pick_val, c->pick_idx,
+                                                                      c->dstate, sample_params(c));
   LAUNCH_OK(c, "argmax_slices_kernel");
   argmax_pick_kernel<<<B, 32, 0, c->stream>>>(c->pick_val, c->pick_idx, ARGMAX_SLICES, c->tokens, c->max_seq, c->dstate,
                                               write_token ? 1 : 0, out_argmax);
@@ -520,6 +531,7 @@ dmtd_status enqueue_pass_fused(dmtd_ctx *c, int kind, int R_lower, bool write_to
   P.part_o = c->f_part_o; P.part_ml = c->f_part_ml; P.amax_val = c->amax_val; P.amax_idx = c->amax_idx;
   P.out_argmax = out_argmax; P.barrier = c->grid_bar; P.error = &c->dstate->error;
   P.wait_limit = kDeviceWaitLimitTicks;
+  P.sample = sample_params(c);
   CUDA_TRY(c, cudaMemsetAsync(c->grid_bar, 0, sizeof(unsigned int), c->stream));
   void *args[] = {&P};
   CUDA_TRY(c, cudaLaunchCooperativeKernel((const void *)dmtd_pass_kernel, dim3(c->n_sms), dim3(PK_THREADS), args,
@@ -1053,6 +1065,14 @@ dmtd_status dmtd_set_tau(dmtd_ctx *c, int32_t tau) {
   c->tau = tau; c->h.tau = tau;
   CUDA_TRY(c, cudaMemcpyAsync(&c->dstate->tau, &c->tau, sizeof(int), cudaMemcpyHostToDevice, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_set_sampling(dmtd_ctx *c, float temperature, uint64_t seed) {
+  if (!c) return DMTD_ERR_INVALID_ARG;
+  if (!(temperature >= 0.f) || std::isinf(temperature)) return fail(c, DMTD_ERR_INVALID_ARG, "set_sampling: temperature must be finite and >= 0");
+  c->temperature = temperature; c->sample_seed = seed;
+  drop_graphs(c);                           // the captured passes carry the old parameters
   return DMTD_OK;
 }
 

@@ -606,14 +606,15 @@ __device__ __forceinline__ void argmax_block_reduce(float best, int bi, float *s
 
 // grid (sequences, ARGMAX_SLICES), 256 threads
 __global__ void argmax_slices_kernel(const float *__restrict__ logits, int ldl, int V, float *__restrict__ part_val,
-                                     int *__restrict__ part_idx) {
+                                     int *__restrict__ part_idx, const DevState *__restrict__ st, SampleParams sp) {
   const int b = blockIdx.x, per = (V + gridDim.y - 1) / gridDim.y;
   const int i0 = blockIdx.y * per, i1 = min(V, i0 + per);
   const float *z = logits + (size_t)b * ldl;
   float best = -INFINITY;
   int bi = 0x7fffffff;
+  const int position = st->n_known;                  // where the picked token will sit
   for (int i = i0 + threadIdx.x; i < i1; i += blockDim.x) {
-    float v = z[i];
+    float v = pick_value(z[i], i, position, b, sp);
     if (v > best) { best = v; bi = i; }
   }
   __shared__ float sv[256];

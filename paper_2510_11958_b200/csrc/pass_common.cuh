@@ -108,6 +108,7 @@ struct PassParams {
   unsigned int *barrier;                  // zero at launch
   int *error;                             // sticky, 0 = fine
   long long wait_limit;                   // clock ticks a device-side wait may take
+  SampleParams sample;                    // greedy pick, or a draw from softmax(logits / T)
   long long *timing;                      // stage time stamps (profiling builds), or NULL
 };
 

@@ -109,11 +109,12 @@ __device__ __noinline__ void argmax_partial(const PassParams &P) {
   const int i0 = blockIdx.x * per, i1 = min(P.vocab, i0 + per);
   float *sv = reinterpret_cast<float *>(S.bstage);
   int *si = reinterpret_cast<int *>(S.bstage) + PK_THREADS;
+  const int position = P.st->n_known;                 // where the picked token will sit
   for (int b = 0; b < P.B; ++b) {
     float best = -INFINITY;
     int bi = 0x7fffffff;
     for (int i = i0 + threadIdx.x; i < i1; i += PK_THREADS) {
-      const float v = __ldcg(P.logits + (size_t)b * P.ldl + i);
+      const float v = pick_value(__ldcg(P.logits + (size_t)b * P.ldl + i), i, position, b, P.sample);
       if (v > best) { best = v; bi = i; }
     }
     pk_sync();

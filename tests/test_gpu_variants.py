@@ -1,6 +1,6 @@
-"""Parity of the two variants beside the default schedule: the ExDy layer allocation (Section 2.1,
+"""Parity of the variants beside the default greedy schedule: the ExDy layer allocation (Section 2.1,
 the paragraph after Eq. 4; Section 3.3) and the masked parallel forward of Eq. 1-5 as one scoring
-pass, both through the C ABI against the CPU oracle."""
+pass, and sampling inside the fused pick, all through the C ABI against the CPU oracle."""
 import numpy as np
 import pytest
 import torch
@@ -150,3 +150,72 @@ def test_masked_forward_equals_scheduled_decode_on_the_gpu(dmtd):
     with pytest.raises(dmtd.DmtdError) as e:
         eng.masked_forward(torch.from_numpy(np.ascontiguousarray(seq)).cuda(), P)
     assert e.value.status == STATUS["STATE"]
+
+
+def _gumbel_noise(V, seed, position, sequence):
+    """Noise of the sampling rule for one (position, sequence), vectorised: Philox4x32-10 with
+    counter (i / 4, position, sequence, 0), word i mod 4, top 24 bits."""
+    m32 = np.uint64(0xFFFFFFFF)
+    c = [np.arange((V + 3) // 4, dtype=np.uint64), np.full((V + 3) // 4, position, np.uint64),
+         np.full((V + 3) // 4, sequence, np.uint64), np.zeros((V + 3) // 4, np.uint64)]
+    k0, k1 = np.uint64(seed & 0xFFFFFFFF), np.uint64(seed >> 32)
+    for _ in range(10):
+        p0, p1 = np.uint64(0xD2511F53) * c[0], np.uint64(0xCD9E8D57) * c[2]
+        c = [(p1 >> np.uint64(32)) ^ c[1] ^ k0, p1 & m32, (p0 >> np.uint64(32)) ^ c[3] ^ k1, p0 & m32]
+        k0, k1 = (k0 + np.uint64(0x9E3779B9)) & m32, (k1 + np.uint64(0xBB67AE85)) & m32
+    words = np.stack(c, 1).reshape(-1)[:V]
+    u = ((words >> np.uint64(8)).astype(np.float64) + 0.5) / 16777216.0
+    return -np.log(-np.log(u))
+
+
+@pytest.mark.parametrize("B,fused", [(1, 1), (1, 0), (3, 1)])
+def test_sampling_matches_oracle_draws(dmtd, B, fused):
+    """Tokens drawn from softmax(logits / T) inside the fused pick (pass kernel at batch 1, per-step
+    kernels otherwise): teacher-forced, the model's own draw at every pass against the oracle's
+    wherever the oracle's decision (logit / T + noise) has a clear margin; the noise is a function
+    of (seed, position, sequence, index) alone, so both sides see the same."""
+    shape = SHAPES["mid"]
+    w = make_weights(shape, seed=0, norm_jitter=0.1)
+    P, n_new, L_d, tau, T, seed = 12, 13, 2, 3, 0.8, 0x1234567887654321
+    prompts = make_prompts(shape.vocab, B, P, seed=1).numpy()
+    forced = make_prompts(shape.vocab, B, n_new, seed=2).numpy()
+    o = oracle.Oracle(shape, w, L_d=L_d, tau=tau, max_batch=B, max_seq=P + n_new + 1)
+    o.set_sampling(T, seed)
+    tok, lg = o.prefill(prompts, forced_first=forced[:, 0])
+    l, am = o.decode_forced(np.ascontiguousarray(forced[:, 1:]))
+    ref_logits, ref_draw = np.concatenate([lg[None], l], 0), np.concatenate([tok[None], am], 0)
+    eng = dmtd.Dmtd(shape, to_cuda(w), L_d=L_d, tau=tau, max_batch=B, max_seq=P + n_new + 1, kv_dtype="f32")
+    eng.set_option("fused_pass", fused)
+    eng.set_sampling(T, seed)
+    got_logits, got_draw = gpu_forced(eng, prompts, forced)
+    assert np.abs(got_logits - ref_logits).max() < 1e-3
+    n_clear = 0
+    for i in range(n_new):
+        for b in range(B):
+            v = ref_logits[i, b] / T + _gumbel_noise(shape.vocab, seed, P + i, b)
+            assert int(np.argmax(v)) == ref_draw[i, b]           # the test's restatement agrees with the oracle
+            top = np.sort(v)[-2:]
+            if top[1] - top[0] > 5e-2:
+                n_clear += 1
+                assert got_draw[i, b] == ref_draw[i, b]
+    assert n_clear >= n_new * B // 2
+    greedy = ref_logits.argmax(-1)
+    assert (ref_draw != greedy).any()                            # the draws are not the greedy picks
+    assert eng.device_state() == o.state()
+
+
+def test_sampling_free_running_is_reproducible(dmtd):
+    shape = SHAPES["mid"]
+    w = to_cuda(make_weights(shape, seed=0))
+    prompts = torch.from_numpy(make_prompts(shape.vocab, 1, 10, seed=1).numpy()).cuda()
+    runs = []
+    for seed in (7, 7, 8):
+        eng = dmtd.Dmtd(shape, w, L_d=2, tau=3, max_batch=1, max_seq=40, kv_dtype="f32")
+        eng.set_sampling(1.0, seed)
+        eng.prefill(prompts)
+        toks = []
+        for _ in range(5):
+            rc, n, out = eng.decode_cycle(3)
+            toks.append(out[:, :n].clone())
+        runs.append(torch.cat(toks, 1).cpu())
+    assert (runs[0] == runs[1]).all() and (runs[0] != runs[2]).any()

@@ -581,3 +581,57 @@ def test_exdy_rejects_bad_split():
     w = make_weights(shape, seed=0)
     with pytest.raises(ValueError):
         oracle.Oracle(shape, w, L_d=3, tau=3, L_e=2)           # 2 + 3 > 4 layers
+
+
+# ----------------------------------------------------------------------------- sampling (extension beside the greedy rule)
+
+def test_philox_known_answers(oracle_lib):
+    """The counter-based generator against its published known-answer vectors: a wrong round
+    constant, a swapped word or nine rounds instead of ten changes every output word."""
+    n = 0
+    for line in open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        w = [int(x, 16) for x in line.split()]
+        assert oracle_lib.philox(w[0:4], w[4:6]) == w[6:10]
+        n += 1
+    assert n == 3
+
+
+def test_gumbel_max_sampling_follows_softmax(oracle_lib):
+    """argmax(z / T + Gumbel noise) is a draw from softmax(z / T): over many positions the
+    frequencies must match the probabilities (a missing temperature, -log(u) in place of
+    -log(-log(u)), or noise shared between indices each fail by many standard deviations)."""
+    z = np.array([1.0, 0.2, -0.5, 2.0, 0.0, 1.5, -1.0, 0.7])
+    T, n = 0.7, 40000
+    p = np.exp(z / T - (z / T).max())
+    p /= p.sum()
+    counts = np.zeros(z.size)
+    for pos in range(n):
+        counts[oracle_lib.sample_token(z, T, 1234, pos, 0)] += 1
+    sigma = np.sqrt(n * p * (1 - p))
+    assert (np.abs(counts - n * p) < 4.5 * sigma).all(), (counts, n * p)
+    # the draw is a function of (seed, position, sequence) only
+    assert oracle_lib.sample_token(z, T, 1234, 17, 0) == oracle_lib.sample_token(z, T, 1234, 17, 0)
+    draws = lambda **kw: [oracle_lib.sample_token(z, T, kw.get("seed", 1), pos, kw.get("seq", 0)) for pos in range(64)]
+    assert draws() != draws(seed=2) and draws() != draws(seq=1)
+    # temperature 0 is the greedy rule
+    assert oracle_lib.sample_token(z, 0.0, 1234, 5, 0) == 3
+
+
+def test_sampled_generation_differs_from_greedy_and_keeps_the_schedule():
+    shape = TINY
+    w = make_weights(shape, seed=0)
+    prompt = make_prompts(shape.vocab, 2, 6, seed=1).numpy()
+    runs = []
+    for temp in (0.0, 1.0):
+        o = oracle.Oracle(shape, w, L_d=2, tau=3, max_batch=2, max_seq=32)
+        o.set_sampling(temp, 99)
+        tok, _ = o.prefill(prompt)
+        toks = [tok]
+        for _ in range(3):
+            rc, t, _ = o.decode_cycle(3)
+            toks += [t[:, i] for i in range(t.shape[1])]
+        runs.append((np.stack(toks, 1), o.state()))
+    assert runs[0][1] == runs[1][1]                       # counters do not depend on how tokens are picked
+    assert (runs[0][0] != runs[1][0]).any()
