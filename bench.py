@@ -237,6 +237,7 @@ def run_native(args, wl, shape):
         eng = Dmtd(shape, weights, L_d=L_d, tau=tau, max_batch=B, max_seq=max_seq, kv_dtype=wl.kv_dtype)
         prompts_host = make_prompts(shape.vocab, B, P, seed=wl.prompt_seed).pin_memory()
         prompts = prompts_host.cuda()
+        memory = {k: round(v / 1e9, 3) for k, v in eng.memory_info().items()}
 
         sampler = ClockSampler(physical_gpu_index(local))
         sampler.start()
@@ -322,7 +323,7 @@ def run_native(args, wl, shape):
         "config": {"workload": wl.name, "shape": wl.shape, "tau": tau, "L_d": L_d, "batch": B,
                    "prompt_len": P, "context_during_timing": [res["ctx_begin"], res["ctx_begin"] + K * tau],
                    "l2": "inputs_exceed_l2 (weights streamed per cycle >> 126 MB)",
-                   "parallelism": "replicas" if world > 1 else "single"},
+                   "parallelism": "replicas" if world > 1 else "single", "device_memory_gb": memory},
         "clocks": clocks,
         "gpu_launches": launches,
         "e2e": {"value": e2e_request, "unit": UNIT,

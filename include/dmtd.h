@@ -261,6 +261,16 @@ dmtd_status dmtd_get_kv(dmtd_ctx *ctx, int32_t layer, void **k, void **v);
  * exercised without making a GPU wait run out.  Synchronises the stream. */
 dmtd_status dmtd_debug_set_error_word(dmtd_ctx *ctx, int32_t word);
 
+/* Device memory the context holds, by purpose.  A bf16 context whose hidden, query and
+ * intermediate sizes are multiples of 64 keeps its weights twice: as the atom stream the
+ * mma.sync kernels and the pass kernel read (passes of up to 4 rows) and as the 16 KiB blocks
+ * the tcgen05 GEMM reads (more rows, and every prefill): 2 x 8.04 GB for the Qwen3-4B shape.
+ * With DMTD_WEIGHT_COPIES=1 in the environment at create only the first is kept. */
+typedef struct {
+  size_t weight_stream_bytes, weight_block_bytes, kv_cache_bytes, workspace_bytes;
+} dmtd_memory_info;
+dmtd_status dmtd_get_memory_info(const dmtd_ctx *ctx, dmtd_memory_info *out);
+
 /* Number of this library's kernels launched on the stream since create (graph replays count
  * their kernel nodes). */
 dmtd_status dmtd_get_launch_count(const dmtd_ctx *ctx, int64_t *out);

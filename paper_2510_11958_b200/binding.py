@@ -259,6 +259,17 @@ class Dmtd:
     def debug_set_error_word(self, word):
         self._check(self.dll.dmtd_debug_set_error_word(self._ctx, int(word)))
 
+    def memory_info(self):
+        """Device bytes held by the context: weights (two layouts), KV cache, workspace."""
+        class _Mem(C.Structure):
+            _fields_ = [(n, C.c_size_t) for n in ("weight_stream_bytes", "weight_block_bytes", "kv_cache_bytes",
+                                                  "workspace_bytes")]
+        m = _Mem()
+        self.dll.dmtd_get_memory_info.argtypes = [C.c_void_p, C.POINTER(_Mem)]
+        self.dll.dmtd_get_memory_info.restype = C.c_int
+        self._check(self.dll.dmtd_get_memory_info(self._ctx, C.byref(m)))
+        return {n: getattr(m, n) for n, _ in _Mem._fields_}
+
     def launch_count(self):
         n = C.c_int64(0)
         self._check(self.dll.dmtd_get_launch_count(self._ctx, C.byref(n)))

@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <numeric>
@@ -47,6 +48,8 @@ struct dmtd_ctx {
   cudaStream_t capture_stream = nullptr;    // graphs are recorded here (the caller's stream may be the legacy one)
   std::string err;
   std::vector<void *> allocs;
+  size_t mem[4] = {0, 0, 0, 0};             // device bytes held: atom-stream weights, tcgen05 block weights, KV cache, the rest
+  int mem_kind = 3;                         // category the next allocations count towards
 
   // model
   std::vector<LayerDev> layers;
@@ -126,6 +129,7 @@ dmtd_status dev_alloc(dmtd_ctx *c, T **p, size_t n) {
   void *q = nullptr;
   CUDA_TRY(c, cudaMalloc(&q, std::max<size_t>(n, 1) * sizeof(T)));
   c->allocs.push_back(q);
+  c->mem[c->mem_kind] += std::max<size_t>(n, 1) * sizeof(T);
   *p = static_cast<T *>(q);
   return DMTD_OK;
 }
@@ -169,7 +173,9 @@ dmtd_status pack_matrix(dmtd_ctx *c, PackedMat *out, int K, const void *const *s
     m.aps = choose_aps(K, aps_cap);
     m.n_slabs = K / 32 / m.aps;
     uint4 *dst = nullptr;
+    c->mem_kind = 0;
     TRY(dev_alloc(c, &dst, (size_t)packed_atoms(m) * 64));
+    c->mem_kind = 3;
     int tile0 = 0;
     for (int i = 0; i < n_src; ++i) {
       if (tile0 * 16 != (int)std::accumulate(Ns, Ns + i, 0))
@@ -184,7 +190,9 @@ dmtd_status pack_matrix(dmtd_ctx *c, PackedMat *out, int K, const void *const *s
     m.w = dst;
   } else {
     float *dst = nullptr;
+    c->mem_kind = 0;
     TRY(dev_alloc(c, &dst, (size_t)N * K));
+    c->mem_kind = 3;
     size_t off = 0;
     for (int i = 0; i < n_src; ++i) {
       CUDA_TRY(c, cudaMemcpyAsync(dst + off, srcs[i], (size_t)Ns[i] * K * 4, cudaMemcpyDeviceToDevice, c->stream));
@@ -214,7 +222,9 @@ dmtd_status pack_umma(dmtd_ctx *c, UmmaMat *out, int K, const void *const *srcs,
   m.N = N; m.K = K; m.n_tiles = (N + TG_ROWS - 1) / TG_ROWS; m.n_kb = K / TG_KB;
   uint4 *dst = nullptr;
   size_t units = (size_t)m.n_tiles * m.n_kb * (TG_WBLOCK / 16);
+  c->mem_kind = 1;
   TRY(dev_alloc(c, &dst, units));
+  c->mem_kind = 3;
   CUDA_TRY(c, cudaMemsetAsync(dst, 0, units * 16, c->stream));
   int row0 = 0;
   for (int i = 0; i < n_src; ++i) {
@@ -729,6 +739,9 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   // weights; every bf16 context whose dimensions fit also gets the copy the tcgen05 GEMM reads:
   // passes of more than 4 rows (batch x cycle length) and the prefill of every context use it
   c->umma_ok = s.weight_dtype == DMTD_BF16 && H % TG_KB == 0 && QD % TG_KB == 0 && I % TG_KB == 0;
+  // DMTD_WEIGHT_COPIES=1 in the environment keeps only the atom stream (half the weight memory):
+  // every projection then runs on the mma.sync kernels, the prefill included (slower from 5 rows up)
+  if (const char *e = getenv("DMTD_WEIGHT_COPIES")) if (atoi(e) == 1) c->umma_ok = false;
   c->layers.resize(s.n_layers);
   // k-slab width of the packed matrices: contexts small enough for the pass kernel (which stages
   // only the slabs a block's share touches, and gains from short ones) get 256-wide slabs;
@@ -781,8 +794,10 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   c->kv_layer_elems = (size_t)max_batch * s.n_kv_heads * max_seq * D;
   {
     unsigned char *p = nullptr;
+    c->mem_kind = 2;
     CTRY(dev_alloc(c, &p, c->kv_layer_elems * s.n_layers * kvb)); c->kc = p;
     CTRY(dev_alloc(c, &p, c->kv_layer_elems * s.n_layers * kvb)); c->vc = p;
+    c->mem_kind = 3;
   }
   CTRY(dev_alloc(c, &c->tokens, (size_t)max_batch * max_seq));
   CTRY(dev_alloc(c, &c->dstate, 1));
@@ -1105,6 +1120,13 @@ dmtd_status dmtd_debug_set_error_word(dmtd_ctx *c, int32_t word) {
   if (!c || word < 0) return DMTD_ERR_INVALID_ARG;
   CUDA_TRY(c, cudaMemcpyAsync(&c->dstate->error, &word, sizeof(int), cudaMemcpyHostToDevice, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return DMTD_OK;
+}
+
+dmtd_status dmtd_get_memory_info(const dmtd_ctx *c, dmtd_memory_info *out) {
+  if (!c || !out) return DMTD_ERR_INVALID_ARG;
+  out->weight_stream_bytes = c->mem[0]; out->weight_block_bytes = c->mem[1];
+  out->kv_cache_bytes = c->mem[2]; out->workspace_bytes = c->mem[3];
   return DMTD_OK;
 }
 

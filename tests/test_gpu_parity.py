@@ -460,3 +460,27 @@ def test_set_tau_at_a_cycle_boundary_in_mid_generation(dmtd):
             assert err < 1e-3
             assert eng.state()["slot"] == 0
             assert eng.device_state() == o.state()
+
+
+def test_memory_info_and_single_weight_copy(dmtd, monkeypatch):
+    """The context reports what it holds; with DMTD_WEIGHT_COPIES=1 the tcgen05 block copy of the
+    weights is not built and the projections of every row count run on the atom stream."""
+    shape = SHAPES["mid"].with_(intermediate=1856)
+    w = make_weights(shape, seed=0, norm_jitter=0.1)
+    B, P, n_new = 6, 9, 7
+    prompts = make_prompts(shape.vocab, B, P, seed=1).numpy()
+    forced = make_prompts(shape.vocab, B, n_new, seed=2).numpy()
+    ref_logits, ref_am, o = oracle_forced(shape, w, 2, 3, prompts, forced)
+    wc = to_cuda(w)
+    seen = {}
+    for copies in ("2", "1"):
+        monkeypatch.setenv("DMTD_WEIGHT_COPIES", copies)
+        eng = _engine(dmtd, shape, wc, 2, 3, B, P + n_new + 1, kv_dtype="f32")
+        m = eng.memory_info()
+        seen[copies] = m
+        n_params = shape.n_layers * (shape.params_per_layer - 2 * shape.hidden - 2 * shape.head_dim) + shape.vocab * shape.hidden
+        assert m["weight_stream_bytes"] >= 2 * n_params          # bf16, padded to whole tiles
+        assert m["kv_cache_bytes"] == 2 * shape.n_layers * B * shape.n_kv_heads * (P + n_new + 1) * shape.head_dim * 4
+        got_logits, got_am = gpu_forced(eng, prompts, forced)
+        check_logits(got_logits, ref_logits, got_am, ref_am)
+    assert seen["2"]["weight_block_bytes"] >= 2 * n_params and seen["1"]["weight_block_bytes"] == 0
