@@ -54,13 +54,17 @@ typedef enum {
   DMTD_ERR_UNSUPPORTED = -7
 } dmtd_status;
 
-enum { DMTD_F32 = 0, DMTD_BF16 = 1 };
+enum { DMTD_F32 = 0, DMTD_BF16 = 1, DMTD_F16 = 2 };   /* DMTD_F16: KV cache only */
 
 typedef struct {
   int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, intermediate, vocab;
   float rope_theta, rms_eps;
   int32_t weight_dtype;        /* DMTD_F32 or DMTD_BF16: storage type of every weight      */
-  int32_t kv_dtype;            /* DMTD_F32 or DMTD_BF16: storage type of the KV cache      */
+  int32_t kv_dtype;            /* DMTD_F32, DMTD_BF16 or DMTD_F16: storage type of the KV    */
+                               /* cache.  bf16 (8 significant bits) moves the logits of the  */
+                               /* 36-layer model by more than 2e-2; fp16 (11 bits, K and V   */
+                               /* are bounded by the QK-norm and the residual scale) by less */
+                               /* than half of that at half of fp32's bytes; fp32 by 1e-4.   */
   int32_t tied_lm_head;        /* must be 1: the LM head is the embedding matrix           */
 } dmtd_model_shape;
 

@@ -11,7 +11,7 @@ import torch
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-_DT = {"f32": 0, "bf16": 1}
+_DT = {"f32": 0, "bf16": 1, "f16": 2}
 
 
 class DmtdError(RuntimeError):
@@ -277,7 +277,7 @@ class Dmtd:
 
 
 def _kv_code(t):
-    return {torch.float32: 0, torch.bfloat16: 1}[t.dtype]
+    return {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}[t.dtype]
 
 
 def attention_decode(q, k, v, pos0, scratch=None):

@@ -25,6 +25,7 @@ struct AttnAccW {
 // Keys of the tile are key_idx0 + row; key index i sits at position (i < n_cached ? j0 + i :
 // pos_new + i - n_cached); query row q may see positions up to row_pos0 + q / G.
 // k_off / v_off: where the tile's K and V (hi parts) sit in the scratch.
+template <class Op>
 __device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *sc, const uint4 (&qh)[4][2], int n_t, int tile0,
                                                   int n_cached, int j0, int pos_new, int row_pos0, int G,
                                                   int k_off = PK_AT_KH, int v_off = PK_AT_VH) {
@@ -43,8 +44,8 @@ __device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *
           for (int kb = 0; kb < 4; ++kb) {
             const uint32_t off = (warp * 16 + nt * 8 + g) * PK_KROW + kb * 64 + t * 16;
             const uint4 Kh = lds128(kh_tile + off);
-            mma_bf16_16816(c[nt], qh[kb][0].x, qh[kb][1].x, qh[kb][0].y, qh[kb][1].y, Kh.x, Kh.y);
-            mma_bf16_16816(c[nt], qh[kb][0].z, qh[kb][1].z, qh[kb][0].w, qh[kb][1].w, Kh.z, Kh.w);
+            Op::mma(c[nt], qh[kb][0].x, qh[kb][1].x, qh[kb][0].y, qh[kb][1].y, Kh.x, Kh.y);
+            Op::mma(c[nt], qh[kb][0].z, qh[kb][1].z, qh[kb][0].w, qh[kb][1].w, Kh.z, Kh.w);
           }
         }
         // causal / range mask: lane holds rows g (e = 0, 1) and g + 8 (e = 2, 3), keys 2t, 2t + 1 of each n-tile
@@ -86,7 +87,7 @@ __device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float p0 = c[i >> 1][(i & 1) * 2], p1 = c[i >> 1][(i & 1) * 2 + 1];
-          ah[i] = pack_bf16x2(p0, p1);
+          ah[i] = Op::pack2(p0, p1);
         }
         const int mi = lane >> 3, rr = lane & 7;
         const uint32_t v_off = (warp * 16 + (mi & 1) * 8 + rr) * PK_VROW + (mi >> 1) * 16;
@@ -96,8 +97,8 @@ __device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *
           ldmatrix_x4_trans(vh_tile + v_off + d2 * 32, b0, b1, b2, b3);
           o[2 * d2][0] *= corr[0]; o[2 * d2][1] *= corr[0]; o[2 * d2][2] *= corr[1]; o[2 * d2][3] *= corr[1];
           o[2 * d2 + 1][0] *= corr[0]; o[2 * d2 + 1][1] *= corr[0]; o[2 * d2 + 1][2] *= corr[1]; o[2 * d2 + 1][3] *= corr[1];
-          mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
-          mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+          Op::mma(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
+          Op::mma(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
         }
       }
 }
@@ -171,7 +172,8 @@ constexpr int ATTN_TC_SMEM = PK_AT_ROWS;         // tiles, Q, partial-output ove
 
 // qkv [B*R][ldq]: q heads already normalised and rotated (not scaled); K and V of the new rows
 // already in the cache.  Cache [b][kv head][max_seq][128] bf16.
-__global__ void __launch_bounds__(PK_THREADS, 2)      // bf16 cache: two blocks per SM overlap load and math
+template <class Op>
+__global__ void __launch_bounds__(PK_THREADS, 2)      // 16-bit cache: two blocks per SM overlap load and math
 attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ kc, const void *__restrict__ vc, int max_seq,
                int nq, int nkv, int R, int RB, int CH, const int *__restrict__ pos0_ptr, float *__restrict__ part_o,
                float *__restrict__ part_ml, int nsplit) {
@@ -198,12 +200,11 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
   const float scale = rsqrtf((float)PK_D);
   for (int qi = warp; qi < nQ; qi += PK_WARPS) {
     const float *src = qkv + (size_t)(b * R + r0 + qi / G) * ldq + (size_t)(kvh * G + qi % G) * PK_D;
-    __nv_bfloat16 *qh = reinterpret_cast<__nv_bfloat16 *>(sc + PK_AT_QH + qi * PK_QROW);
+    typename Op::T *qh = reinterpret_cast<typename Op::T *>(sc + PK_AT_QH + qi * PK_QROW);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float v = src[lane + 32 * j] * scale;
-      const __nv_bfloat16 h = __float2bfloat16_rn(v);
-      qh[lane + 32 * j] = h;
+      qh[lane + 32 * j] = Op::from_float(v);
     }
   }
   const size_t head_off = ((size_t)b * nkv + kvh) * max_seq * PK_D;
@@ -216,8 +217,8 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
   const int n_keys = j1 - j0;
   // bf16 cache: two tile buffers (the lo-part areas are free here), tile i+1 in flight while
   // tile i is multiplied
-  const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(kc) + head_off;
-  const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(vc) + head_off;
+  const typename Op::T *kb = reinterpret_cast<const typename Op::T *>(kc) + head_off;
+  const typename Op::T *vb = reinterpret_cast<const typename Op::T *>(vc) + head_off;
   auto fetch = [&](int tile0, int buf) {
     const int n_t = min(PK_TK, n_keys - tile0);
     const uint32_t k_t = smem_u32(sc + (buf ? PK_AT_KL : PK_AT_KH)), v_t = smem_u32(sc + (buf ? PK_AT_VL : PK_AT_VH));
@@ -249,7 +250,7 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
         qh[kbk][1] = lds128(qh_tile + (g + 8) * PK_QROW + kbk * 64 + t * 16);
       }
     }
-    attn_tile_compute_w(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH,
+    attn_tile_compute_w<Op>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH,
                              buf ? PK_AT_VL : PK_AT_VH);
     __syncthreads();                                    // done with this buffer before it is refilled
   }

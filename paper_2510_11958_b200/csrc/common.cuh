@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -105,6 +106,38 @@ __device__ __forceinline__ float pick_value(float z, int i, int position, int se
   const float u = ((float)(w >> 8) + 0.5f) * (1.0f / 16777216.0f);
   return z * sp.inv_temperature - logf(-logf(u));
 }
+
+// The same with fp16 inputs (an fp16 KV cache: 11 significant bits against bf16's 8).
+__device__ __forceinline__ void mma_f16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                              uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};\n"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// 16-bit operand types of the tensor-core attention kernel.
+struct OpBf16 {
+  using T = __nv_bfloat16;
+  static __device__ __forceinline__ T from_float(float v) { return __float2bfloat16_rn(v); }
+  static __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+  }
+  static __device__ __forceinline__ void mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1) { mma_bf16_16816(d, a0, a1, a2, a3, b0, b1); }
+};
+struct OpF16 {
+  using T = __half;
+  static __device__ __forceinline__ T from_float(float v) { return __float2half_rn(v); }
+  static __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+  }
+  static __device__ __forceinline__ void mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1) { mma_f16_16816(d, a0, a1, a2, a3, b0, b1); }
+};
 
 __device__ __forceinline__ uint4 ldg_stream(const uint4 *p) {
   uint4 v;

@@ -335,7 +335,8 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
       attn_f32_kernel<<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_F32_SMEM, c->stream>>>(
           c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
     } else {
-      attn_tc_kernel<<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
+      using Op = typename std::conditional<std::is_same<KVT, __half>::value, OpF16, OpBf16>::type;
+      attn_tc_kernel<Op><<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
           c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
     }
   } else {
@@ -353,12 +354,14 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
 }
 
 dmtd_status launch_attention(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit) {
-  bool kvbf = c->s.kv_dtype == DMTD_BF16;
+  const int kv = c->s.kv_dtype;
   if (c->s.head_dim == 128)
-    return kvbf ? launch_attention_t<128, __nv_bfloat16>(c, layer, B, R, pos0, nsplit)
-                : launch_attention_t<128, float>(c, layer, B, R, pos0, nsplit);
-  return kvbf ? launch_attention_t<64, __nv_bfloat16>(c, layer, B, R, pos0, nsplit)
-              : launch_attention_t<64, float>(c, layer, B, R, pos0, nsplit);
+    return kv == DMTD_BF16 ? launch_attention_t<128, __nv_bfloat16>(c, layer, B, R, pos0, nsplit)
+         : kv == DMTD_F16 ? launch_attention_t<128, __half>(c, layer, B, R, pos0, nsplit)
+                          : launch_attention_t<128, float>(c, layer, B, R, pos0, nsplit);
+  return kv == DMTD_BF16 ? launch_attention_t<64, __nv_bfloat16>(c, layer, B, R, pos0, nsplit)
+       : kv == DMTD_F16 ? launch_attention_t<64, __half>(c, layer, B, R, pos0, nsplit)
+                        : launch_attention_t<64, float>(c, layer, B, R, pos0, nsplit);
 }
 
 dmtd_status launch_rope_table(dmtd_ctx *c, const int *pos0, int R) {
@@ -448,7 +451,10 @@ dmtd_status configure_kernels(dmtd_ctx *c) {
   CUDA_TRY(c, cudaFuncSetAttribute(gemv_bf16_kernel<4>, dyn, 100 * 1024));
   CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc05_kernel, dyn, TG_STAGES * (TG_WBLOCK + TG_MAX_COLS * 128) + 128));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_f32_kernel, dyn, ATTN_F32_SMEM));
-  CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel, dyn, ATTN_TC_SMEM));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<OpBf16>, dyn, ATTN_TC_SMEM));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<OpF16>, dyn, ATTN_TC_SMEM));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<64, __half>, dyn, 64 * 1024));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<128, __half>, dyn, 64 * 1024));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<64, float>, dyn, 64 * 1024));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<64, __nv_bfloat16>, dyn, 64 * 1024));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<128, float>, dyn, 64 * 1024));
@@ -472,7 +478,7 @@ bool fused_matrix_ok(const PackedMat &m, int grid) {
 dmtd_status setup_fused(dmtd_ctx *c) {
   const dmtd_model_shape &s = c->s;
   c->fused_ok = false;
-  if (!is_bf16(c) || s.head_dim != PK_D || s.n_layers > PK_MAX_LAYERS) return DMTD_OK;
+  if (!is_bf16(c) || s.head_dim != PK_D || s.n_layers > PK_MAX_LAYERS || s.kv_dtype == DMTD_F16) return DMTD_OK;
   if (s.n_q_heads / s.n_kv_heads > PK_MAX_GROUP || s.hidden % 8 || s.hidden > PK_XS_FLOATS) return DMTD_OK;
   int coop = 0;
   CUDA_TRY(c, cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
@@ -496,7 +502,7 @@ dmtd_status setup_fused(dmtd_ctx *c) {
     const LayerDev &ld = c->layers[l];
     h[l].qkv = ld.qkv; h[l].o = ld.o; h[l].gu = ld.gu; h[l].down = ld.down;
     h[l].w_in = ld.w_in; h[l].w_post = ld.w_post; h[l].w_qn = ld.w_qn; h[l].w_kn = ld.w_kn;
-    const size_t kvb = s.kv_dtype == DMTD_BF16 ? 2 : 4;
+    const size_t kvb = s.kv_dtype == DMTD_F32 ? 4 : 2;
     h[l].kc = static_cast<unsigned char *>(c->kc) + (size_t)l * c->kv_layer_elems * kvb;
     h[l].vc = static_cast<unsigned char *>(c->vc) + (size_t)l * c->kv_layer_elems * kvb;
   }
@@ -698,7 +704,7 @@ dmtd_status validate_shape(const dmtd_model_shape *s, int L_d, int tau, int max_
   if (s->n_q_heads / s->n_kv_heads > ATTN_QR) return fail(nullptr, DMTD_ERR_SHAPE, "at most 16 query heads per kv head");
   if (s->head_dim != 64 && s->head_dim != 128) return fail(nullptr, DMTD_ERR_SHAPE, "head_dim must be 64 or 128");
   if (s->weight_dtype != DMTD_F32 && s->weight_dtype != DMTD_BF16) return fail(nullptr, DMTD_ERR_SHAPE, "weight_dtype");
-  if (s->kv_dtype != DMTD_F32 && s->kv_dtype != DMTD_BF16) return fail(nullptr, DMTD_ERR_SHAPE, "kv_dtype");
+  if (s->kv_dtype != DMTD_F32 && s->kv_dtype != DMTD_BF16 && s->kv_dtype != DMTD_F16) return fail(nullptr, DMTD_ERR_SHAPE, "kv_dtype");
   int mult = s->weight_dtype == DMTD_BF16 ? 32 : 4;
   if (s->hidden % mult || s->intermediate % mult)
     return fail(nullptr, DMTD_ERR_SHAPE, "hidden and intermediate must be multiples of %d", mult);
@@ -790,7 +796,7 @@ dmtd_status dmtd_create(const dmtd_model_shape *shape, int32_t L_d, int32_t tau,
   }
 
   // sequence state
-  size_t kvb = s.kv_dtype == DMTD_BF16 ? 2 : 4;
+  size_t kvb = s.kv_dtype == DMTD_F32 ? 4 : 2;
   c->kv_layer_elems = (size_t)max_batch * s.n_kv_heads * max_seq * D;
   {
     unsigned char *p = nullptr;
@@ -1110,7 +1116,7 @@ dmtd_status dmtd_set_option(dmtd_ctx *c, const char *name, int64_t value) {
 
 dmtd_status dmtd_get_kv(dmtd_ctx *c, int32_t layer, void **k, void **v) {
   if (!c || layer < 0 || layer >= c->s.n_layers) return DMTD_ERR_INVALID_ARG;
-  size_t kvb = c->s.kv_dtype == DMTD_BF16 ? 2 : 4;
+  size_t kvb = c->s.kv_dtype == DMTD_F32 ? 4 : 2;
   if (k) *k = static_cast<unsigned char *>(c->kc) + (size_t)layer * c->kv_layer_elems * kvb;
   if (v) *v = static_cast<unsigned char *>(c->vc) + (size_t)layer * c->kv_layer_elems * kvb;
   return DMTD_OK;
@@ -1180,7 +1186,7 @@ dmtd_status attention_check(const float *q, const void *k, const void *v, int kv
                             int D, int max_seq, int pos0, const float *out) {
   if (!q || !k || !v || !out || B < 1 || R < 1 || pos0 < 0 || max_seq < 1)
     return fail(nullptr, DMTD_ERR_INVALID_ARG, "attention: null pointer or non-positive size");
-  if (kv_dtype != DMTD_F32 && kv_dtype != DMTD_BF16) return fail(nullptr, DMTD_ERR_SHAPE, "attention: kv_dtype");
+  if (kv_dtype != DMTD_F32 && kv_dtype != DMTD_BF16 && kv_dtype != DMTD_F16) return fail(nullptr, DMTD_ERR_SHAPE, "attention: kv_dtype");
   if (D != 64 && D != 128) return fail(nullptr, DMTD_ERR_SHAPE, "attention: head_dim must be 64 or 128");
   if (nq < 1 || nkv < 1 || nq % nkv || nq / nkv > ATTN_QR)
     return fail(nullptr, DMTD_ERR_SHAPE, "attention: n_q_heads must be a multiple of n_kv_heads, at most 16 per kv head");
@@ -1205,9 +1211,10 @@ dmtd_status attention_launch_t(const float *q, const void *k, const void *v, int
           q, ld, static_cast<const float *>(k), static_cast<const float *>(v), max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o,
           part_ml, p.nsplit);
     } else {
-      e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM);
+      using Op = typename std::conditional<std::is_same<KVT, __half>::value, OpF16, OpBf16>::type;
+      e = cudaFuncSetAttribute(attn_tc_kernel<Op>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_TC_SMEM);
       if (e != cudaSuccess) return fail(nullptr, DMTD_ERR_CUDA, "attention: %s", cudaGetErrorString(e));
-      attn_tc_kernel<<<dim3(p.nsplit, nkv * n_rb, B), PK_THREADS, ATTN_TC_SMEM, stream>>>(
+      attn_tc_kernel<Op><<<dim3(p.nsplit, nkv * n_rb, B), PK_THREADS, ATTN_TC_SMEM, stream>>>(
           q, ld, k, v, max_seq, nq, nkv, R, RB, p.CH, pos_dev, part_o, part_ml, p.nsplit);
     }
   } else {
@@ -1228,12 +1235,14 @@ dmtd_status attention_launch_t(const float *q, const void *k, const void *v, int
 dmtd_status attention_launch(const float *q, const void *k, const void *v, int kv_dtype, int B, int R, int nq, int nkv,
                              int D, int max_seq, int pos0, unsigned char *scratch, const AttnPlan &p, float *out,
                              cudaStream_t stream) {
-  bool bf = kv_dtype == DMTD_BF16;
-  if (D == 128)
-    return bf ? attention_launch_t<128, __nv_bfloat16>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream)
-              : attention_launch_t<128, float>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream);
-  return bf ? attention_launch_t<64, __nv_bfloat16>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream)
-            : attention_launch_t<64, float>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream);
+  if (D == 128) {
+    if (kv_dtype == DMTD_BF16) return attention_launch_t<128, __nv_bfloat16>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream);
+    if (kv_dtype == DMTD_F16) return attention_launch_t<128, __half>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream);
+    return attention_launch_t<128, float>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream);
+  }
+  if (kv_dtype == DMTD_BF16) return attention_launch_t<64, __nv_bfloat16>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream);
+  if (kv_dtype == DMTD_F16) return attention_launch_t<64, __half>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream);
+  return attention_launch_t<64, float>(q, k, v, B, R, nq, nkv, max_seq, pos0, scratch, p, out, stream);
 }
 
 }  // namespace

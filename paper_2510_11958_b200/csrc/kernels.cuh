@@ -271,6 +271,7 @@ template <> __device__ __forceinline__ float to_kv<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 to_kv<__nv_bfloat16>(float v) {
   return __float2bfloat16_rn(v);
 }
+template <> __device__ __forceinline__ __half to_kv<__half>(float v) { return __float2half_rn(v); }
 
 // One warp per (row, head); heads are q heads, then k heads, then v heads.  q is normalised
 // and rotated in place (fp32); k is normalised, rotated and stored in the cache; v is stored.
@@ -348,6 +349,16 @@ template <> __device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bflo
   }
 }
 
+template <> __device__ __forceinline__ void load8<__half>(const __half *p, float (&f)[8]) {
+  uint4 v = *reinterpret_cast<const uint4 *>(p);
+  const __half2 *h = reinterpret_cast<const __half2 *>(&v);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 x = __half22float2(h[j]);
+    f[2 * j] = x.x;
+    f[2 * j + 1] = x.y;
+  }
+}
 template <int D, typename KVT>
 __global__ void __launch_bounds__(ATTN_WARPS * 32)
 attn_partial_kernel(const float *__restrict__ qkv, int ldq, const KVT *__restrict__ kc,

@@ -240,11 +240,14 @@ def test_errors(dmtd):
     ("f32", 40, 1, 8, 2, 128, 1500, 1536),       # a batch large enough for long slices: 4 tiles per block, ragged
     ("f32", 24, 3, 8, 2, 128, 1000, 1024),       # the same with a refill chunk (12 query rows per tile)
     ("bf16", 40, 1, 8, 2, 128, 1500, 1536),      # several double-buffered tiles per block
+    ("f16", 1, 1, 32, 8, 128, 700, 1024),        # fp16 cache: the tensor-core kernel with fp16 operands
+    ("f16", 24, 3, 8, 2, 128, 1000, 1024),
+    ("f16", 2, 3, 4, 2, 64, 100, 128),           # head_dim 64: the one-warp-per-key-group kernel
 ])
 def test_attention_decode_matches_oracle(dmtd, oracle_lib, kvdt, B, R, nq, nkv, D, pos0, max_seq):
     """dmtd_attention_decode against the oracle's attention on the same (rounded) K and V."""
     g = torch.Generator().manual_seed(11)
-    dt = torch.float32 if kvdt == "f32" else torch.bfloat16
+    dt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[kvdt]
     q = torch.randn(B, R, nq, D, generator=g)
     k = torch.randn(B, nkv, max_seq, D, generator=g).to(dt)
     v = torch.randn(B, nkv, max_seq, D, generator=g).to(dt)
@@ -256,7 +259,8 @@ def test_attention_decode_matches_oracle(dmtd, oracle_lib, kvdt, B, R, nq, nkv, 
                                    v[b, :, :n].double().permute(1, 0, 2).numpy(), pos0)
         # head_dim 128 with a bf16 cache runs on the tensor cores: Q and P are rounded to bf16 as well
         # (2^-9 relative each); with an fp32 cache the arithmetic is plain fp32
-        tol = 5e-3 if (kvdt == "bf16" and D == 128) else 2e-5
+        # ... and with an fp16 cache to fp16 (2^-12 relative each)
+        tol = 5e-3 if (kvdt == "bf16" and D == 128) else 6e-4 if (kvdt == "f16" and D == 128) else 2e-5
         assert np.abs(got[b].double().cpu().numpy() - ref).max() <= tol * max(1.0, np.abs(ref).max())
 
 
