@@ -259,8 +259,10 @@ dmtd_status launch_gemv_nt(dmtd_ctx *c, const PackedMat &W, const float *act, in
 // weight tile with up to 128 activation rows (a sweep); prefill chunks of more rows are several
 // sweeps in one launch (up to TG_MAX_SWEEPS), ordered so that the sweeps of one weight tile run
 // together and share it through L2.
+// With `norm_w` the activations are RMSNorm(act rows) * norm_w, computed while the blocks are written, and
+// the output rows are cleared first (the projections after a norm write a fresh buffer).
 dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, int lda, int M, float *out, int ldo,
-                             int gate_up_I = 0) {
+                             int gate_up_I = 0, const float *norm_w = nullptr) {
   const int SET = TG_MAX_COLS / 2;                       // rows per sweep
   for (int m0 = 0; m0 < M; m0 += TG_MAX_SWEEPS * SET) {
     GemmTcParams P{};
@@ -283,10 +285,20 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
     if (P.n_sweeps == 1 && W.n_tiles > c->n_sms * per_sm_of(TG_STAGES) && W.n_tiles <= c->n_sms * per_sm_of(2)) P.stages = 2;
     const int slots = c->n_sms * per_sm_of(P.stages);
     P.ksplit = std::max(1, std::min(W.n_kb, slots / (W.n_tiles * P.n_sweeps)));
-    long long units = (long long)W.n_kb * 8 * P.n_cols;
-    act_blocks_kernel<<<dim3((int)std::min<long long>((units + 255) / 256, 4096), P.n_sweeps), 256, 0, c->stream>>>(
-        act + (size_t)m0 * lda, lda, P.rows, W.K, P.n_cols, c->act_blocks, gate_up_I);
-    LAUNCH_OK(c, "act_blocks_kernel");
+    if (norm_w) {
+      const int n_groups = P.n_sweeps * (P.n_cols / 2 / NAB_ROWS);
+      const size_t zero_n4 = (size_t)P.rows * ldo / 4;                  // ldo is a multiple of 4 (checked by the caller)
+      const int n_zero = (int)std::min<size_t>((zero_n4 + 1023) / 1024, 2 * c->n_sms);
+      norm_act_blocks_kernel<<<n_groups + n_zero, 256, 0, c->stream>>>(
+          act + (size_t)m0 * lda, lda, norm_w, c->s.rms_eps, P.rows, W.K, P.n_cols, c->act_blocks, n_groups,
+          reinterpret_cast<float4 *>(out + (size_t)m0 * ldo), zero_n4);
+      LAUNCH_OK(c, "norm_act_blocks_kernel");
+    } else {
+      long long units = (long long)W.n_kb * 8 * P.n_cols;
+      act_blocks_kernel<<<dim3((int)std::min<long long>((units + 255) / 256, 4096), P.n_sweeps), 256, 0, c->stream>>>(
+          act + (size_t)m0 * lda, lda, P.rows, W.K, P.n_cols, c->act_blocks, gate_up_I);
+      LAUNCH_OK(c, "act_blocks_kernel");
+    }
     int smem = smem_of(P.stages);
     // launched with programmatic stream serialisation: its blocks may start (allocate tensor
     // memory, request their first weight blocks) while act_blocks_kernel is still running
@@ -391,17 +403,27 @@ dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos
   const dmtd_model_shape &s = c->s;
   const LayerDev &lw = c->layers[l];
   int M = B * R, H = s.hidden, I = s.intermediate, QD = s.n_q_heads * s.head_dim;
-  prep_norm_kernel<<<dim3(M, (c->ldqkv + PREP_ZERO_COLS - 1) / PREP_ZERO_COLS), 256, 0, c->stream>>>(
-      x, H, lw.w_in, H, s.rms_eps, c->act, c->lda, c->qkv, c->ldqkv, c->ldqkv);
-  LAUNCH_OK(c, "prep_norm_kernel");
-  TRY(launch_gemv(c, lw.qkv, lw.qkv_u, c->act, c->lda, M, c->qkv, c->ldqkv));
+  // the tcgen05 path normalises while it writes its activation blocks
+  const bool tc = lw.qkv_u.w && c->use_umma && M > 4 && c->ldqkv % 4 == 0 && c->ldgu % 4 == 0;
+  if (tc) {
+    TRY(launch_gemm_tc05(c, lw.qkv_u, x, H, M, c->qkv, c->ldqkv, 0, lw.w_in));
+  } else {
+    prep_norm_kernel<<<dim3(M, (c->ldqkv + PREP_ZERO_COLS - 1) / PREP_ZERO_COLS), 256, 0, c->stream>>>(
+        x, H, lw.w_in, H, s.rms_eps, c->act, c->lda, c->qkv, c->ldqkv, c->ldqkv);
+    LAUNCH_OK(c, "prep_norm_kernel");
+    TRY(launch_gemv(c, lw.qkv, lw.qkv_u, c->act, c->lda, M, c->qkv, c->ldqkv));
+  }
   TRY(launch_attention(c, l, B, R, pos0, splits_for(c, pos_end)));
   (void)QD;
   TRY(launch_gemv(c, lw.o, lw.o_u, c->act, c->lda, M, x, H));
-  prep_norm_kernel<<<dim3(M, (c->ldgu + PREP_ZERO_COLS - 1) / PREP_ZERO_COLS), 256, 0, c->stream>>>(
-      x, H, lw.w_post, H, s.rms_eps, c->act, c->lda, c->gu, c->ldgu, c->ldgu);
-  LAUNCH_OK(c, "prep_norm_kernel");
-  TRY(launch_gemv(c, lw.gu, lw.gu_u, c->act, c->lda, M, c->gu, c->ldgu));
+  if (tc) {
+    TRY(launch_gemm_tc05(c, lw.gu_u, x, H, M, c->gu, c->ldgu, 0, lw.w_post));
+  } else {
+    prep_norm_kernel<<<dim3(M, (c->ldgu + PREP_ZERO_COLS - 1) / PREP_ZERO_COLS), 256, 0, c->stream>>>(
+        x, H, lw.w_post, H, s.rms_eps, c->act, c->lda, c->gu, c->ldgu, c->ldgu);
+    LAUNCH_OK(c, "prep_norm_kernel");
+    TRY(launch_gemv(c, lw.gu, lw.gu_u, c->act, c->lda, M, c->gu, c->ldgu));
+  }
   if (lw.down_u.w && c->use_umma && M > 4) {
     // the tcgen05 path gates while it writes its activation blocks
     TRY(launch_gemm_tc05(c, lw.down_u, c->gu, c->ldgu, M, x, H, I));
@@ -424,11 +446,15 @@ SampleParams sample_params(const dmtd_ctx *c) {
 // Step a9/a10: final norm, tied LM head, greedy pick, token feedback.
 dmtd_status run_head(dmtd_ctx *c, int B, bool write_token, int *out_argmax, float *out_logits, size_t out_pitch_floats = 0) {
   const dmtd_model_shape &s = c->s;
-  prep_norm_kernel<<<dim3(B, (c->ldl + PREP_ZERO_COLS - 1) / PREP_ZERO_COLS), 256, 0, c->stream>>>(
-      c->x_up, s.hidden, c->w_final, s.hidden, s.rms_eps, c->act, c->lda,
-                                             c->logits, c->ldl, c->ldl);
-  LAUNCH_OK(c, "prep_norm_kernel");
-  TRY(launch_gemv(c, c->embed, c->embed_u, c->act, c->lda, B, c->logits, c->ldl));
+  if (c->embed_u.w && c->use_umma && B > 4 && c->ldl % 4 == 0) {
+    TRY(launch_gemm_tc05(c, c->embed_u, c->x_up, s.hidden, B, c->logits, c->ldl, 0, c->w_final));
+  } else {
+    prep_norm_kernel<<<dim3(B, (c->ldl + PREP_ZERO_COLS - 1) / PREP_ZERO_COLS), 256, 0, c->stream>>>(
+        c->x_up, s.hidden, c->w_final, s.hidden, s.rms_eps, c->act, c->lda,
+                                               c->logits, c->ldl, c->ldl);
+    LAUNCH_OK(c, "prep_norm_kernel");
+    TRY(launch_gemv(c, c->embed, c->embed_u, c->act, c->lda, B, c->logits, c->ldl));
+  }
   if (out_logits)
     CUDA_TRY(c, cudaMemcpy2DAsync(out_logits, (out_pitch_floats ? out_pitch_floats : (size_t)s.vocab) * 4, c->logits,
                                   (size_t)c->ldl * 4, (size_t)s.vocab * 4, B, cudaMemcpyDeviceToDevice, c->stream));

@@ -232,6 +232,72 @@ __global__ void act_blocks_kernel(const float *__restrict__ act_all, int lda, in
   }
 }
 
+// RMSNorm and the activation blocks in one kernel (steps a2 / a6 / a9, first half, on the tcgen05
+// path): block g < n_groups takes 4 rows (a sweep of the GEMM is n_cols / 2 rows, padded with zero
+// rows), sums their squares, and writes their hi and lo columns of every k block; the blocks
+// behind them clear the buffer the GEMM accumulates into.  x [rows][ldx] fp32; K values per row.
+constexpr int NAB_ROWS = 4;
+__global__ void __launch_bounds__(256) norm_act_blocks_kernel(const float *__restrict__ x, int ldx, const float *__restrict__ w,
+                                                              float eps, int rows_all, int K, int n_cols,
+                                                              uint4 *__restrict__ blocks_all, int n_groups,
+                                                              float4 *__restrict__ zero, size_t zero_n4) {
+  // the GEMM that follows may be scheduled already: it waits for this grid before it reads the blocks
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if ((int)blockIdx.x >= n_groups) {
+    const size_t n_z = gridDim.x - n_groups;
+    for (size_t i = (size_t)(blockIdx.x - n_groups) * blockDim.x + threadIdx.x; i < zero_n4; i += n_z * blockDim.x)
+      zero[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    return;
+  }
+  const int sweep_rows = n_cols / 2, groups_per_sweep = sweep_rows / NAB_ROWS;
+  const int sweep = blockIdx.x / groups_per_sweep, m_in0 = (blockIdx.x % groups_per_sweep) * NAB_ROWS;
+  const int m0 = sweep * (TG_MAX_COLS / 2) + m_in0;                 // first row of the group (sweeps are 128 rows apart)
+  const int n_kb = K / TG_KB;
+  uint4 *blocks = blocks_all + (size_t)sweep * n_kb * (n_cols * 8);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __shared__ float part[8], inv[NAB_ROWS];
+  {
+    // two warps per row
+    const int r = warp >> 1, m = m0 + r;
+    float ss = 0.f;
+    if (m < rows_all) {
+      const float4 *xr = reinterpret_cast<const float4 *>(x + (size_t)m * ldx);
+      for (int k4 = (warp & 1) * 32 + lane; k4 < K / 4; k4 += 64) {
+        const float4 v = xr[k4];
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      }
+    }
+    ss = warp_sum(ss);
+    if (lane == 0) part[warp] = ss;
+  }
+  __syncthreads();
+  if (threadIdx.x < NAB_ROWS) inv[threadIdx.x] = rsqrtf((part[2 * threadIdx.x] + part[2 * threadIdx.x + 1]) / (float)K + eps);
+  __syncthreads();
+  // unit = (k block, k chunk of 8, row of the group): this thread writes the row's hi and lo columns
+  const int total = n_kb * 8 * NAB_ROWS;
+  for (int u = threadIdx.x; u < total; u += blockDim.x) {
+    const int r = u % NAB_ROWS, c = (u / NAB_ROWS) % 8, kb = u / (NAB_ROWS * 8);
+    const int m = m0 + r, k = kb * TG_KB + c * 8;
+    uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
+    if (m < rows_all) {
+      const float4 a = *reinterpret_cast<const float4 *>(x + (size_t)m * ldx + k);
+      const float4 b = *reinterpret_cast<const float4 *>(x + (size_t)m * ldx + k + 4);
+      const float4 wa = __ldg(reinterpret_cast<const float4 *>(w + k)), wb = __ldg(reinterpret_cast<const float4 *>(w + k + 4));
+      const float s = inv[r];
+      const float f[8] = {a.x * s * wa.x, a.y * s * wa.y, a.z * s * wa.z, a.w * s * wa.w,
+                          b.x * s * wb.x, b.y * s * wb.y, b.z * s * wb.z, b.w * s * wb.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        hi[j] = pack_bf16x2(f[2 * j], f[2 * j + 1]);
+        lo[j] = pack_bf16x2(f[2 * j] - __uint_as_float(hi[j] << 16), f[2 * j + 1] - __uint_as_float(hi[j] & 0xffff0000u));
+      }
+    }
+    uint4 *dst = blocks + ((size_t)kb * 8 + c) * n_cols + 2 * (m_in0 + r);
+    dst[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    dst[1] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  }
+}
+
 // Weights [N][K] bf16 row-major (rows [row0, row0 + N_src) of the fused matrix) -> 16 KiB blocks.
 __global__ void pack_umma_kernel(const __nv_bfloat16 *__restrict__ src, int N_src, int K, int row0, int n_kb,
                                  uint4 *__restrict__ dst) {
