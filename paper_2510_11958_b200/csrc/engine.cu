@@ -262,7 +262,7 @@ dmtd_status launch_gemv_nt(dmtd_ctx *c, const PackedMat &W, const float *act, in
 // With `norm_w` the activations are RMSNorm(act rows) * norm_w, computed while the blocks are written, and
 // the output rows are cleared first (the projections after a norm write a fresh buffer).
 dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, int lda, int M, float *out, int ldo,
-                             int gate_up_I = 0, const float *norm_w = nullptr) {
+                             int gate_up_I = 0, const float *norm_w = nullptr, int merge_nsplit = 0) {
   const int SET = TG_MAX_COLS / 2;                       // rows per sweep
   for (int m0 = 0; m0 < M; m0 += TG_MAX_SWEEPS * SET) {
     GemmTcParams P{};
@@ -285,11 +285,21 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
     if (P.n_sweeps == 1 && W.n_tiles > c->n_sms * per_sm_of(TG_STAGES) && W.n_tiles <= c->n_sms * per_sm_of(2)) P.stages = 2;
     const int slots = c->n_sms * per_sm_of(P.stages);
     P.ksplit = std::max(1, std::min(W.n_kb, slots / (W.n_tiles * P.n_sweeps)));
-    if (norm_w) {
+    if (merge_nsplit > 0) {
+      // `act` is unused: the activations are the attention's key slices, merged on the way
+      const int n_groups = P.n_sweeps * (P.n_cols / 2 / NAB_ROWS);
+      const int ky = std::max(1, std::min(W.n_kb, 4 * c->n_sms / std::max(1, n_groups)));
+      merge_act_blocks_kernel<<<dim3(n_groups, ky), 256, 0, c->stream>>>(
+          c->part_o + (size_t)m0 * c->s.n_q_heads * merge_nsplit * c->s.head_dim,
+          c->part_ml + (size_t)m0 * c->s.n_q_heads * merge_nsplit * 2, merge_nsplit, c->s.n_q_heads, c->s.head_dim, P.rows, P.n_cols,
+          c->act_blocks);
+      LAUNCH_OK(c, "merge_act_blocks_kernel");
+    } else if (norm_w) {
       const int n_groups = P.n_sweeps * (P.n_cols / 2 / NAB_ROWS);
       const size_t zero_n4 = (size_t)P.rows * ldo / 4;                  // ldo is a multiple of 4 (checked by the caller)
       const int n_zero = (int)std::min<size_t>((zero_n4 + 1023) / 1024, 2 * c->n_sms);
-      norm_act_blocks_kernel<<<n_groups + n_zero, 256, 0, c->stream>>>(
+      const int ky = std::max(1, std::min(W.n_kb, 4 * c->n_sms / std::max(1, n_groups)));
+      norm_act_blocks_kernel<<<dim3(n_groups + (n_zero + ky - 1) / ky, ky), 256, 0, c->stream>>>(
           act + (size_t)m0 * lda, lda, norm_w, c->s.rms_eps, P.rows, W.K, P.n_cols, c->act_blocks, n_groups,
           reinterpret_cast<float4 *>(out + (size_t)m0 * ldo), zero_n4);
       LAUNCH_OK(c, "norm_act_blocks_kernel");
@@ -330,7 +340,7 @@ dmtd_status launch_gemv(dmtd_ctx *c, const PackedMat &W, const UmmaMat &U, const
 }
 
 template <int D, typename KVT>
-dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit) {
+dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit, bool merge) {
   const dmtd_model_shape &s = c->s;
   int M = B * R, heads = s.n_q_heads + 2 * s.n_kv_heads, G = s.n_q_heads / s.n_kv_heads;
   KVT *kc = static_cast<KVT *>(c->kc) + (size_t)layer * c->kv_layer_elems;
@@ -358,6 +368,7 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
       nsplit);
   }
   LAUNCH_OK(c, "attn_partial_kernel");
+  if (!merge) return DMTD_OK;               // the O projection's activation-block kernel merges the slices
   int n_rh = M * s.n_q_heads;
   attn_merge_kernel<D><<<(n_rh + 3) / 4, 128, 0, c->stream>>>(c->part_o, c->part_ml, nsplit, n_rh, s.n_q_heads,
                                                              c->act, c->lda);
@@ -365,15 +376,15 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
   return DMTD_OK;
 }
 
-dmtd_status launch_attention(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit) {
+dmtd_status launch_attention(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit, bool merge = true) {
   const int kv = c->s.kv_dtype;
   if (c->s.head_dim == 128)
-    return kv == DMTD_BF16 ? launch_attention_t<128, __nv_bfloat16>(c, layer, B, R, pos0, nsplit)
-         : kv == DMTD_F16 ? launch_attention_t<128, __half>(c, layer, B, R, pos0, nsplit)
-                          : launch_attention_t<128, float>(c, layer, B, R, pos0, nsplit);
-  return kv == DMTD_BF16 ? launch_attention_t<64, __nv_bfloat16>(c, layer, B, R, pos0, nsplit)
-       : kv == DMTD_F16 ? launch_attention_t<64, __half>(c, layer, B, R, pos0, nsplit)
-                        : launch_attention_t<64, float>(c, layer, B, R, pos0, nsplit);
+    return kv == DMTD_BF16 ? launch_attention_t<128, __nv_bfloat16>(c, layer, B, R, pos0, nsplit, merge)
+         : kv == DMTD_F16 ? launch_attention_t<128, __half>(c, layer, B, R, pos0, nsplit, merge)
+                          : launch_attention_t<128, float>(c, layer, B, R, pos0, nsplit, merge);
+  return kv == DMTD_BF16 ? launch_attention_t<64, __nv_bfloat16>(c, layer, B, R, pos0, nsplit, merge)
+       : kv == DMTD_F16 ? launch_attention_t<64, __half>(c, layer, B, R, pos0, nsplit, merge)
+                        : launch_attention_t<64, float>(c, layer, B, R, pos0, nsplit, merge);
 }
 
 dmtd_status launch_rope_table(dmtd_ctx *c, const int *pos0, int R) {
@@ -413,9 +424,12 @@ dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos
     LAUNCH_OK(c, "prep_norm_kernel");
     TRY(launch_gemv(c, lw.qkv, lw.qkv_u, c->act, c->lda, M, c->qkv, c->ldqkv));
   }
-  TRY(launch_attention(c, l, B, R, pos0, splits_for(c, pos_end)));
+  const int nsplit = splits_for(c, pos_end);
+  const bool fuse_merge = tc && NAB_ROWS * s.n_q_heads * nsplit <= MAB_MAX_SLOTS;
+  TRY(launch_attention(c, l, B, R, pos0, nsplit, !fuse_merge));
   (void)QD;
-  TRY(launch_gemv(c, lw.o, lw.o_u, c->act, c->lda, M, x, H));
+  if (fuse_merge) TRY(launch_gemm_tc05(c, lw.o_u, nullptr, 0, M, x, H, 0, nullptr, nsplit));
+  else TRY(launch_gemv(c, lw.o, lw.o_u, c->act, c->lda, M, x, H));
   if (tc) {
     TRY(launch_gemm_tc05(c, lw.gu_u, x, H, M, c->gu, c->ldgu, 0, lw.w_post));
   } else {

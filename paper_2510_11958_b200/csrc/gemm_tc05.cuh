@@ -244,8 +244,9 @@ __global__ void __launch_bounds__(256) norm_act_blocks_kernel(const float *__res
   // the GEMM that follows may be scheduled already: it waits for this grid before it reads the blocks
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if ((int)blockIdx.x >= n_groups) {
-    const size_t n_z = gridDim.x - n_groups;
-    for (size_t i = (size_t)(blockIdx.x - n_groups) * blockDim.x + threadIdx.x; i < zero_n4; i += n_z * blockDim.x)
+    const size_t n_z = (size_t)(gridDim.x - n_groups) * gridDim.y;
+    for (size_t i = ((size_t)(blockIdx.x - n_groups) * gridDim.y + blockIdx.y) * blockDim.x + threadIdx.x; i < zero_n4;
+         i += n_z * blockDim.x)
       zero[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     return;
   }
@@ -273,10 +274,12 @@ __global__ void __launch_bounds__(256) norm_act_blocks_kernel(const float *__res
   __syncthreads();
   if (threadIdx.x < NAB_ROWS) inv[threadIdx.x] = rsqrtf((part[2 * threadIdx.x] + part[2 * threadIdx.x + 1]) / (float)K + eps);
   __syncthreads();
-  // unit = (k block, k chunk of 8, row of the group): this thread writes the row's hi and lo columns
-  const int total = n_kb * 8 * NAB_ROWS;
+  // unit = (k block, k chunk of 8, row of the group): this thread writes the row's hi and lo columns;
+  // blockIdx.y takes a share of the k blocks (every share needs the whole row's sum of squares)
+  const int kb_lo = n_kb * blockIdx.y / gridDim.y, kb_hi = n_kb * (blockIdx.y + 1) / gridDim.y;
+  const int total = (kb_hi - kb_lo) * 8 * NAB_ROWS;
   for (int u = threadIdx.x; u < total; u += blockDim.x) {
-    const int r = u % NAB_ROWS, c = (u / NAB_ROWS) % 8, kb = u / (NAB_ROWS * 8);
+    const int r = u % NAB_ROWS, c = (u / NAB_ROWS) % 8, kb = kb_lo + u / (NAB_ROWS * 8);
     const int m = m0 + r, k = kb * TG_KB + c * 8;
     uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
     if (m < rows_all) {
@@ -286,6 +289,72 @@ __global__ void __launch_bounds__(256) norm_act_blocks_kernel(const float *__res
       const float s = inv[r];
       const float f[8] = {a.x * s * wa.x, a.y * s * wa.y, a.z * s * wa.z, a.w * s * wa.w,
                           b.x * s * wb.x, b.y * s * wb.y, b.z * s * wb.z, b.w * s * wb.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        hi[j] = pack_bf16x2(f[2 * j], f[2 * j + 1]);
+        lo[j] = pack_bf16x2(f[2 * j] - __uint_as_float(hi[j] << 16), f[2 * j + 1] - __uint_as_float(hi[j] & 0xffff0000u));
+      }
+    }
+    uint4 *dst = blocks + ((size_t)kb * 8 + c) * n_cols + 2 * (m_in0 + r);
+    dst[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    dst[1] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  }
+}
+
+// The merge of the attention's key slices (step a4, second half) and the activation blocks of the O
+// projection in one kernel: block g takes 4 rows, works out the weight of every (row, head, slice)
+// from the slices' running max and sum, and writes the merged head outputs as hi and lo columns.
+// part_o [(row * nq + head) * nsplit + slice][D], part_ml the same with (max, sum); K = nq * D.
+constexpr int MAB_MAX_SLOTS = 2048;            // (rows of a group) x heads x slices the weights of a group may take
+__global__ void __launch_bounds__(256) merge_act_blocks_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
+                                                               int nsplit, int nq, int D, int rows_all, int n_cols,
+                                                               uint4 *__restrict__ blocks_all) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int K = nq * D, n_kb = K / TG_KB;
+  const int sweep_rows = n_cols / 2, groups_per_sweep = sweep_rows / NAB_ROWS;
+  const int sweep = blockIdx.x / groups_per_sweep, m_in0 = (blockIdx.x % groups_per_sweep) * NAB_ROWS;
+  const int m0 = sweep * (TG_MAX_COLS / 2) + m_in0;
+  uint4 *blocks = blocks_all + (size_t)sweep * n_kb * (n_cols * 8);
+  __shared__ float wgt[MAB_MAX_SLOTS];
+  // weights: one thread per (row, head)
+  for (int i = threadIdx.x; i < NAB_ROWS * nq; i += blockDim.x) {
+    const int r = i / nq, h = i % nq, m = m0 + r;
+    float *wr = wgt + (size_t)i * nsplit;
+    if (m >= rows_all) { for (int s = 0; s < nsplit; ++s) wr[s] = 0.f; continue; }
+    const float *ml = part_ml + ((size_t)m * nq + h) * nsplit * 2;
+    float mx = -INFINITY;
+    for (int s = 0; s < nsplit; ++s)
+      if (ml[2 * s + 1] > 0.f) mx = fmaxf(mx, ml[2 * s]);
+    float l = 0.f;
+    for (int s = 0; s < nsplit; ++s) {
+      const float ls = ml[2 * s + 1];
+      const float f = ls > 0.f ? __expf(ml[2 * s] - mx) : 0.f;
+      wr[s] = f;
+      l += ls * f;
+    }
+    const float inv = 1.f / l;
+    for (int s = 0; s < nsplit; ++s) wr[s] *= inv;
+  }
+  __syncthreads();
+  const int kb_lo = n_kb * blockIdx.y / gridDim.y, kb_hi = n_kb * (blockIdx.y + 1) / gridDim.y;   // this block's share of the k blocks
+  const int total = (kb_hi - kb_lo) * 8 * NAB_ROWS;
+  for (int u = threadIdx.x; u < total; u += blockDim.x) {
+    const int r = u % NAB_ROWS, c = (u / NAB_ROWS) % 8, kb = kb_lo + u / (NAB_ROWS * 8);
+    const int m = m0 + r, k = kb * TG_KB + c * 8, h = k / D, d0 = k - h * D;
+    uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
+    if (m < rows_all) {
+      float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      const float *wr = wgt + (size_t)(r * nq + h) * nsplit;
+      const float *po = part_o + ((size_t)m * nq + h) * nsplit * D + d0;
+      for (int s = 0; s < nsplit; ++s) {
+        const float ws = wr[s];
+        if (ws != 0.f) {                                   // empty slices hold nothing that may be read
+          const float4 a = *reinterpret_cast<const float4 *>(po + (size_t)s * D);
+          const float4 b = *reinterpret_cast<const float4 *>(po + (size_t)s * D + 4);
+          f[0] += ws * a.x; f[1] += ws * a.y; f[2] += ws * a.z; f[3] += ws * a.w;
+          f[4] += ws * b.x; f[5] += ws * b.y; f[6] += ws * b.z; f[7] += ws * b.w;
+        }
+      }
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         hi[j] = pack_bf16x2(f[2 * j], f[2 * j + 1]);
