@@ -103,6 +103,146 @@ __device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *
       }
 }
 
+// The same tile with the operands swapped, for at most 8 query rows (one new position of up to 8
+// query heads per KV head: every decode pass of a batch).  With the query rows on the M axis an
+// m16 tile is three quarters padding at 4 rows, and mma.sync issue, not HBM, bounds the kernel
+// (128 MMAs per 64-key tile).  Here the 16 keys of the warp are the M axis of S^T = K Q^T and the
+// 128 output dimensions the M axis of O^T = V^T P^T, the query rows the 8 columns: 64 MMAs per tile.
+// Accumulator layout: thread (g, t) holds columns (query rows) 2t, 2t + 1 of rows g and g + 8.
+struct AttnAccS {
+  float m_run[2], l_part[2];       // per query row 2t, 2t + 1: running max, this lane's share of the running sum
+  float o[8][4];                   // O^T: m-tile dt = dimensions 16 dt .. + 15
+};
+
+template <class Op>
+__device__ __forceinline__ void attn_tile_compute_swap(AttnAccS &A, unsigned char *sc, const uint4 (&qh)[4], int n_t, int tile0,
+                                                       int j0, int row_pos0, int G, int k_off, int v_off) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const uint32_t kh_tile = smem_u32(sc + k_off);
+  const uint32_t vh_tile = smem_u32(sc + v_off);
+  if (warp * 16 >= n_t) return;
+  // S^T = K Q^T: A = the warp's 16 key rows (the same permutation of the 32 dimensions of a k block
+  // on both operands: a lane's 16 bytes are dimensions 8t .. 8t + 7), B = the query rows
+  float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int kb = 0; kb < 4; ++kb) {
+    const uint32_t off = (warp * 16 + g) * PK_KROW + kb * 64 + t * 16;
+    const uint4 K0 = lds128(kh_tile + off), K1 = lds128(kh_tile + off + 8 * PK_KROW);
+    Op::mma(c, K0.x, K1.x, K0.y, K1.y, qh[kb].x, qh[kb].y);
+    Op::mma(c, K0.z, K1.z, K0.w, K1.w, qh[kb].z, qh[kb].w);
+  }
+  // mask: rows are keys g, g + 8 of the warp's 16, columns query rows 2t, 2t + 1
+  float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const int kl = warp * 16 + g + (e >> 1) * 8, q = 2 * t + (e & 1);
+    const bool ok = kl < n_t && j0 + tile0 + kl <= row_pos0 + q / G;
+    c[e] = ok ? c[e] : -INFINITY;
+    mx[e & 1] = fmaxf(mx[e & 1], c[e]);
+  }
+  float corr[2];
+#pragma unroll
+  for (int hq = 0; hq < 2; ++hq) {
+    // over the warp's 16 keys: the 8 lanes that share t
+    mx[hq] = fmaxf(mx[hq], __shfl_xor_sync(0xffffffffu, mx[hq], 4));
+    mx[hq] = fmaxf(mx[hq], __shfl_xor_sync(0xffffffffu, mx[hq], 8));
+    mx[hq] = fmaxf(mx[hq], __shfl_xor_sync(0xffffffffu, mx[hq], 16));
+    const float m_new = fmaxf(A.m_run[hq], mx[hq]);
+    corr[hq] = m_new > -INFINITY ? __expf(A.m_run[hq] - m_new) : 1.f;
+    A.m_run[hq] = m_new;
+  }
+  float psum[2] = {0.f, 0.f};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float p = c[e] > -INFINITY ? __expf(c[e] - A.m_run[e & 1]) : 0.f;
+    c[e] = p;
+    psum[e & 1] += p;
+  }
+  A.l_part[0] = A.l_part[0] * corr[0] + psum[0];
+  A.l_part[1] = A.l_part[1] * corr[1] + psum[1];
+  // P^T as the B operand (k = key, n = query row): lane (g, t) needs keys 2t, 2t + 1 (and + 8) of query
+  // row g; they sit in lanes (2t, g / 2) and (2t + 1, g / 2), element g & 1 of each pair
+  const uint32_t x = Op::pack2(c[0], c[1]), y = Op::pack2(c[2], c[3]);
+  const int src_a = (2 * t) * 4 + (g >> 1), src_b = (2 * t + 1) * 4 + (g >> 1);
+  const uint32_t xa = __shfl_sync(0xffffffffu, x, src_a), xb = __shfl_sync(0xffffffffu, x, src_b);
+  const uint32_t ya = __shfl_sync(0xffffffffu, y, src_a), yb = __shfl_sync(0xffffffffu, y, src_b);
+  const uint32_t sel = (g & 1) ? 0x7632u : 0x5410u;       // high or low halves of the two words
+  const uint32_t b0 = __byte_perm(xa, xb, sel), b1 = __byte_perm(ya, yb, sel);
+  // O^T += V^T P^T: A = V^T (m = dimension, k = key) through ldmatrix.trans of the key rows
+  const int mi = lane >> 3, rr = lane & 7;
+  const uint32_t v_row = (warp * 16 + (mi >> 1) * 8 + rr) * PK_VROW + (mi & 1) * 16;
+#pragma unroll
+  for (int dt = 0; dt < 8; ++dt) {
+    uint32_t a0, a1, a2, a3;
+    ldmatrix_x4_trans(vh_tile + v_row + dt * 32, a0, a1, a2, a3);
+    A.o[dt][0] *= corr[0]; A.o[dt][1] *= corr[1]; A.o[dt][2] *= corr[0]; A.o[dt][3] *= corr[1];
+    Op::mma(A.o[dt], a0, a1, a2, a3, b0, b1);
+  }
+}
+
+// Combine of the swapped layout: the warps' partial outputs O^T go to shared memory as [warp][query
+// row][dimension], then as in attn_combine_store_w.
+__device__ __forceinline__ void attn_combine_store_swap(AttnAccS &A, unsigned char *sc, int nQ, int G, int row0, int head0,
+                                                        int nq, int slot_stride, int split, float *part_o, float *part_ml) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  float *const o_s = reinterpret_cast<float *>(sc + PK_AT_OS);
+  float *const red_m = reinterpret_cast<float *>(sc + PK_AT_RED);
+  float *const red_l = red_m + PK_WARPS * PK_QR;
+  pk_sync();                                            // tiles consumed: their space becomes o_s
+#pragma unroll
+  for (int hq = 0; hq < 2; ++hq) {
+    float l = A.l_part[hq];
+    l += __shfl_xor_sync(0xffffffffu, l, 4);
+    l += __shfl_xor_sync(0xffffffffu, l, 8);
+    l += __shfl_xor_sync(0xffffffffu, l, 16);
+    if (g == 0) { red_m[warp * PK_QR + 2 * t + hq] = A.m_run[hq]; red_l[warp * PK_QR + 2 * t + hq] = l; }
+  }
+  if (warp < 4) {
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int q = 2 * t + (e & 1), d = dt * 16 + g + (e >> 1) * 8;
+        if (q < nQ) o_s[(warp * PK_QR + q) * PK_OROW + d] = A.o[dt][e];
+      }
+    }
+  }
+  pk_sync();
+  // warps 4 - 7 took no keys: their running max stays -inf and their share is skipped
+  if ((int)threadIdx.x < nQ) {
+    const int qi = threadIdx.x;
+    float m = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) m = fmaxf(m, red_m[w * PK_QR + qi]);
+    float l = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float mw = red_m[w * PK_QR + qi];
+      const float f = mw > -INFINITY ? __expf(mw - m) : 0.f;
+      l += red_l[w * PK_QR + qi] * f;
+      red_l[w * PK_QR + qi] = f;
+    }
+    const size_t slot = ((size_t)(row0 + qi / G) * nq + head0 + qi % G) * slot_stride + split;
+    part_ml[slot * 2] = m;
+    part_ml[slot * 2 + 1] = l;
+  }
+  pk_sync();
+  for (int idx = threadIdx.x; idx < nQ * (PK_D / 4); idx += PK_THREADS) {
+    const int qi = idx / (PK_D / 4), d4 = idx % (PK_D / 4);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float f = red_l[w * PK_QR + qi];
+      if (f != 0.f) {
+        const float4 v = *reinterpret_cast<const float4 *>(o_s + (w * PK_QR + qi) * PK_OROW + d4 * 4);
+        acc.x += v.x * f; acc.y += v.y * f; acc.z += v.z * f; acc.w += v.w * f;
+      }
+    }
+    const size_t slot = ((size_t)(row0 + qi / G) * nq + head0 + qi % G) * slot_stride + split;
+    *reinterpret_cast<float4 *>(part_o + slot * PK_D + d4 * 4) = acc;
+  }
+}
+
 // Combine the warps of the block into the slice's partial result: unnormalised output with its
 // max and sum, written to part_o / part_ml at slot (row0 + q / G, head0 + q % G, split), where a
 // (row, head) owns `slot_stride` consecutive slots.
@@ -208,12 +348,6 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
     }
   }
   const size_t head_off = ((size_t)b * nkv + kvh) * max_seq * PK_D;
-  AttnAccW A;
-  A.m_run[0] = A.m_run[1] = -INFINITY;
-  A.l_part[0] = A.l_part[1] = 0.f;
-#pragma unroll
-  for (int dt = 0; dt < 16; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
-  uint4 qh[4][2];
   const int n_keys = j1 - j0;
   // bf16 cache: two tile buffers (the lo-part areas are free here), tile i+1 in flight while
   // tile i is multiplied
@@ -234,6 +368,39 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
   };
   fetch(0, 0);
   int buf = 0;
+  if (nQ <= 8) {
+    // at most 8 query rows (a decode pass): keys and output dimensions on the M axis of the MMAs
+    AttnAccS A;
+    A.m_run[0] = A.m_run[1] = -INFINITY;
+    A.l_part[0] = A.l_part[1] = 0.f;
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
+    uint4 qs[4];
+    for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK, buf ^= 1) {
+      const int n_t = min(PK_TK, n_keys - tile0);
+      if (tile0 + PK_TK < n_keys) {
+        fetch(tile0 + PK_TK, buf ^ 1);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+      } else {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+      }
+      __syncthreads();                                  // tile (and, the first time, Q) visible to all
+      if (tile0 == 0) {
+#pragma unroll
+        for (int kbk = 0; kbk < 4; ++kbk) qs[kbk] = lds128(qh_tile + g * PK_QROW + kbk * 64 + t * 16);
+      }
+      attn_tile_compute_swap<Op>(A, sc, qs, n_t, tile0, j0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH, buf ? PK_AT_VL : PK_AT_VH);
+      __syncthreads();                                  // done with this buffer before it is refilled
+    }
+    attn_combine_store_swap(A, sc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
+    return;
+  }
+  AttnAccW A;
+  A.m_run[0] = A.m_run[1] = -INFINITY;
+  A.l_part[0] = A.l_part[1] = 0.f;
+#pragma unroll
+  for (int dt = 0; dt < 16; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
+  uint4 qh[4][2];
   for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK, buf ^= 1) {
     const int n_t = min(PK_TK, n_keys - tile0);
     if (tile0 + PK_TK < n_keys) {
