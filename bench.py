@@ -391,6 +391,7 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="qwen3_4b_b1")
     ap.add_argument("--tau", type=int, default=None)
+    ap.add_argument("--kv-dtype", default=None, choices=["f32", "bf16", "f16"], help="KV cache type (default: the workload's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-tau1", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -406,6 +407,9 @@ def main():
         args.steps = 84 if args.impl == "native" else 10
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
     wl = WORKLOADS[args.workload]
+    if args.kv_dtype:
+        import dataclasses
+        wl = dataclasses.replace(wl, kv_dtype=args.kv_dtype)
     args.tau = args.tau or wl.tau
     shape = SHAPES[wl.shape]
     if args.gpus > 1 and "RANK" not in os.environ and args.impl == "native":

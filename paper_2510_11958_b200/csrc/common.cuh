@@ -121,6 +121,7 @@ __device__ __forceinline__ void mma_f16_16816(float (&d)[4], uint32_t a0, uint32
 struct OpBf16 {
   using T = __nv_bfloat16;
   static __device__ __forceinline__ T from_float(float v) { return __float2bfloat16_rn(v); }
+  static __device__ __forceinline__ float to_float(T v) { return __bfloat162float(v); }
   static __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
@@ -131,6 +132,7 @@ struct OpBf16 {
 struct OpF16 {
   using T = __half;
   static __device__ __forceinline__ T from_float(float v) { return __float2half_rn(v); }
+  static __device__ __forceinline__ float to_float(T v) { return __half2float(v); }
   static __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     __half2 v = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);

@@ -518,7 +518,7 @@ bool fused_matrix_ok(const PackedMat &m, int grid) {
 dmtd_status setup_fused(dmtd_ctx *c) {
   const dmtd_model_shape &s = c->s;
   c->fused_ok = false;
-  if (!is_bf16(c) || s.head_dim != PK_D || s.n_layers > PK_MAX_LAYERS || s.kv_dtype == DMTD_F16) return DMTD_OK;
+  if (!is_bf16(c) || s.head_dim != PK_D || s.n_layers > PK_MAX_LAYERS) return DMTD_OK;
   if (s.n_q_heads / s.n_kv_heads > PK_MAX_GROUP || s.hidden % 8 || s.hidden > PK_XS_FLOATS) return DMTD_OK;
   int coop = 0;
   CUDA_TRY(c, cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
@@ -580,7 +580,7 @@ dmtd_status enqueue_pass_fused(dmtd_ctx *c, int kind, int R_lower, bool write_to
   P.R_lo = (kind == 1 && lo > 0) ? R_lower : 1; P.B = c->B;
   P.H = s.hidden; P.I = s.intermediate; P.nq = s.n_q_heads; P.nkv = s.n_kv_heads; P.vocab = s.vocab;
   P.max_seq = c->max_seq; P.ldl = c->ldl; P.eps = s.rms_eps;
-  P.kind = kind; P.write_token = write_token ? 1 : 0; P.kv_f32 = s.kv_dtype == DMTD_F32 ? 1 : 0;
+  P.kind = kind; P.write_token = write_token ? 1 : 0; P.kv_f32 = s.kv_dtype == DMTD_F32 ? 1 : 0; P.kv_f16 = s.kv_dtype == DMTD_F16 ? 1 : 0;
   P.tokens = c->tokens; P.st = c->dstate;
   P.x_lo = c->x_lo; P.x_up = c->x_up; P.qkv = c->qkv; P.gu = c->gu; P.logits = c->logits;
   P.timing = c->pass_timing;

@@ -80,14 +80,16 @@ __device__ __forceinline__ void attn_plan_device(const PassParams &P, int pos0, 
 }
 
 // 8 values -> 16 bytes of bf16.
+template <class Op>
 __device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
-  return make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+  return make_uint4(Op::pack2(f[0], f[1]), Op::pack2(f[2], f[3]), Op::pack2(f[4], f[5]), Op::pack2(f[6], f[7]));
 }
 
 // Step a3 for one (sequence, kv head): one warp per head vector of the pass's rows (staged in
 // shared memory as q heads | k | v per row).  Query rows go to the Q tile (scaled by 1/sqrt(d));
 // K and V rows go to the new-row area as floats already rounded to the cache's type and, from
 // the block that owns slice 0, into the cache.
+template <class Op>
 __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLayer &Ly, unsigned char *sc, int b, int kvh,
                                               int R, int pos0, bool write_cache) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -125,20 +127,19 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
       }
     }
     if (kind == 0) {
-      __nv_bfloat16 *qh = reinterpret_cast<__nv_bfloat16 *>(sc + PK_PA_QH + task * PK_QROW);
+      typename Op::T *qh = reinterpret_cast<typename Op::T *>(sc + PK_PA_QH + task * PK_QROW);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const __nv_bfloat16 h = __float2bfloat16_rn(v[j]);
-        qh[lane + 32 * j] = h;
+        qh[lane + 32 * j] = Op::from_float(v[j]);
       }
     } else {
       float *row = reinterpret_cast<float *>(sc + PK_PA_NEW) + ((kind == 2 ? PK_MAX_ROWS : 0) + r) * PK_D;
       const size_t at = (((size_t)b * P.nkv + kvh) * P.max_seq + pos) * PK_D;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const __nv_bfloat16 h = __float2bfloat16_rn(v[j]);
-        row[lane + 32 * j] = __bfloat162float(h);
-        if (write_cache) reinterpret_cast<__nv_bfloat16 *>(kind == 1 ? Ly.kc : Ly.vc)[at + lane + 32 * j] = h;
+        const typename Op::T h = Op::from_float(v[j]);
+        row[lane + 32 * j] = Op::to_float(h);
+        if (write_cache) reinterpret_cast<typename Op::T *>(kind == 1 ? Ly.kc : Ly.vc)[at + lane + 32 * j] = h;
       }
     }
   }
@@ -158,6 +159,7 @@ struct AttnAcc {
 // k_off / v_off: where the tile's K and V (hi parts) sit in the scratch.  The Q fragments are
 // read from shared memory in a rolled loop: the code stays short (instruction fetch, not
 // arithmetic, bounds a stage that runs once per layer).
+template <class Op>
 __device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc, int n_t, int tile0, int n_cached, int j0,
                                                   int pos_new, int row_pos0, int G, int k_off = PK_PA_KH,
                                                   int v_off = PK_PA_VH) {
@@ -181,8 +183,8 @@ __device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc,
     for (int nt = 0; nt < 2; ++nt) {
       const uint32_t off = (kg * 16 + nt * 8 + g) * PK_KROW + kb * 64 + t * 16;
       const uint4 Kh = lds128(kh_tile + off);
-      mma_bf16_16816(c[nt], q0.x, q1.x, q0.y, q1.y, Kh.x, Kh.y);
-      mma_bf16_16816(c[nt], q0.z, q1.z, q0.w, q1.w, Kh.z, Kh.w);
+      Op::mma(c[nt], q0.x, q1.x, q0.y, q1.y, Kh.x, Kh.y);
+      Op::mma(c[nt], q0.z, q1.z, q0.w, q1.w, Kh.z, Kh.w);
     }
   }
   // causal / range mask: lane holds rows g (e = 0, 1) and g + 8 (e = 2, 3), keys 2t, 2t + 1 of each n-tile
@@ -224,7 +226,7 @@ __device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc,
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const float p0 = c[i >> 1][(i & 1) * 2], p1 = c[i >> 1][(i & 1) * 2 + 1];
-    ah[i] = pack_bf16x2(p0, p1);
+    ah[i] = Op::pack2(p0, p1);
   }
   const int mi = lane >> 3, rr = lane & 7;
   const uint32_t v_row = (kg * 16 + (mi & 1) * 8 + rr) * PK_VROW + (mi >> 1) * 16 + dh * 128;
@@ -234,8 +236,8 @@ __device__ __forceinline__ void attn_tile_compute(AttnAcc &A, unsigned char *sc,
     ldmatrix_x4_trans(vh_tile + v_row + d2 * 32, b0, b1, b2, b3);
     o[2 * d2][0] *= corr[0]; o[2 * d2][1] *= corr[0]; o[2 * d2][2] *= corr[1]; o[2 * d2][3] *= corr[1];
     o[2 * d2 + 1][0] *= corr[0]; o[2 * d2 + 1][1] *= corr[0]; o[2 * d2 + 1][2] *= corr[1]; o[2 * d2 + 1][3] *= corr[1];
-    mma_bf16_16816(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
-    mma_bf16_16816(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+    Op::mma(o[2 * d2], ah[0], ah[1], ah[2], ah[3], b0, b1);
+    Op::mma(o[2 * d2 + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
   }
 }
 
@@ -307,6 +309,7 @@ __device__ __forceinline__ void attn_combine_store(AttnAcc &A, unsigned char *sc
 // shared memory, each warp taking 16 keys of a 64-key tile with its own running max and sum.
 // The slice's unnormalised partial output goes to global memory with its max and sum; the
 // prologue of the O projection merges the slices.
+template <class Op>
 __device__ __noinline__ void attention_stage(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
   const PassShared S = pass_shared();
   const int G = P.nq / P.nkv, nQ = R * G;
@@ -321,7 +324,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
   const uint32_t qh_tile = smem_u32(sc + PK_PA_QH);
   // a 16-byte part (8 values) of a tile row: parts 0..15 are K, 16..31 are V
   auto put_part = [&](int row, int part, const float (&f)[8]) {
-    const uint4 hi = pack8(f);
+    const uint4 hi = pack8<Op>(f);
     const uint32_t off = part < 16 ? row * PK_KROW + part * 16 : row * PK_VROW + (part - 16) * 16;
     sts128((part < 16 ? kh_tile : vh_tile) + off, hi);
   };
@@ -338,8 +341,8 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     auto fetch_cached = [&](int tile0) {
       const int n_c = min(PK_TK, n_cached - tile0);
       // bf16 cache: asynchronous copies, 16 bytes each
-      const __nv_bfloat16 *kb = reinterpret_cast<const __nv_bfloat16 *>(Ly.kc) + head_off;
-      const __nv_bfloat16 *vb = reinterpret_cast<const __nv_bfloat16 *>(Ly.vc) + head_off;
+      const typename Op::T *kb = reinterpret_cast<const typename Op::T *>(Ly.kc) + head_off;
+      const typename Op::T *vb = reinterpret_cast<const typename Op::T *>(Ly.vc) + head_off;
 #pragma unroll 1
       for (int c = threadIdx.x; c < n_c * 32; c += PK_THREADS) {
         const int row = c >> 5, part = c & 31;
@@ -371,7 +374,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     for (int i = threadIdx.x; i < 2 * PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(qh_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
     stage_wait(P, S);
     PK_SUBSTAMP(3);
-    attn_new_rows(P, Ly, sc, b, kvh, R, pos0, split == 0);
+    attn_new_rows<Op>(P, Ly, sc, b, kvh, R, pos0, split == 0);
     PK_SUBSTAMP(4);
 
     AttnAcc A;
@@ -402,7 +405,7 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
       cp_async_wait_all();
       pk_sync();
       PK_SUBSTAMP(10);
-      attn_tile_compute(A, sc, n_t, tile0, n_cached, j0, pos0, pos0, G);
+      attn_tile_compute<Op>(A, sc, n_t, tile0, n_cached, j0, pos0, pos0, G);
     }
     PK_SUBSTAMP(5);
     attn_combine_store(A, sc, nQ, G, b * R, kvh * G, P.nq, PK_NSPLIT_CAP, split, P.part_o, P.part_ml);

@@ -97,7 +97,8 @@ struct PassParams {
   int H, I, nq, nkv, vocab, max_seq, ldl;
   float eps;
   int kind;                               // 1 full pass, 2 decoding layers only (counter update)
-  int kv_f32;                             // the KV cache holds fp32 (else bf16)
+  int kv_f32;                             // the KV cache holds fp32 (else a 16-bit type)
+  int kv_f16;                             // ... fp16 (else bf16)
   int write_token;
   int *tokens;
   DevState *st;

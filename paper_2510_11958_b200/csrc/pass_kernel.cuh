@@ -258,7 +258,8 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
     } else if (ph == 1) {
       // a3 + a4: QK-norm, RoPE, KV append, attention over the key slices
       if (P.kv_f32) attention_stage_f32(P, Ly, R, pos0);
-      else attention_stage(P, Ly, R, pos0);
+      else if (P.kv_f16) attention_stage<OpF16>(P, Ly, R, pos0);
+      else attention_stage<OpBf16>(P, Ly, R, pos0);
     } else if (ph == 2) {
       // a4 merge of the key slices + a5: O projection into the residual rows
       grid_zero(P.gu, M_max * ldgu);

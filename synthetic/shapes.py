@@ -73,13 +73,13 @@ WORKLOADS = {
     # static length, fixed generation length); sizes follow the build's baseline configs.
     "tiny_b1": Workload("tiny_b1", "tiny", L_d=2, tau=3, batch=1, prompt_len=32, gen_len=24),
     # KV cache type: a bf16 cache alone moves the logits of the 36-layer model by more than the logit
-    # tolerance, so the workloads whose logits are held to it use fp32 (batch 1, where the cache is 1 % of
-    # the bytes) or fp16 (batch 32: half of fp32's bytes, tensor-core attention, within the tolerance at
-    # full depth); bf16 where the workload says so.
+    # tolerance, so the workloads whose logits are held to it use fp16 (half of fp32's bytes, tensor-core
+    # attention, 7e-3 on the logits at full depth; an fp32 cache gives 2e-4 and is what the remaining
+    # tests use); bf16 where the workload says so.
     "qwen3_4b_b1": Workload("qwen3_4b_b1", "qwen3_4b", L_d=8, tau=3, batch=1, prompt_len=512,
-                            gen_len=256, kv_dtype="f32"),
+                            gen_len=256, kv_dtype="f16"),
     "qwen3_4b_l4_b1": Workload("qwen3_4b_l4_b1", "qwen3_4b_l4", L_d=2, tau=3, batch=1, prompt_len=512,
-                               gen_len=64, kv_dtype="f32"),
+                               gen_len=64, kv_dtype="f16"),
     "qwen3_4b_b32": Workload("qwen3_4b_b32", "qwen3_4b", L_d=8, tau=3, batch=32, prompt_len=1024,
                              gen_len=512, kv_dtype="f16"),
     # the same batch on the 4-layer model: small enough to list every launch under a profiler

@@ -57,9 +57,10 @@ def _kv_views(eng, layer, B, nkv, max_seq, D):
 
 
 def test_config2_full_depth_prompt_512_teacher_forced(dmtd):
-    """Config 2 at its own sizes: 36 layers, full vocabulary, 512-token prompt, fp32 KV cache, the
-    persistent pass kernel on every decode pass.  97 tokens: the prefill's and 96 decode passes
-    (32 whole cycles), logits of every pass against the oracle."""
+    """Config 2 at its own sizes: 36 layers, full vocabulary, 512-token prompt, the persistent pass
+    kernel on every decode pass, with the fp16 KV cache the benchmark workload uses and with an fp32
+    one.  97 tokens: the prefill's and 96 decode passes (32 whole cycles), logits of every pass
+    against the oracle."""
     shape = SHAPES["qwen3_4b"]
     P, n_new, L_d, tau = 512, 97, 8, 3
     w = make_weights(shape, seed=0)
@@ -68,13 +69,15 @@ def test_config2_full_depth_prompt_512_teacher_forced(dmtd):
     ref_logits, ref_am, o = oracle_forced(shape, w, L_d, tau, prompts, forced)
     wc = to_cuda(w)
     del w
-    eng = dmtd.Dmtd(shape, wc, L_d=L_d, tau=tau, max_batch=1, max_seq=P + n_new + 1, kv_dtype="f32")
-    l0 = eng.launch_count()
-    got_logits, got_am = gpu_forced(eng, prompts, forced)
-    err, clear = check_logits(got_logits, ref_logits, got_am, ref_am)
-    assert eng.device_state() == o.state()
-    print(f"config 2, {n_new - 1} decode passes: max|dlogit|={err:.2e}, clear-margin steps {clear:.0%}, "
-          f"launches {eng.launch_count() - l0}")
+    for kv in ("f16", "f32"):
+        eng = dmtd.Dmtd(shape, wc, L_d=L_d, tau=tau, max_batch=1, max_seq=P + n_new + 1, kv_dtype=kv)
+        l0 = eng.launch_count()
+        got_logits, got_am = gpu_forced(eng, prompts, forced)
+        err, clear = check_logits(got_logits, ref_logits, got_am, ref_am)
+        assert eng.device_state() == o.state()
+        print(f"config 2, {n_new - 1} decode passes, {kv} cache: max|dlogit|={err:.2e}, clear-margin steps {clear:.0%}, "
+              f"launches {eng.launch_count() - l0}")
+        eng.close()
 
 
 def test_full_depth_bf16_kv_cache_measured_bound(dmtd):
@@ -91,7 +94,7 @@ def test_full_depth_bf16_kv_cache_measured_bound(dmtd):
     wc = to_cuda(w)
     del w
     seen = {}
-    for kv, fused in (("f32", 1), ("bf16", 1), ("bf16", 0), ("f16", 0)):
+    for kv, fused in (("f32", 1), ("bf16", 1), ("bf16", 0), ("f16", 0), ("f16", 1)):
         eng = dmtd.Dmtd(shape, wc, L_d=L_d, tau=tau, max_batch=1, max_seq=P + n_new + 1, kv_dtype=kv)
         eng.set_option("fused_pass", fused)
         got_logits, got_am = gpu_forced(eng, prompts, forced)
@@ -104,8 +107,9 @@ def test_full_depth_bf16_kv_cache_measured_bound(dmtd):
     assert seen[("f32", 1)] <= LOGIT_ATOL
     assert seen[("bf16", 1)] <= BF16_KV_FULL_DEPTH_BOUND
     assert seen[("bf16", 0)] <= BF16_KV_FULL_DEPTH_BOUND
-    # an fp16 cache (the batch-32 workload's: half of fp32's bytes, tensor-core attention) meets the tolerance
+    # an fp16 cache (the batch-1 and batch-32 workloads': half of fp32's bytes, tensor-core attention) meets the tolerance
     assert seen[("f16", 0)] <= LOGIT_ATOL
+    assert seen[("f16", 1)] <= LOGIT_ATOL
 
 
 @pytest.mark.parametrize("tau,kv", [(1, "f16"), (2, "f16"), (3, "f16"), (4, "f16"), (3, "f32")])

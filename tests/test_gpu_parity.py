@@ -275,6 +275,8 @@ FUSED_CASES = [
     ("b1_tau4_long_prompt_f32kv", 2, 4, 1, 1300, 9, "f32"),    # two key tiles per slice
     ("b1_tau3_long_prompt_bf16kv", 2, 3, 1, 1300, 7, "bf16"),
     ("b2_tau2_f32kv", 4, 2, 2, 9, 8, "f32"),
+    ("b1_tau3_f16kv", 2, 3, 1, 37, 13, "f16"),
+    ("b1_tau4_long_prompt_f16kv", 2, 4, 1, 1300, 9, "f16"),
 ]
 
 
