@@ -26,10 +26,12 @@ struct AttnAccW {
 // pos_new + i - n_cached); query row q may see positions up to row_pos0 + q / G.
 // k_off / v_off: where the tile's K and V (hi parts) sit in the scratch.
 template <class Op>
+// kg: which 16 keys of the tile this call takes (the decode kernel gives every warp its own group,
+// the prefill kernel walks all four with every warp).
 __device__ __forceinline__ void attn_tile_compute_w(AttnAccW &A, unsigned char *sc, const uint4 (&qh)[4][2], int n_t, int tile0,
                                                   int n_cached, int j0, int pos_new, int row_pos0, int G,
-                                                  int k_off = PK_AT_KH, int v_off = PK_AT_VH) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+                                                  int k_off, int v_off, int kg) {
+  const int warp = kg, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const uint32_t kh_tile = smem_u32(sc + k_off);
   const uint32_t vh_tile = smem_u32(sc + v_off);
   float (&m_run)[2] = A.m_run;
@@ -418,10 +420,109 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
       }
     }
     attn_tile_compute_w<Op>(A, sc, qh, n_t, tile0, 0x7fffffff, j0, 0, pos0 + r0, G, buf ? PK_AT_KL : PK_AT_KH,
-                             buf ? PK_AT_VL : PK_AT_VH);
+                             buf ? PK_AT_VL : PK_AT_VH, warp);
     __syncthreads();                                    // done with this buffer before it is refilled
   }
   attn_combine_store_w(A, sc, nQ, G, b * R + r0, kvh * G, nq, nsplit, split, part_o, part_ml);
+}
+
+// Causal attention of a chunk of R new positions per sequence (the prefill, Section 2.2: all prompt
+// rows through all layers) for a 16-bit cache, flash-attention style: a block takes 8 x (16 / G)
+// consecutive positions of one (sequence, kv head), every warp owns 16 query rows (16 / G positions
+// x G heads) with their running max, sum and output in registers, and all warps share the 64-key
+// tiles of K and V that stream through shared memory once per block.  No key slices and no merge:
+// the normalised rows go straight to out [B*R][ld].  (The decode kernel above, run over 4-position
+// row blocks, re-read the keys before every row block: the prefill was bound by L2, not by HBM.)
+constexpr int ATTN_PF_Q = PK_AT_QH;                                    // Q tiles [warp][16][PK_QROW] behind the two K / V buffers
+constexpr int ATTN_PF_SMEM = ATTN_PF_Q + PK_WARPS * PK_QR * PK_QROW;
+
+template <class Op>
+__global__ void __launch_bounds__(PK_THREADS, 2)
+attn_prefill_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ kc, const void *__restrict__ vc, int max_seq,
+                    int nq, int nkv, int R, const int *__restrict__ pos0_ptr, float *__restrict__ out, int ld) {
+  extern __shared__ __align__(1024) unsigned char sc[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int G = nq / nkv, PW = PK_QR / G, QB = PK_WARPS * PW;         // positions per warp and per block
+  const int kvh = blockIdx.y, b = blockIdx.z;
+  const int r0 = blockIdx.x * QB, r1 = min(R, r0 + QB);
+  const int pos0 = *pos0_ptr;
+  const int wr0 = r0 + warp * PW, wr1 = min(R, wr0 + PW);             // this warp's positions [wr0, wr1) of the chunk
+  // Q tile of the warp: row i = (position wr0 + i / G, head kvh * G + i % G), scaled by 1/sqrt(d); rows past the chunk zero
+  const float scale = rsqrtf((float)PK_D);
+  typename Op::T *qt = reinterpret_cast<typename Op::T *>(sc + ATTN_PF_Q + warp * PK_QR * PK_QROW);
+  for (int i = 0; i < PK_QR; ++i) {
+    const int r = wr0 + i / G;
+    const float *src = qkv + (size_t)(b * R + min(r, R - 1)) * ldq + (size_t)(kvh * G + i % G) * PK_D;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      qt[i * (PK_QROW / 2) + lane + 32 * j] = Op::from_float(r < R ? src[lane + 32 * j] * scale : 0.f);
+  }
+  __syncwarp();
+  uint4 qh[4][2];
+  const uint32_t q_u32 = smem_u32(qt);
+#pragma unroll
+  for (int kbk = 0; kbk < 4; ++kbk) {
+    qh[kbk][0] = lds128(q_u32 + g * PK_QROW + kbk * 64 + t * 16);
+    qh[kbk][1] = lds128(q_u32 + (g + 8) * PK_QROW + kbk * 64 + t * 16);
+  }
+  const size_t head_off = ((size_t)b * nkv + kvh) * max_seq * PK_D;
+  const typename Op::T *kb = reinterpret_cast<const typename Op::T *>(kc) + head_off;
+  const typename Op::T *vb = reinterpret_cast<const typename Op::T *>(vc) + head_off;
+  const int n_keys = pos0 + r1;                                       // the block's last position sees keys [0, pos0 + r1)
+  auto fetch = [&](int tile0, int buf) {
+    const int n_t = min(PK_TK, n_keys - tile0);
+    const uint32_t k_t = smem_u32(sc + (buf ? PK_AT_KL : PK_AT_KH)), v_t = smem_u32(sc + (buf ? PK_AT_VL : PK_AT_VH));
+    for (int c = threadIdx.x; c < n_t * 32; c += PK_THREADS) {
+      const int row = c >> 5, part = c & 31;
+      const uint32_t dst = part < 16 ? k_t + row * PK_KROW + part * 16 : v_t + row * PK_VROW + (part - 16) * 16;
+      cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(tile0 + row) * PK_D + (part & 15) * 8);
+    }
+    const int n16 = min(PK_TK, (n_t + 15) & ~15);
+    for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS)      // P = 0 times stale bits must stay 0
+      sts128(v_t + (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16, make_uint4(0u, 0u, 0u, 0u));
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  AttnAccW A;
+  A.m_run[0] = A.m_run[1] = -INFINITY;
+  A.l_part[0] = A.l_part[1] = 0.f;
+#pragma unroll
+  for (int dt = 0; dt < 16; ++dt) A.o[dt][0] = A.o[dt][1] = A.o[dt][2] = A.o[dt][3] = 0.f;
+  fetch(0, 0);
+  int buf = 0;
+  const int last_pos = pos0 + wr1 - 1;                                // the warp's last row sees keys up to here
+  for (int tile0 = 0; tile0 < n_keys; tile0 += PK_TK, buf ^= 1) {
+    const int n_t = min(PK_TK, n_keys - tile0);
+    if (tile0 + PK_TK < n_keys) {
+      fetch(tile0 + PK_TK, buf ^ 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();                                    // the tile is visible to all
+    if (wr0 < wr1) {
+#pragma unroll 1
+      for (int kg = 0; kg < 4; ++kg)
+        if (tile0 + kg * 16 <= last_pos)
+          attn_tile_compute_w<Op>(A, sc, qh, n_t, tile0, 0x7fffffff, 0, 0, pos0 + wr0, G, buf ? PK_AT_KL : PK_AT_KH,
+                                  buf ? PK_AT_VL : PK_AT_VH, kg);
+    }
+    __syncthreads();                                    // done with this buffer before it is refilled
+  }
+  // normalise and store: lane (g, t) holds rows g and g + 8, columns 8 dt + 2t, + 1
+#pragma unroll
+  for (int hr = 0; hr < 2; ++hr) {
+    float l = A.l_part[hr];
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    const int i = g + 8 * hr, r = wr0 + i / G;
+    if (r < wr1) {
+      const float inv = 1.f / l;
+      float *dst = out + (size_t)(b * R + r) * ld + (size_t)(kvh * G + i % G) * PK_D + 2 * t;
+#pragma unroll
+      for (int dt = 0; dt < 16; ++dt)
+        *reinterpret_cast<float2 *>(dst + dt * 8) = make_float2(A.o[dt][2 * hr] * inv, A.o[dt][2 * hr + 1] * inv);
+    }
+  }
 }
 
 // The same step for an fp32 cache in plain FMAs (three mma.sync per product would be needed for

@@ -340,7 +340,7 @@ dmtd_status launch_gemv(dmtd_ctx *c, const PackedMat &W, const UmmaMat &U, const
 }
 
 template <int D, typename KVT>
-dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit, bool merge) {
+dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit, bool merge, bool flash) {
   const dmtd_model_shape &s = c->s;
   int M = B * R, heads = s.n_q_heads + 2 * s.n_kv_heads, G = s.n_q_heads / s.n_kv_heads;
   KVT *kc = static_cast<KVT *>(c->kc) + (size_t)layer * c->kv_layer_elems;
@@ -350,6 +350,17 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
       c->qkv, c->ldqkv, s.n_q_heads, s.n_kv_heads, R, lw.w_qn, lw.w_kn, s.rms_eps, c->rope_tab, pos0, kc, vc,
       c->max_seq);
   LAUNCH_OK(c, "qk_norm_rope_append_kernel");
+  if constexpr (D == PK_D && !std::is_same<KVT, float>::value) {
+    if (flash) {
+      // a chunk of many positions per sequence (the prefill): the causal kernel, rows straight into `act`
+      using Op = typename std::conditional<std::is_same<KVT, __half>::value, OpF16, OpBf16>::type;
+      const int QB = PK_WARPS * (PK_QR / G);
+      attn_prefill_kernel<Op><<<dim3((R + QB - 1) / QB, s.n_kv_heads, B), PK_THREADS, ATTN_PF_SMEM, c->stream>>>(
+          c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, pos0, c->act, c->lda);
+      LAUNCH_OK(c, "attn_prefill_kernel");
+      return DMTD_OK;
+    }
+  }
   int RB = std::max(1, ATTN_QR / G), n_rb = (R + RB - 1) / RB;
   if (D == PK_D && c->use_tc_attention) {
     // head_dim 128: the tensor-core kernel with a bf16 cache, the FMA kernel with an fp32 cache
@@ -376,15 +387,23 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
   return DMTD_OK;
 }
 
-dmtd_status launch_attention(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit, bool merge = true) {
+// Chunks of at least this many positions per sequence run the causal prefill kernel (16-bit cache, head_dim 128).
+constexpr int kFlashMinRows = 16;
+bool flash_attention_ok(const dmtd_ctx *c, int R) {
+  const int G = c->s.n_q_heads / c->s.n_kv_heads;
+  return c->use_tc_attention && c->s.head_dim == PK_D && c->s.kv_dtype != DMTD_F32 && R >= kFlashMinRows && PK_QR % G == 0;
+}
+
+dmtd_status launch_attention(dmtd_ctx *c, int layer, int B, int R, const int *pos0, int nsplit, bool merge = true,
+                             bool flash = false) {
   const int kv = c->s.kv_dtype;
   if (c->s.head_dim == 128)
-    return kv == DMTD_BF16 ? launch_attention_t<128, __nv_bfloat16>(c, layer, B, R, pos0, nsplit, merge)
-         : kv == DMTD_F16 ? launch_attention_t<128, __half>(c, layer, B, R, pos0, nsplit, merge)
-                          : launch_attention_t<128, float>(c, layer, B, R, pos0, nsplit, merge);
-  return kv == DMTD_BF16 ? launch_attention_t<64, __nv_bfloat16>(c, layer, B, R, pos0, nsplit, merge)
-       : kv == DMTD_F16 ? launch_attention_t<64, __half>(c, layer, B, R, pos0, nsplit, merge)
-                        : launch_attention_t<64, float>(c, layer, B, R, pos0, nsplit, merge);
+    return kv == DMTD_BF16 ? launch_attention_t<128, __nv_bfloat16>(c, layer, B, R, pos0, nsplit, merge, flash)
+         : kv == DMTD_F16 ? launch_attention_t<128, __half>(c, layer, B, R, pos0, nsplit, merge, flash)
+                          : launch_attention_t<128, float>(c, layer, B, R, pos0, nsplit, merge, flash);
+  return kv == DMTD_BF16 ? launch_attention_t<64, __nv_bfloat16>(c, layer, B, R, pos0, nsplit, merge, flash)
+       : kv == DMTD_F16 ? launch_attention_t<64, __half>(c, layer, B, R, pos0, nsplit, merge, flash)
+                        : launch_attention_t<64, float>(c, layer, B, R, pos0, nsplit, merge, flash);
 }
 
 dmtd_status launch_rope_table(dmtd_ctx *c, const int *pos0, int R) {
@@ -425,8 +444,9 @@ dmtd_status run_layer(dmtd_ctx *c, int l, float *x, int B, int R, const int *pos
     TRY(launch_gemv(c, lw.qkv, lw.qkv_u, c->act, c->lda, M, c->qkv, c->ldqkv));
   }
   const int nsplit = splits_for(c, pos_end);
-  const bool fuse_merge = tc && NAB_ROWS * s.n_q_heads * nsplit <= MAB_MAX_SLOTS;
-  TRY(launch_attention(c, l, B, R, pos0, nsplit, !fuse_merge));
+  const bool flash = flash_attention_ok(c, R);
+  const bool fuse_merge = tc && !flash && NAB_ROWS * s.n_q_heads * nsplit <= MAB_MAX_SLOTS;
+  TRY(launch_attention(c, l, B, R, pos0, nsplit, !fuse_merge, flash));
   (void)QD;
   if (fuse_merge) TRY(launch_gemm_tc05(c, lw.o_u, nullptr, 0, M, x, H, 0, nullptr, nsplit));
   else TRY(launch_gemv(c, lw.o, lw.o_u, c->act, c->lda, M, x, H));
@@ -493,6 +513,8 @@ dmtd_status configure_kernels(dmtd_ctx *c) {
   CUDA_TRY(c, cudaFuncSetAttribute(attn_f32_kernel, dyn, ATTN_F32_SMEM));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<OpBf16>, dyn, ATTN_TC_SMEM));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<OpF16>, dyn, ATTN_TC_SMEM));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_prefill_kernel<OpBf16>, dyn, ATTN_PF_SMEM));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_prefill_kernel<OpF16>, dyn, ATTN_PF_SMEM));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<64, __half>, dyn, 64 * 1024));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<128, __half>, dyn, 64 * 1024));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<64, float>, dyn, 64 * 1024));
