@@ -45,7 +45,7 @@ namespace dmtd {
 // what the rings hold is what HBM delivers while the stage threads sit in a barrier.  The other
 // way: every other load of the SM waits behind the copies in flight.
 #ifndef DMTD_PASS_CHUNK
-#define DMTD_PASS_CHUNK 7
+#define DMTD_PASS_CHUNK 8
 #endif
 #ifndef DMTD_PASS_SLOTS
 #define DMTD_PASS_SLOTS 2
@@ -149,6 +149,18 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+// the same with an L2 eviction priority: a stream that is read once should not push what the stages share
+// through L2 (activations, partial sums, KV rows, the kernel's own instructions) out of it
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar), "l"(pol)
                : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

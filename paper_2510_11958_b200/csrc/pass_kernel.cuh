@@ -37,17 +37,34 @@ constexpr int PK_TIMING_SLOTS = 4096;
       t[1] = ns;                                                                                     \
     }                                                                                                \
   } while (0)
+// ... and, for the projections of the pass's last layer, when each chunk of the streams of warps 0 and 7 of
+// the first block was there to be consumed: slots 2048 + 64 * projection + 32 * (warp == 7) hold the clock
+// before and after the wait for every chunk, and at the end of the warp's share.
+#define PK_CHUNK_STAMP(i)                                                                            \
+  do {                                                                                               \
+    if (chunk_log >= 0 && (i) < 32 && lane == 0 && (warp == 0 || warp == 7) && blockIdx.x == 0 && P.timing) \
+      P.timing[chunk_log + (warp ? 32 : 0) + (i)] = clock64();                                       \
+  } while (0)
+#define PK_CHUNK_LOG_ARG , int chunk_log
 #else
 #define PK_STAMP() do {} while (0)
 #define PK_STAMP_WALL(i) do {} while (0)
+#define PK_CHUNK_STAMP(i) do {} while (0)
+#define PK_CHUNK_LOG_ARG
 #endif
+
+#ifndef DMTD_PASS_NACC
+#define DMTD_PASS_NACC 2
+#endif
+constexpr int PK_NACC = DMTD_PASS_NACC;
 
 // out[m][n] += sum_k W[n][k] act[m][k] over this warp's share of W, streamed through its ring.
 // Weights are the A operand of mma.m16n8k16 (register order, straight from the ring), the
 // activation hi/lo columns the B operand.  One atom per trip of a loop that is not unrolled:
 // the loop stays a few dozen instructions, holds everything in registers, and the other warps
 // of the block hide the shared-memory latency.
-__device__ __noinline__ bool gemv_consume(const PassParams &P, const PackedMat &W, int M, float *__restrict__ out, int ldo) {
+__device__ __noinline__ bool gemv_consume(const PassParams &P, const PackedMat &W, int M, float *__restrict__ out,
+                                          int ldo PK_CHUNK_LOG_ARG) {
   const PassShared S = pass_shared();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   WarpPipe pp = S.pipes[warp];
@@ -60,43 +77,97 @@ __device__ __noinline__ bool gemv_consume(const PassParams &P, const PackedMat &
   int T = in_slab / aps, a = in_slab - T * aps;
   uint32_t b_addr = smem_u32(S.bstage) + (s - s_first) * 8 * row_bytes + g * row_bytes + t * 16;
   const bool need_b = g < 2 * M;                          // columns beyond 2M belong to no activation row
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  int left = w1 - w0;
+  const int tile_mask = (PK_CHUNK_ATOMS % aps == 0 && (aps & (aps - 1)) == 0) ? aps - 1 : 0;
+  // The loop is bound by the number of instructions a warp issues per atom (two warps per scheduler:
+  // every instruction costs its full latency), not by the MMAs or by shared memory.  So: the
+  // activation fragments of the slab's (at most 8) atoms live in registers, loaded once per slab; the
+  // share is walked in segments (the atoms of one 16-row tile that lie in one chunk) whose body is
+  // unrolled over the position inside the tile, so that nothing but two loads and two MMAs is left per
+  // atom; the bookkeeping (chunk hand-over, the tile's reductions) is per segment.
+  uint4 Bq[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    Bq[k] = make_uint4(0u, 0u, 0u, 0u);
+    if (need_b && k < aps) Bq[k] = lds128(b_addr + k * 64);
+  }
+  // PK_NACC accumulators taken in turn (measured: 2, 4, 8 and 16 give 0.65, 0.74, 0.76 and 0.83 us per 8-atom
+  // chunk: the loop is bound by the rate at which the SM takes mma.sync, about one m16n8k16 per 32 cycles and
+  // scheduler, not by the chain through an accumulator)
+  float acc[PK_NACC][4];
+#pragma unroll
+  for (int i = 0; i < PK_NACC; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+  int left = w1 - w0, slot_left = 0;
+  uint32_t ptr = 0;
+#ifdef DMTD_PASS_TIMING
+  int chunk_i = 0;
+#endif
   while (left > 0) {
-    const int n = min(PK_CHUNK_ATOMS, left);
-    if (!pipe_wait(P, pp)) {
-      if (lane == 0) S.pipes[warp] = pp;
-      return false;
+    if (slot_left == 0) {
+      PK_CHUNK_STAMP(chunk_i++);
+      if (!pipe_wait(P, pp)) {
+        if (lane == 0) S.pipes[warp] = pp;
+        return false;
+      }
+      PK_CHUNK_STAMP(chunk_i++);
+      ptr = pp.ring + (pp.consumed % PK_SLOTS) * PK_CHUNK_BYTES + lane * 16;
+      slot_left = min(PK_CHUNK_ATOMS - (a & tile_mask), left);          // as pipe_issue cut it
     }
-    const uint32_t slot_addr = pp.ring + (pp.consumed % PK_SLOTS) * PK_CHUNK_BYTES + lane * 16;
-#pragma unroll 1
-    for (int u = 0; u < n; ++u) {
-      const uint4 A0 = lds128(slot_addr + u * 1024), A1 = lds128(slot_addr + u * 1024 + 512);
-      uint4 Bv = make_uint4(0u, 0u, 0u, 0u);
-      if (need_b) Bv = lds128(b_addr + a * 64);
-      mma_bf16_16816(acc, A0.x, A1.x, A0.y, A1.y, Bv.x, Bv.y);
-      mma_bf16_16816(acc, A0.z, A1.z, A0.w, A1.w, Bv.z, Bv.w);
-      ++a;
-      --left;
-      if (a == aps || left == 0) {
-        // accumulator columns 2t (hi) and 2t+1 (lo) belong to activation row t
-        const int n_lo = T * 16 + g;
-        if (t < M) {
-          if (n_lo < N) atomicAdd(out + (size_t)t * ldo + n_lo, acc[0] + acc[1]);
-          if (n_lo + 8 < N) atomicAdd(out + (size_t)t * ldo + n_lo + 8, acc[2] + acc[3]);
+    const int a_hi = min(aps, a + min(left, slot_left));
+    if (a == 0 && a_hi == 8) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const uint4 A0 = lds128(ptr + k * 1024), A1 = lds128(ptr + k * 1024 + 512);
+        mma_bf16_16816(acc[(2 * k) % PK_NACC], A0.x, A1.x, A0.y, A1.y, Bq[k].x, Bq[k].y);
+        mma_bf16_16816(acc[(2 * k + 1) % PK_NACC], A0.z, A1.z, A0.w, A1.w, Bq[k].z, Bq[k].w);
+      }
+      ptr += 8 * 1024;
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (k >= a && k < a_hi) {
+          const uint4 A0 = lds128(ptr), A1 = lds128(ptr + 512);
+          mma_bf16_16816(acc[(2 * k) % PK_NACC], A0.x, A1.x, A0.y, A1.y, Bq[k].x, Bq[k].y);
+          mma_bf16_16816(acc[(2 * k + 1) % PK_NACC], A0.z, A1.z, A0.w, A1.w, Bq[k].z, Bq[k].w);
+          ptr += 1024;
         }
-        acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
-        a = 0;
-        if (++T == n_tiles) { T = 0; b_addr += 8 * row_bytes; }
       }
     }
-    pp.consumed += 1;
-    __syncwarp();
-    if (lane == 0) {
-      fence_proxy_async();
-      pipe_issue(P, pp);
+    left -= a_hi - a;
+    slot_left -= a_hi - a;
+    a = a_hi;
+    if (slot_left == 0) {
+      pp.consumed += 1;
+      __syncwarp();
+      if (lane == 0) {
+        fence_proxy_async();
+        pipe_issue(P, pp);
+      }
+    }
+    if (a == aps || left == 0) {
+      // accumulator columns 2t (hi) and 2t+1 (lo) belong to activation row t
+      const int n_lo = T * 16 + g;
+      float lo = 0.f, hi = 0.f;
+#pragma unroll
+      for (int i = 0; i < PK_NACC; ++i) {
+        lo += acc[i][0] + acc[i][1];
+        hi += acc[i][2] + acc[i][3];
+        acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+      }
+      if (t < M) {
+        if (n_lo < N) atomicAdd(out + (size_t)t * ldo + n_lo, lo);
+        if (n_lo + 8 < N) atomicAdd(out + (size_t)t * ldo + n_lo + 8, hi);
+      }
+      a = 0;
+      if (++T == n_tiles && left > 0) {
+        T = 0;
+        b_addr += 8 * row_bytes;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          if (need_b && k < aps) Bq[k] = lds128(b_addr + k * 64);
+      }
     }
   }
+  PK_CHUNK_STAMP(chunk_i++);
   if (lane == 0) S.pipes[warp] = pp;
   __syncwarp();
   return true;
@@ -278,7 +349,12 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
       W = &Ly.down; out = x; ldo = P.H;
     }
     PK_STAMP();
+#ifdef DMTD_PASS_TIMING
+    const int chunk_log = (!head && li == nL - 1 && ph != 1) ? 2048 + 64 * (ph - (ph > 1)) : -1;
+    if (W && !gemv_consume(P, *W, M, out, ldo, chunk_log)) *S.abort_flag = 1;
+#else
     if (W && !gemv_consume(P, *W, M, out, ldo)) *S.abort_flag = 1;
+#endif
     PK_STAMP();
     ok = grid_barrier(P, bar_target);
     PK_STAMP();

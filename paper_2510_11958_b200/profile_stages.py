@@ -39,7 +39,7 @@ def main():
     ap.add_argument("--workload", default="qwen3_4b_b1")
     ap.add_argument("--kind", default="full", choices=["full", "upper"])
     ap.add_argument("--ghz", type=float, default=None, help="SM clock for tick -> us (default: measured in the launch itself)")
-    ap.add_argument("--kv", default=None, choices=["bf16", "f32"], help="KV cache type (default: the workload's)")
+    ap.add_argument("--kv", default=None, choices=["bf16", "f16", "f32"], help="KV cache type (default: the workload's)")
     ap.add_argument("--prompt-len", type=int, default=None, help="prompt length (default: the workload's)")
     ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
                     help="a dmtd_set_option setting for the run, e.g. prefetch_chunks=0 (repeatable)")
@@ -104,6 +104,16 @@ def main():
             if t[6] > t[2]:
                 print("  multiplied = scores %.2f, sync %.2f, softmax %.2f, sync %.2f, P V %.2f (fp32 cache only)" %
                       tuple(v / (args.ghz * 1e3) for v in (t[3] - t[2], t[4] - t[3], t[5] - t[4], t[6] - t[5], a[5] - t[6])))
+        if blk == 0:
+            print("  last layer, the chunks of a warp's share: waited + consumed (us); last figure: the share took")
+            for pi, pname in enumerate(("qkv", "o", "gate/up", "down")):
+                for wi, wname in enumerate(("warp 0", "warp 7")):
+                    c = s[2048 + 64 * pi + 32 * wi: 2048 + 64 * pi + 32 * wi + 32]
+                    c = c[c > 0]
+                    if len(c) > 2:
+                        d = np.diff(c) / (args.ghz * 1e3)
+                        print(f"    {pname:8s}{wname}: " + " ".join(f"{d[i]:.2f}+{d[i + 1]:.2f}" for i in range(0, len(d) - 1, 2)) +
+                              f" | {(c[-1] - c[0]) / (args.ghz * 1e3):.2f}")
         c0, w0, c1, w1 = (int(v) for v in s[SLOTS - 4:])
         print(f"  kernel entry to exit: {(w1 - w0) / 1e3:.1f} us by the wall clock, SM clock {(c1 - c0) / max(w1 - w0, 1):.3f} GHz; "
               f"entry to first stamp {(s[0] - c0) / (args.ghz * 1e3):.1f} us, last stamp to exit {(c1 - s[n - 1]) / (args.ghz * 1e3):.1f} us")
