@@ -235,6 +235,9 @@ def run_native(args, wl, shape):
         weights = make_weights(shape, seed=wl.weight_seed, device="cuda")
         wh = host_copy(weights) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
         eng = Dmtd(shape, weights, L_d=L_d, tau=tau, max_batch=B, max_seq=max_seq, kv_dtype=wl.kv_dtype)
+        for kv in args.option:
+            name, value = kv.split("=")
+            eng.set_option(name, int(value))
         prompts_host = make_prompts(shape.vocab, B, P, seed=wl.prompt_seed).pin_memory()
         prompts = prompts_host.cuda()
         memory = {k: round(v / 1e9, 3) for k, v in eng.memory_info().items()}
@@ -405,6 +408,8 @@ def main():
     ap.add_argument("--workload", default="qwen3_4b_b1")
     ap.add_argument("--tau", type=int, default=None)
     ap.add_argument("--kv-dtype", default=None, choices=["f32", "bf16", "f16"], help="KV cache type (default: the workload's)")
+    ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
+                    help="a dmtd_set_option setting of the measured engine, e.g. tcgen05_gemm_stages=4 (repeatable)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-tau1", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

@@ -56,6 +56,7 @@ struct dmtd_ctx {
   PackedMat embed{};
   UmmaMat embed_u{};
   bool umma_ok = false, use_umma = true;    // tcgen05 GEMM for projections of more than 4 rows
+  int gemm_stages = 0;                      // pipeline stages of its blocks; 0: chosen per launch
   uint4 *act_blocks = nullptr;
   float *w_final = nullptr;
   double *inv_freq = nullptr;
@@ -281,8 +282,14 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
     while (tmem_cols < P.n_cols) tmem_cols <<= 1;
     auto smem_of = [&](int st) { return st * (TG_WBLOCK + P.n_cols * 128) + 128; };
     auto per_sm_of = [&](int st) { return std::max(1, std::min((227 * 1024) / (smem_of(st) + 1024), 512 / tmem_cols)); };
-    P.stages = TG_STAGES;
-    if (P.n_sweeps == 1 && W.n_tiles > c->n_sms * per_sm_of(TG_STAGES) && W.n_tiles <= c->n_sms * per_sm_of(2)) P.stages = 2;
+    // stages: what keeps the most weight blocks in flight per SM (stages x resident blocks: a block streams at the
+    // rate its bytes in flight allow), more resident blocks on a tie (their fill and epilogue overlap)
+    const int max_stages = std::min(TG_STAGES, (227 * 1024 - 1024 - 128) / (TG_WBLOCK + P.n_cols * 128));
+    P.stages = 2;
+    for (int st = 2; st <= max_stages; ++st)
+      if (st * per_sm_of(st) > P.stages * per_sm_of(P.stages)) P.stages = st;
+    if (c->gemm_stages >= 2) P.stages = std::min(c->gemm_stages, max_stages);
+    if (P.n_sweeps == 1 && W.n_tiles > c->n_sms * per_sm_of(P.stages) && W.n_tiles <= c->n_sms * per_sm_of(2)) P.stages = 2;
     const int slots = c->n_sms * per_sm_of(P.stages);
     P.ksplit = std::max(1, std::min(W.n_kb, slots / (W.n_tiles * P.n_sweeps)));
     if (merge_nsplit > 0) {
@@ -509,7 +516,7 @@ dmtd_status configure_kernels(dmtd_ctx *c) {
   CUDA_TRY(c, cudaFuncSetAttribute(gemv_bf16_kernel<1>, dyn, 100 * 1024));
   CUDA_TRY(c, cudaFuncSetAttribute(gemv_bf16_kernel<2>, dyn, 100 * 1024));
   CUDA_TRY(c, cudaFuncSetAttribute(gemv_bf16_kernel<4>, dyn, 100 * 1024));
-  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc05_kernel, dyn, TG_STAGES * (TG_WBLOCK + TG_MAX_COLS * 128) + 128));
+  CUDA_TRY(c, cudaFuncSetAttribute(gemm_tc05_kernel, dyn, 227 * 1024 - 1024));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_f32_kernel, dyn, ATTN_F32_SMEM));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<OpBf16>, dyn, ATTN_TC_SMEM));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<OpF16>, dyn, ATTN_TC_SMEM));
@@ -1166,6 +1173,10 @@ dmtd_status dmtd_set_option(dmtd_ctx *c, const char *name, int64_t value) {
     if (value < 0 || value + c->L_d > c->s.n_layers)
       return fail(c, DMTD_ERR_SHAPE, "encoding_layers must be in [0, n_layers - L_d]");
     c->L_e = (int)value; drop_graphs(c); return DMTD_OK;
+  }
+  if (!strcmp(name, "tcgen05_gemm_stages")) {
+    if (value != 0 && (value < 2 || value > TG_STAGES)) return fail(c, DMTD_ERR_INVALID_ARG, "tcgen05_gemm_stages takes 0 (chosen per launch) or 2..%d", TG_STAGES);
+    c->gemm_stages = (int)value; drop_graphs(c); return DMTD_OK;
   }
   if (value != 0 && value != 1) return fail(c, DMTD_ERR_INVALID_ARG, "option %s takes 0 or 1", name);
   if (!strcmp(name, "cuda_graph")) { c->use_graph = value != 0; return DMTD_OK; }

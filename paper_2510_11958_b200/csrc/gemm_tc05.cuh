@@ -21,7 +21,7 @@
 namespace dmtd {
 
 constexpr int TG_THREADS = 192;
-constexpr int TG_STAGES = 4;
+constexpr int TG_STAGES = 6;                 // most pipeline stages a block may be given
 constexpr int TG_ROWS = 128;                 // weight rows per tile (MMA M)
 constexpr int TG_KB = 64;                    // k per pipeline stage: four MMAs of K = 16
 constexpr int TG_WBLOCK = TG_ROWS * TG_KB * 2;      // 16384 bytes

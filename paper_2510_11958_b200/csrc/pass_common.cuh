@@ -38,8 +38,10 @@
 namespace dmtd {
 
 // Ring geometry (overridable at build time for sweeps).  Measured on the Qwen3-4B shape, batch 1,
-// us per layer of a full pass: chunks of 4 / 5 / 6 / 7 / 8 atoms in 2 slots 66.9 / 64.9 / 63.6 /
-// 63.5 / 64.8; 3 slots of 5 atoms 64.6, 4 slots of 4 atoms 64.7.  Two things pull one way: the copy
+// with a consumer loop that took one atom per trip, us per layer of a full pass: chunks of 4 / 5 / 6 /
+// 7 / 8 atoms in 2 slots 66.9 / 64.9 / 63.6 / 63.5 / 64.8; 3 slots of 5 atoms 64.6, 4 slots of 4 atoms
+// 64.7.  The loop that multiplies a whole 16-row tile (8 atoms at 256-wide k-slabs) in straight-line
+// code wants a chunk to be a tile: 8 atoms (861 against 850 tokens/s with 7).  Two things pull one way: the copy
 // engine of an SM spends ~100 cycles per bulk copy whatever its size (a plain stream of 4 KiB copies
 // tops out at 60 GB/s per SM, of 8 KiB copies at 100 GB/s; the SM's share of HBM is 44 GB/s), and
 // what the rings hold is what HBM delivers while the stage threads sit in a barrier.  The other
