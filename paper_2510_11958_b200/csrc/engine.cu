@@ -260,6 +260,20 @@ dmtd_status launch_gemv_nt(dmtd_ctx *c, const PackedMat &W, const float *act, in
 // weight tile with up to 128 activation rows (a sweep); prefill chunks of more rows are several
 // sweeps in one launch (up to TG_MAX_SWEEPS), ordered so that the sweeps of one weight tile run
 // together and share it through L2.
+// Launch with programmatic stream serialisation: the kernel's blocks may become resident while the
+// kernel before it in the stream is still running; it calls griddepcontrol.wait before it touches
+// anything that kernel (or one before it) writes.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // With `norm_w` the activations are RMSNorm(act rows) * norm_w, computed while the blocks are written, and
 // the output rows are cleared first (the projections after a norm write a fresh buffer).
 dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, int lda, int M, float *out, int ldo,
@@ -296,24 +310,24 @@ dmtd_status launch_gemm_tc05(dmtd_ctx *c, const UmmaMat &W, const float *act, in
       // `act` is unused: the activations are the attention's key slices, merged on the way
       const int n_groups = P.n_sweeps * (P.n_cols / 2 / NAB_ROWS);
       const int ky = std::max(1, std::min(W.n_kb, 4 * c->n_sms / std::max(1, n_groups)));
-      merge_act_blocks_kernel<<<dim3(n_groups, ky), 256, 0, c->stream>>>(
-          c->part_o + (size_t)m0 * c->s.n_q_heads * merge_nsplit * c->s.head_dim,
-          c->part_ml + (size_t)m0 * c->s.n_q_heads * merge_nsplit * 2, merge_nsplit, c->s.n_q_heads, c->s.head_dim, P.rows, P.n_cols,
-          c->act_blocks);
+      CUDA_TRY(c, launch_pdl(merge_act_blocks_kernel, dim3(n_groups, ky), dim3(256), 0, c->stream,
+                             c->part_o + (size_t)m0 * c->s.n_q_heads * merge_nsplit * c->s.head_dim,
+                             c->part_ml + (size_t)m0 * c->s.n_q_heads * merge_nsplit * 2, merge_nsplit, c->s.n_q_heads,
+                             c->s.head_dim, P.rows, P.n_cols, c->act_blocks));
       LAUNCH_OK(c, "merge_act_blocks_kernel");
     } else if (norm_w) {
       const int n_groups = P.n_sweeps * (P.n_cols / 2 / NAB_ROWS);
       const size_t zero_n4 = (size_t)P.rows * ldo / 4;                  // ldo is a multiple of 4 (checked by the caller)
       const int n_zero = (int)std::min<size_t>((zero_n4 + 1023) / 1024, 2 * c->n_sms);
       const int ky = std::max(1, std::min(W.n_kb, 4 * c->n_sms / std::max(1, n_groups)));
-      norm_act_blocks_kernel<<<dim3(n_groups + (n_zero + ky - 1) / ky, ky), 256, 0, c->stream>>>(
-          act + (size_t)m0 * lda, lda, norm_w, c->s.rms_eps, P.rows, W.K, P.n_cols, c->act_blocks, n_groups,
-          reinterpret_cast<float4 *>(out + (size_t)m0 * ldo), zero_n4);
+      CUDA_TRY(c, launch_pdl(norm_act_blocks_kernel, dim3(n_groups + (n_zero + ky - 1) / ky, ky), dim3(256), 0, c->stream,
+                             act + (size_t)m0 * lda, lda, norm_w, c->s.rms_eps, P.rows, W.K, P.n_cols, c->act_blocks, n_groups,
+                             reinterpret_cast<float4 *>(out + (size_t)m0 * ldo), zero_n4));
       LAUNCH_OK(c, "norm_act_blocks_kernel");
     } else {
       long long units = (long long)W.n_kb * 8 * P.n_cols;
-      act_blocks_kernel<<<dim3((int)std::min<long long>((units + 255) / 256, 4096), P.n_sweeps), 256, 0, c->stream>>>(
-          act + (size_t)m0 * lda, lda, P.rows, W.K, P.n_cols, c->act_blocks, gate_up_I);
+      CUDA_TRY(c, launch_pdl(act_blocks_kernel, dim3((int)std::min<long long>((units + 255) / 256, 4096), P.n_sweeps), dim3(256), 0,
+                             c->stream, act + (size_t)m0 * lda, lda, P.rows, W.K, P.n_cols, c->act_blocks, gate_up_I));
       LAUNCH_OK(c, "act_blocks_kernel");
     }
     int smem = smem_of(P.stages);

@@ -97,6 +97,10 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc05_kernel(const __grid_c
   int tmem_cols = 32;
   while (tmem_cols < P.n_cols) tmem_cols <<= 1;
 
+  // the kernel after this one (the next projection's activation-block kernel, launched the same way) may become
+  // resident now; it waits for this grid's completion before it reads or writes anything, and the GEMM behind it
+  // can then request its first weight blocks while this grid's last blocks finish
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2 * S + 1; ++s) mbar_init(smem_u32(bars + s), 1);
     *gave_up = 0;
@@ -204,6 +208,9 @@ __global__ void act_blocks_kernel(const float *__restrict__ act_all, int lda, in
   uint4 *blocks = blocks_all + (size_t)blockIdx.y * (K / TG_KB) * (n_cols * 8);
   // the GEMM that follows may be scheduled already: it waits for this grid before it reads the blocks
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // ... and this grid may itself have started before the kernel before it has finished (the GEMM of the previous
+  // projection lets its dependents in at once): nothing is read or written before that kernel is complete
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n_kb = K / TG_KB;
   const long long total = (long long)n_kb * 8 * n_cols;            // 16-byte units
   for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (long long)gridDim.x * blockDim.x) {
@@ -243,6 +250,9 @@ __global__ void __launch_bounds__(256) norm_act_blocks_kernel(const float *__res
                                                               float4 *__restrict__ zero, size_t zero_n4) {
   // the GEMM that follows may be scheduled already: it waits for this grid before it reads the blocks
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // ... and this grid may itself have started before the kernel before it has finished (the GEMM of the previous
+  // projection lets its dependents in at once): nothing is read or written before that kernel is complete
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if ((int)blockIdx.x >= n_groups) {
     const size_t n_z = (size_t)(gridDim.x - n_groups) * gridDim.y;
     for (size_t i = ((size_t)(blockIdx.x - n_groups) * gridDim.y + blockIdx.y) * blockDim.x + threadIdx.x; i < zero_n4;
@@ -310,6 +320,9 @@ __global__ void __launch_bounds__(256) merge_act_blocks_kernel(const float *__re
                                                                int nsplit, int nq, int D, int rows_all, int n_cols,
                                                                uint4 *__restrict__ blocks_all) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // ... and this grid may itself have started before the kernel before it has finished (the GEMM of the previous
+  // projection lets its dependents in at once): nothing is read or written before that kernel is complete
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int K = nq * D, n_kb = K / TG_KB;
   const int sweep_rows = n_cols / 2, groups_per_sweep = sweep_rows / NAB_ROWS;
   const int sweep = blockIdx.x / groups_per_sweep, m_in0 = (blockIdx.x % groups_per_sweep) * NAB_ROWS;
