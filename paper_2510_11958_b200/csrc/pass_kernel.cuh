@@ -356,6 +356,14 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
     if (W && !gemv_consume(P, *W, M, out, ldo)) *S.abort_flag = 1;
 #endif
     PK_STAMP();
+#ifdef DMTD_PASS_TIMING
+    // every block's wall clock at the end of its share of the last layer's projections (slots 3200 + 160 * projection + block)
+    if (threadIdx.x == 0 && P.timing && !head && li == nL - 1 && ph != 1 && gridDim.x <= 160) {
+      long long ns;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+      P.timing[3200 + 160 * (ph - (ph > 1)) + blockIdx.x] = ns;
+    }
+#endif
     ok = grid_barrier(P, bar_target);
     PK_STAMP();
   }

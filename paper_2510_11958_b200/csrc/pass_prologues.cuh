@@ -36,6 +36,7 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
                                            const float *w_norm, const PackedMat &W) {
   const PassShared S = pass_shared();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, H = P.H;
+  PK_PROSTAMP(0);
   // one copy per row, each issued by its own lane of the first warp
   if (threadIdx.x == 0) stage_begin(S, (uint32_t)(M * H * 4));
   if (warp == 0) {
@@ -54,7 +55,9 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
     wv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (u < nu) wv[j] = __ldg(reinterpret_cast<const float4 *>(w_norm + sp.first * sp.KS) + u);
   }
+  PK_PROSTAMP(1);
   stage_wait(P, S);
+  PK_PROSTAMP(2);
 #pragma unroll 1
   for (int m = 0; m < M; ++m) {
     float ss = 0.f;
@@ -67,6 +70,7 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
     if (lane == 0) S.red[warp * PK_MAX_ROWS + m] = ss;
   }
   pk_sync();
+  PK_PROSTAMP(3);
 #pragma unroll 1
   for (int m = 0; m < M; ++m) {
     float v = 0.f;
@@ -84,7 +88,9 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
       }
     }
   }
+  PK_PROSTAMP(4);
   pk_sync();
+  PK_PROSTAMP(5);
 }
 
 // SwiGLU gate (step a6, second half) for the k-slabs this block needs of the down projection.

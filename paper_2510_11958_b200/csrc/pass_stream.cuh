@@ -5,6 +5,17 @@
 
 namespace dmtd {
 
+// Profiling builds: clock64() of thread 0 of the first block at points inside a norm prologue (slots 3072 ..)
+// and the grid barrier (3088 ..); the values of the last call stay.
+#ifdef DMTD_PASS_TIMING
+#define PK_PROSTAMP(i)                                                                 \
+  do {                                                                                 \
+    if (threadIdx.x == 0 && blockIdx.x == 0 && P.timing) P.timing[3072 + (i)] = clock64(); \
+  } while (0)
+#else
+#define PK_PROSTAMP(i) do {} while (0)
+#endif
+
 // Position in one warp's weight stream: its share of every matrix of the pass, in pass order.
 // Atom counts are 32-bit: the host checks atoms * blocks < 2^31 for every matrix.
 struct StreamCursor {
@@ -111,7 +122,9 @@ __device__ __forceinline__ bool pipe_wait(const PassParams &P, const WarpPipe &p
 // Grid-wide barrier: every block arrives once per stage; `target` counts arrivals so far.
 __device__ __noinline__ bool grid_barrier(const PassParams &P, unsigned &target) {
   const PassShared S = pass_shared();
+  PK_PROSTAMP(16);
   pk_sync();
+  PK_PROSTAMP(17);
   if (threadIdx.x == 0) {
     target += gridDim.x;
     if (*S.abort_flag) {
@@ -130,7 +143,9 @@ __device__ __noinline__ bool grid_barrier(const PassParams &P, unsigned &target)
       }
     }
   }
+  PK_PROSTAMP(18);
   pk_sync();
+  PK_PROSTAMP(19);
   return *S.abort_flag == 0;
 }
 

@@ -114,6 +114,20 @@ def main():
                         d = np.diff(c) / (args.ghz * 1e3)
                         print(f"    {pname:8s}{wname}: " + " ".join(f"{d[i]:.2f}+{d[i + 1]:.2f}" for i in range(0, len(d) - 1, 2)) +
                               f" | {(c[-1] - c[0]) / (args.ghz * 1e3):.2f}")
+        if blk == 0:
+            us = lambda a: " ".join(f"{v / (args.ghz * 1e3):.2f}" for v in np.diff(a))
+            print("  inside the last norm prologue (rows and norm weights requested, rows landed, squares summed, "
+                  "columns written, block barrier): " + us(s[3072:3078]))
+            for pi, pname in enumerate(("qkv", "o", "gate/up", "down")):
+                f = s[3200 + 160 * pi: 3200 + 160 * pi + 160]
+                f = f[f > 0].astype(np.float64)
+                if len(f):
+                    f = (f - f.min()) / 1e3
+                    order = np.argsort(f)
+                    print(f"  last layer, {pname}: blocks done within {f.max():.2f} us of the first (median {np.median(f):.2f}); "
+                          f"last five blocks {[int(v) for v in order[-5:]]} at " + " ".join(f"{v:.2f}" for v in f[order[-5:]]) +
+                          f"; by block index, means of 4 groups of 37: " + " ".join(f"{f[i * 37:(i + 1) * 37].mean():.2f}" for i in range(4)))
+            print("  inside the last grid barrier (block barrier, arrive + poll, block barrier): " + us(s[3088:3092]))
         c0, w0, c1, w1 = (int(v) for v in s[SLOTS - 4:])
         print(f"  kernel entry to exit: {(w1 - w0) / 1e3:.1f} us by the wall clock, SM clock {(c1 - c0) / max(w1 - w0, 1):.3f} GHz; "
               f"entry to first stamp {(s[0] - c0) / (args.ghz * 1e3):.1f} us, last stamp to exit {(c1 - s[n - 1]) / (args.ghz * 1e3):.1f} us")
