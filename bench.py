@@ -142,7 +142,13 @@ def run_reference(args, wl, shape):
 
 # DRAM traffic / algorithmic bytes of the dominant kernel, from ncu captures of exactly the kernel
 # and the shape named here (profiles/); any other workload reports traffic = null.
-NCU_TRAFFIC_RATIO = {}
+NCU_TRAFFIC_RATIO = {
+    # profiles/dmtd_pass_kernel_qwen3_4b_l4_b1_ncu_full.md: the three launches of a cycle on the 4-layer model read
+    # and wrote 3.9854 GB for 3.9660 GB of weights and KV; the 36-layer workload runs the same kernel on the same
+    # layer and head shapes, and its traffic grows with the bytes streamed
+    ("qwen3_4b_l4_b1", "fused"): 1.0049,
+    ("qwen3_4b_b1", "fused"): 1.0049,
+}
 
 
 def measure_workload(eng, wl, shape, prompts, tau, K, W, replicas, want_tau1=True):
