@@ -28,9 +28,14 @@
 //    4 KiB chunk (shared-memory atomic, table look-ups, two divisions, slot records) sits
 //    between a slot becoming free and its next request, and the stream ran at half speed.
 //    Fixed per-warp shares keep that path to a few dozen instructions.
-//  * mma.sync issues about once per 30 cycles per SM sub-partition here: enough for the weight
-//    loop (one atom per ~90 cycles), too slow for attention with bf16 hi/lo pairs, which is
-//    why the fp32-cache attention stage uses FMAs.
+//  * mma.sync issues once per 32 cycles per SM sub-partition here (the hmma sub-pipe counter of ncu):
+//    with two warps per sub-partition and two MMAs per atom that is 128 of the 150 cycles the weight
+//    loop takes per atom and warp - 2.3 times the SM's share of HBM, so the loop keeps up, and a ring
+//    filled during a barrier is drained at that rate.  It is too slow for attention with bf16 hi/lo
+//    pairs, which is why the fp32-cache attention stage uses FMAs.
+//  * the weight loop must stay short: with one atom per trip and the tile bookkeeping inside it
+//    (about 45 instructions per atom, each at its full latency with two warps per sub-partition) a
+//    warp took 260 cycles per atom, exactly the SM's share of HBM, and never waited for a chunk.
 #pragma once
 
 #include "common.cuh"
