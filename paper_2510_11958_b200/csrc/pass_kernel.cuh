@@ -331,6 +331,12 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
       if (P.kv_f32) attention_stage_f32(P, Ly, R, pos0);
       else if (P.kv_f16) attention_stage<OpF16>(P, Ly, R, pos0);
       else attention_stage<OpBf16>(P, Ly, R, pos0);
+      if (PK_ATTN_PF_ATOMS > 0) {
+        int nsplit, CH;
+        attn_plan_device(P, pos0, nsplit, CH);
+        const int items = P.B * P.nkv * nsplit;
+        if ((int)blockIdx.x >= items) prefetch_matrix_part(Ly.gu, (int)blockIdx.x - items, (int)gridDim.x - items);
+      }
     } else if (ph == 2) {
       // a4 merge of the key slices + a5: O projection into the residual rows
       grid_zero(P.gu, M_max * ldgu);
@@ -348,6 +354,10 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
       swiglu_prologue(P, M, Ly.down);
       W = &Ly.down; out = x; ldo = P.H;
     }
+    // the prologue's own loads are done: ask L2 for the next atoms of the warp's stream (HBM is idle until the
+    // projection has drained the ring)
+    if (PK_PRO_PF_ATOMS > 0 && lane == 0 && ph != 1 && ph != 2)
+      prefetch_own_stream(S.pipes[warp].cur, (!head && ph == 3) ? PK_ATTN_PF_ATOMS : 0);
     PK_STAMP();
 #ifdef DMTD_PASS_TIMING
     const int chunk_log = (!head && li == nL - 1 && ph != 1) ? 2048 + 64 * (ph - (ph > 1)) : -1;
@@ -358,10 +368,10 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
     PK_STAMP();
 #ifdef DMTD_PASS_TIMING
     // every block's wall clock at the end of its share of the last layer's projections (slots 3200 + 160 * projection + block)
-    if (threadIdx.x == 0 && P.timing && !head && li == nL - 1 && ph != 1 && gridDim.x <= 160) {
+    if (threadIdx.x == 0 && P.timing && !head && li == nL - 1 && gridDim.x <= 160) {
       long long ns;
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
-      P.timing[3200 + 160 * (ph - (ph > 1)) + blockIdx.x] = ns;
+      P.timing[3200 + 160 * (ph == 1 ? 4 : ph - (ph > 1)) + blockIdx.x] = ns;
     }
 #endif
     ok = grid_barrier(P, bar_target);

@@ -118,7 +118,7 @@ def main():
             us = lambda a: " ".join(f"{v / (args.ghz * 1e3):.2f}" for v in np.diff(a))
             print("  inside the last norm prologue (rows and norm weights requested, rows landed, squares summed, "
                   "columns written, block barrier): " + us(s[3072:3078]))
-            for pi, pname in enumerate(("qkv", "o", "gate/up", "down")):
+            for pi, pname in enumerate(("qkv", "o", "gate/up", "down", "attention")):
                 f = s[3200 + 160 * pi: 3200 + 160 * pi + 160]
                 f = f[f > 0].astype(np.float64)
                 if len(f):
