@@ -310,11 +310,9 @@ __device__ __forceinline__ void attn_combine_store(AttnAcc &A, unsigned char *sc
 // The slice's unnormalised partial output goes to global memory with its max and sum; the
 // prologue of the O projection merges the slices.
 template <class Op>
-__device__ __noinline__ void attention_stage(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
+__device__ __noinline__ void attention_stage(const PassParams &P, const PassLayer &Ly, int R, int pos0, int nsplit, int CH) {
   const PassShared S = pass_shared();
   const int G = P.nq / P.nkv, nQ = R * G;
-  int nsplit, CH;
-  attn_plan_device(P, pos0, nsplit, CH);
   const int items = P.B * P.nkv * nsplit;
   if ((int)blockIdx.x >= items) return;
 

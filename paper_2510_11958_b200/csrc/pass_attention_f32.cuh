@@ -249,11 +249,9 @@ __device__ __forceinline__ void attn_f32_combine(unsigned char *sc, float (&acc)
 // Steps a3 + a4 for the items (sequence, kv head, key slice) of this block, fp32 cache.
 // Per 64-key tile: scores by (key, quarter-of-d) threads with the K row in registers; softmax
 // statistics by one warp per query row; P V by (key group = warp, 4 output dims = lane) threads.
-__device__ __noinline__ void attention_stage_f32(const PassParams &P, const PassLayer &Ly, int R, int pos0) {
+__device__ __noinline__ void attention_stage_f32(const PassParams &P, const PassLayer &Ly, int R, int pos0, int nsplit, int CH) {
   const PassShared S = pass_shared();
   const int G = P.nq / P.nkv, nQ = R * G;
-  int nsplit, CH;
-  attn_plan_device(P, pos0, nsplit, CH);
   const int items = P.B * P.nkv * nsplit;
   if ((int)blockIdx.x >= items) return;
   unsigned char *const sc = S.bstage;

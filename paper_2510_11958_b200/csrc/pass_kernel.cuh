@@ -300,6 +300,10 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
   // Stage list: five stages per layer, then the LM head.  Every stage is a prologue that puts
   // the activations this block needs into shared memory, the block's share of one projection,
   // and a grid barrier.  The attention stage has no projection.
+  // the key slices of the attention stages depend on the context length only: worked out once per pass
+  int nsplit_lo, CH_lo, nsplit_up, CH_up;
+  attn_plan_device(P, lo_len, nsplit_lo, CH_lo);
+  attn_plan_device(P, newest, nsplit_up, CH_up);
   const int n_stages = nL * 5 + 1;
   for (int stage = 0; stage < n_stages && ok; ++stage) {
     const int li = stage / 5, ph = stage - li * 5;
@@ -308,6 +312,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
     const bool lower = !head && l < P.l_split;
     const int R = lower ? P.R_lo : 1, M = P.B * R, pos0 = lower ? lo_len : newest;
     float *x = lower ? P.x_lo : P.x_up;
+    const int nsplit = lower ? nsplit_lo : nsplit_up, CH = lower ? CH_lo : CH_up;      // key slices of the attention stage
     const PassLayer &Ly = S.layers[head ? 0 : li];
     const PackedMat *W = nullptr;
     float *out = nullptr;
@@ -328,20 +333,16 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
       W = &Ly.qkv; out = P.qkv; ldo = ldqkv;
     } else if (ph == 1) {
       // a3 + a4: QK-norm, RoPE, KV append, attention over the key slices
-      if (P.kv_f32) attention_stage_f32(P, Ly, R, pos0);
-      else if (P.kv_f16) attention_stage<OpF16>(P, Ly, R, pos0);
-      else attention_stage<OpBf16>(P, Ly, R, pos0);
+      if (P.kv_f32) attention_stage_f32(P, Ly, R, pos0, nsplit, CH);
+      else if (P.kv_f16) attention_stage<OpF16>(P, Ly, R, pos0, nsplit, CH);
+      else attention_stage<OpBf16>(P, Ly, R, pos0, nsplit, CH);
       if (PK_ATTN_PF_ATOMS > 0) {
-        int nsplit, CH;
-        attn_plan_device(P, pos0, nsplit, CH);
         const int items = P.B * P.nkv * nsplit;
         if ((int)blockIdx.x >= items) prefetch_matrix_part(Ly.gu, (int)blockIdx.x - items, (int)gridDim.x - items);
       }
     } else if (ph == 2) {
       // a4 merge of the key slices + a5: O projection into the residual rows
       grid_zero(P.gu, M_max * ldgu);
-      int nsplit, CH;
-      attn_plan_device(P, pos0, nsplit, CH);
       merge_prologue(P, M, nsplit, Ly.o);
       W = &Ly.o; out = x; ldo = P.H;
     } else if (ph == 3) {

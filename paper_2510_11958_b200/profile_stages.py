@@ -98,6 +98,9 @@ def main():
             a = s[SLOTS - 20:SLOTS - 12]
             print("  inside the last layer's attention stage (entry, rows requested, cached tile fetched, rows landed, "
                   "rows normed, tiles done, partials stored, exit): " + " ".join(f"{v / (args.ghz * 1e3):.2f}" for v in np.diff(a)))
+            i_bar = 1 + (n_layers - 1) * 15 + 2                 # stamp after the last layer's QKV barrier; + 1: after its attention stage
+            print("  last layer: %.2f us from the QKV barrier's end to the attention stage's first stamp, %.2f us from its last stamp to the stage's end"
+                  % ((a[0] - s[i_bar]) / (args.ghz * 1e3), (s[i_bar + 1] - a[7]) / (args.ghz * 1e3)))
             t = s[SLOTS - 12:SLOTS - 5]
             print("  last tile: sync %.2f, new rows placed %.2f, copies landed + sync %.2f, multiplied %.2f" %
                   tuple(v / (args.ghz * 1e3) for v in (t[0] - a[4], t[1] - t[0], t[2] - t[1], a[5] - t[2])))
