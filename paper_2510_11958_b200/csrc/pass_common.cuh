@@ -83,7 +83,7 @@ constexpr int PK_OFF_BSTAGE = PK_OFF_RING + PK_RING_BYTES;
 constexpr int PK_OFF_XS = PK_OFF_BSTAGE + PK_BSTAGE_BYTES;                    // directly behind bstage
 constexpr int PK_OFF_BARS = PK_OFF_XS + PK_XS_BYTES;
 constexpr int PK_OFF_SMALL = PK_OFF_BARS + PK_WARPS * PK_SLOTS * 8;
-constexpr int PK_SMALL_BYTES = 1024;
+constexpr int PK_SMALL_BYTES = 2048;
 constexpr int PK_OFF_LAYERS = PK_OFF_SMALL + PK_SMALL_BYTES;
 
 enum { PK_ERR_NONE = 0, PK_ERR_TOKEN = 1, PK_ERR_COPY_WAIT = 2, PK_ERR_BARRIER_WAIT = 3 };
@@ -197,6 +197,20 @@ __device__ __forceinline__ void pk_sync() { __syncthreads(); }
 
 struct WarpPipe;
 
+// Where this block's and its warps' shares of a matrix begin and end (atoms of the stream), which k-slabs the
+// block's share touches, and where in its slab a warp's share starts.  Every layer has the same five matrix shapes
+// (QKV, O, gate+up, down; the tied head), so the plans are worked out once per launch: between two grid barriers
+// everything is serial latency, and the divisions of these index computations were a measurable part of it.
+enum { PK_MAT_QKV = 0, PK_MAT_O = 1, PK_MAT_GU = 2, PK_MAT_DOWN = 3, PK_MAT_HEAD = 4, PK_MAT_KINDS = 5 };
+struct MatPlan {
+  int c0, c1;                     // the block's atoms [c0, c1)
+  int s_first, s_count;           // k-slabs the block's share touches
+  int w0[PK_WARPS], w1[PK_WARPS]; // the warps' atoms
+  int ws[PK_WARPS], wT[PK_WARPS], wa[PK_WARPS];   // slab, 16-row tile and atom in the tile where a warp's share starts
+};
+
+static_assert(PK_MAT_KINDS * sizeof(MatPlan) <= 1024, "matrix plans do not fit the small area");
+
 struct PassShared {
   unsigned char *ring;      // [warp][slot][PK_CHUNK_BYTES]
   unsigned char *bstage;    // activation columns of up to two k-slabs; attention scratch (with xs)
@@ -207,6 +221,7 @@ struct PassShared {
   uint64_t *stage_bar;      // completion of the bulk copies that stage a prologue's inputs
   float *red;               // [PK_WARPS][PK_MAX_ROWS]
   WarpPipe *pipes;          // [PK_WARPS] ring state of every warp between stages
+  MatPlan *plans;           // [PK_MAT_KINDS]
   PassLayer *layers;        // layers [l_begin, l_end) of this pass
 };
 
@@ -224,6 +239,7 @@ __device__ __forceinline__ PassShared pass_shared() {
   S.stage_bar = reinterpret_cast<uint64_t *>(pk_smem + PK_OFF_SMALL + 8);
   S.red = reinterpret_cast<float *>(pk_smem + PK_OFF_SMALL + 64);
   S.pipes = reinterpret_cast<WarpPipe *>(pk_smem + PK_OFF_SMALL + 256);
+  S.plans = reinterpret_cast<MatPlan *>(pk_smem + PK_OFF_SMALL + 1024);
   S.layers = reinterpret_cast<PassLayer *>(pk_smem + PK_OFF_LAYERS);
   return S;
 }

@@ -63,18 +63,18 @@ constexpr int PK_NACC = DMTD_PASS_NACC;
 // activation hi/lo columns the B operand.  One atom per trip of a loop that is not unrolled:
 // the loop stays a few dozen instructions, holds everything in registers, and the other warps
 // of the block hide the shared-memory latency.
-__device__ __noinline__ bool gemv_consume(const PassParams &P, const PackedMat &W, int M, float *__restrict__ out,
+__device__ __noinline__ bool gemv_consume(const PassParams &P, const PackedMat &W, int kind, int M, float *__restrict__ out,
                                           int ldo PK_CHUNK_LOG_ARG) {
   const PassShared S = pass_shared();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   WarpPipe pp = S.pipes[warp];
   const int aps = W.aps, n_tiles = W.n_tiles, N = W.N;
-  int c0, c1, w0, w1;
-  stream_ranges(W, warp, c0, c1, w0, w1);
+  const MatPlan &pl = S.plans[kind];
+  const int w0 = pl.w0[warp], w1 = pl.w1[warp];
   if (w0 >= w1) return true;
-  const int slab_atoms = n_tiles * aps, row_bytes = b_row_bytes(aps * 32);
-  const int s_first = c0 / slab_atoms, s = w0 / slab_atoms, in_slab = w0 - s * slab_atoms;
-  int T = in_slab / aps, a = in_slab - T * aps;
+  const int row_bytes = b_row_bytes(aps * 32);
+  const int s_first = pl.s_first, s = pl.ws[warp];
+  int T = pl.wT[warp], a = pl.wa[warp];
   uint32_t b_addr = smem_u32(S.bstage) + (s - s_first) * 8 * row_bytes + g * row_bytes + t * 16;
   const bool need_b = g < 2 * M;                          // columns beyond 2M belong to no activation row
   const int tile_mask = (PK_CHUNK_ATOMS % aps == 0 && (aps & (aps - 1)) == 0) ? aps - 1 : 0;
@@ -265,6 +265,8 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
     fence_mbar_init();
   }
   pk_sync();
+  plans_fill(P, S);
+  pk_sync();
 
   const int lo_len = P.st->lo_len, newest = P.st->newest;
   {
@@ -305,8 +307,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
   attn_plan_device(P, lo_len, nsplit_lo, CH_lo);
   attn_plan_device(P, newest, nsplit_up, CH_up);
   const int n_stages = nL * 5 + 1;
-  for (int stage = 0; stage < n_stages && ok; ++stage) {
-    const int li = stage / 5, ph = stage - li * 5;
+  for (int stage = 0, li = 0, ph = 0; stage < n_stages && ok; ++stage, ph = ph == 4 ? 0 : ph + 1, li += ph == 0) {
     const bool head = li == nL;
     const int l = P.l_begin + li;
     const bool lower = !head && l < P.l_split;
@@ -319,16 +320,16 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
     int ldo = 0;
     if (head) {
       // a9: final norm, tied head
-      norm_prologue(P, P.x_up, (size_t)P.H, M, P.w_final, P.embed);
+      norm_prologue(P, P.x_up, (size_t)P.H, M, P.w_final, P.embed, PK_MAT_HEAD);
       W = &P.embed; out = P.logits; ldo = P.ldl;
     } else if (ph == 0) {
       // a2: RMSNorm, QKV projection; a8 at the first decoding layer of a full pass: the newest
       // row of each sequence is read straight from the lower stack's rows and copied to x_up
       if (has_lower && l == P.l_split) {
         select_rows(P);
-        norm_prologue(P, P.x_lo + (size_t)(P.R_lo - 1) * P.H, (size_t)P.R_lo * P.H, M, Ly.w_in, Ly.qkv);
+        norm_prologue(P, P.x_lo + (size_t)(P.R_lo - 1) * P.H, (size_t)P.R_lo * P.H, M, Ly.w_in, Ly.qkv, PK_MAT_QKV);
       } else {
-        norm_prologue(P, x, (size_t)P.H, M, Ly.w_in, Ly.qkv);
+        norm_prologue(P, x, (size_t)P.H, M, Ly.w_in, Ly.qkv, PK_MAT_QKV);
       }
       W = &Ly.qkv; out = P.qkv; ldo = ldqkv;
     } else if (ph == 1) {
@@ -347,7 +348,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
       W = &Ly.o; out = x; ldo = P.H;
     } else if (ph == 3) {
       // a6: RMSNorm, gate and up projections
-      norm_prologue(P, x, (size_t)P.H, M, Ly.w_post, Ly.gu);
+      norm_prologue(P, x, (size_t)P.H, M, Ly.w_post, Ly.gu, PK_MAT_GU);
       W = &Ly.gu; out = P.gu; ldo = ldgu;
     } else {
       // a6 gate + a7: down projection into the residual rows
@@ -362,9 +363,9 @@ __global__ void __launch_bounds__(PK_THREADS, 1) dmtd_pass_kernel(const __grid_c
     PK_STAMP();
 #ifdef DMTD_PASS_TIMING
     const int chunk_log = (!head && li == nL - 1 && ph != 1) ? 2048 + 64 * (ph - (ph > 1)) : -1;
-    if (W && !gemv_consume(P, *W, M, out, ldo, chunk_log)) *S.abort_flag = 1;
+    if (W && !gemv_consume(P, *W, head ? PK_MAT_HEAD : ph - (ph > 1), M, out, ldo, chunk_log)) *S.abort_flag = 1;
 #else
-    if (W && !gemv_consume(P, *W, M, out, ldo)) *S.abort_flag = 1;
+    if (W && !gemv_consume(P, *W, head ? PK_MAT_HEAD : ph - (ph > 1), M, out, ldo)) *S.abort_flag = 1;
 #endif
     PK_STAMP();
 #ifdef DMTD_PASS_TIMING

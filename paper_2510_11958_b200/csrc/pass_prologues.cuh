@@ -33,7 +33,7 @@ __device__ __forceinline__ bool stage_wait(const PassParams &P, const PassShared
 // RMSNorm of M rows (row r at x + r * row_stride), written as bf16 hi/lo columns for the
 // k-slabs this block needs of matrix W (steps a2 / a6 / a9, first half).
 __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, size_t row_stride, int M,
-                                           const float *w_norm, const PackedMat &W) {
+                                           const float *w_norm, const PackedMat &W, int kind) {
   const PassShared S = pass_shared();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, H = P.H;
   PK_PROSTAMP(0);
@@ -46,7 +46,7 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
       stage_copy(S, S.xs + lane * H, x + (size_t)lane * row_stride, (uint32_t)(H * 4));
     }
   }
-  const SlabSpan sp = slab_span(W);
+  const SlabSpan sp = slab_span(S, W, kind);
   const int ks4 = sp.KS / 4, nu = sp.count * ks4;
   float4 wv[PK_SPAN_UNITS];
 #pragma unroll
@@ -94,9 +94,9 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
 }
 
 // SwiGLU gate (step a6, second half) for the k-slabs this block needs of the down projection.
-__device__ __noinline__ void swiglu_prologue(const PassParams &P, int M, const PackedMat &W) {
+__device__ __noinline__ void swiglu_prologue(const PassParams &P, int M, const PackedMat &W, int kind = PK_MAT_DOWN) {
   const PassShared S = pass_shared();
-  const SlabSpan sp = slab_span(W);
+  const SlabSpan sp = slab_span(S, W, kind);
   const int ks4 = sp.KS / 4, ldgu = 2 * P.I, total = sp.count * M * ks4;
   // two copies (gate values, up values) per (slab, row) i = sl * M + m, spread over the lanes of the first warp
   if (threadIdx.x == 0) stage_begin(S, (uint32_t)(sp.count * M * 2 * sp.KS * 4));
@@ -129,10 +129,10 @@ __device__ __noinline__ void swiglu_prologue(const PassParams &P, int M, const P
 // Online-softmax merge of the key slices (step a4, second half) for the heads this block's share
 // of the O projection multiplies, written as bf16 hi/lo columns: one warp per (row, head), one
 // lane per 4 output values, every slice's partial output loaded before any is used.
-__device__ __noinline__ void merge_prologue(const PassParams &P, int M, int nsplit, const PackedMat &W) {
+__device__ __noinline__ void merge_prologue(const PassParams &P, int M, int nsplit, const PackedMat &W, int kind = PK_MAT_O) {
   const PassShared S = pass_shared();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const SlabSpan sp = slab_span(W);
+  const SlabSpan sp = slab_span(S, W, kind);
   const int heads_per_slab = sp.KS / PK_D, n_heads = sp.count * heads_per_slab;
 #pragma unroll 1
   for (int pair = warp; pair < M * n_heads; pair += PK_WARPS) {

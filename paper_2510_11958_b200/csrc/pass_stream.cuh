@@ -32,7 +32,7 @@ struct WarpPipe {
   unsigned issued, consumed;
   StreamCursor cur;
 };
-static_assert(sizeof(WarpPipe) * PK_WARPS <= PK_SMALL_BYTES - 256, "pipe state does not fit");
+static_assert(sizeof(WarpPipe) * PK_WARPS <= 1024 - 256, "pipe state does not fit");
 
 __device__ __forceinline__ const PackedMat &pass_matrix(const PassParams &P, const PassShared &S, int q) {
   int n_layer_mats = 4 * (P.l_end - P.l_begin);
@@ -105,6 +105,31 @@ __device__ __forceinline__ void prefetch_own_stream(const StreamCursor &cur, int
   }
 }
 
+__device__ __forceinline__ const PackedMat &matrix_of_kind(const PassParams &P, const PassShared &S, int kind) {
+  if (kind == PK_MAT_HEAD) return P.embed;
+  const PassLayer &L = S.layers[0];
+  return kind == PK_MAT_QKV ? L.qkv : kind == PK_MAT_O ? L.o : kind == PK_MAT_GU ? L.gu : L.down;
+}
+// Kernel entry: one thread per (matrix kind, warp) fills the plans (S.layers must be in place).
+__device__ __forceinline__ void plans_fill(const PassParams &P, const PassShared &S) {
+  const int kind = threadIdx.x / PK_WARPS, warp = threadIdx.x % PK_WARPS;
+  if (kind >= PK_MAT_KINDS) return;
+  if (kind != PK_MAT_HEAD && P.l_end == P.l_begin) return;
+  const PackedMat &W = matrix_of_kind(P, S, kind);
+  MatPlan &pl = S.plans[kind];
+  int c0, c1, w0, w1;
+  stream_ranges(W, warp, c0, c1, w0, w1);
+  const int slab_atoms = W.n_tiles * W.aps;
+  pl.w0[warp] = w0; pl.w1[warp] = w1;
+  const int s = w0 / slab_atoms, in_slab = w0 - s * slab_atoms;
+  pl.ws[warp] = s; pl.wT[warp] = in_slab / W.aps; pl.wa[warp] = in_slab % W.aps;
+  if (warp == 0) {
+    pl.c0 = c0; pl.c1 = c1;
+    pl.s_first = c0 < c1 ? c0 / slab_atoms : 0;
+    pl.s_count = c0 < c1 ? (c1 - 1) / slab_atoms - pl.s_first + 1 : 0;
+  }
+}
+
 __device__ __forceinline__ void cursor_init(StreamCursor &c, const PassParams &P, int warp) {
   c.mat = -1; c.n_mats = 4 * (P.l_end - P.l_begin) + 1; c.warp = warp;
   c.pos = c.end = 0; c.tile_mask = 0; c.base = nullptr;
@@ -116,9 +141,8 @@ __device__ __noinline__ bool cursor_next_matrix(StreamCursor &c, const PassParam
   while (c.pos >= c.end) {
     if (++c.mat >= c.n_mats) { c.mat = c.n_mats; return false; }
     const PackedMat &W = pass_matrix(P, S, c.mat);
-    int c0, c1, w0, w1;
-    stream_ranges(W, c.warp, c0, c1, w0, w1);
-    c.pos = w0; c.end = w1; c.base = W.w;
+    const MatPlan &pl = S.plans[c.mat >= 4 * (P.l_end - P.l_begin) ? PK_MAT_HEAD : (c.mat & 3)];
+    c.pos = pl.w0[c.warp]; c.end = pl.w1[c.warp]; c.base = W.w;
     c.tile_mask = (PK_CHUNK_ATOMS % W.aps == 0 && (W.aps & (W.aps - 1)) == 0) ? W.aps - 1 : 0;
   }
   return true;
@@ -238,16 +262,12 @@ __device__ __forceinline__ void store_act4(unsigned char *slab_base, int row_byt
 
 // Which k-slabs this block's share of W touches.
 struct SlabSpan { int first, count, KS, row_bytes; };
-__device__ __forceinline__ SlabSpan slab_span(const PackedMat &W) {
-  int c0, c1, w0, w1;
-  stream_ranges(W, 0, c0, c1, w0, w1);
+__device__ __forceinline__ SlabSpan slab_span(const PassShared &S, const PackedMat &W, int kind) {
   SlabSpan sp;
   sp.KS = W.aps * 32;
   sp.row_bytes = b_row_bytes(sp.KS);
-  const int slab_atoms = W.n_tiles * W.aps;
-  if (c0 >= c1) { sp.first = 0; sp.count = 0; return sp; }
-  sp.first = c0 / slab_atoms;
-  sp.count = (c1 - 1) / slab_atoms - sp.first + 1;
+  sp.first = S.plans[kind].s_first;
+  sp.count = S.plans[kind].s_count;
   return sp;
 }
 
