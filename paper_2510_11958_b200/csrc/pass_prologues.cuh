@@ -14,8 +14,10 @@ constexpr int PK_SPAN_UNITS = 3;     // float4 units of a block's k-slab span pe
 // Inputs of a prologue come into shared memory as bulk copies issued by one thread: no load
 // instruction waits in a register, and the whole input costs one trip to L2.  stage_begin
 // (thread 0) arms the barrier, stage_copy adds a copy, stage_wait (all threads) waits for them.
-__device__ __forceinline__ void stage_begin(const PassShared &S, uint32_t bytes) {
-  fence_proxy_async_global();           // the copies must see what other blocks wrote before the grid barrier
+// fence: the thread that calls this also issues the copies (the copies must see what other blocks wrote before
+// the grid barrier: a proxy fence by every thread that issues some, once).
+__device__ __forceinline__ void stage_begin(const PassShared &S, uint32_t bytes, bool fence = true) {
+  if (fence) fence_proxy_async_global();
   mbar_expect_tx(smem_u32(S.stage_bar), bytes);
 }
 __device__ __forceinline__ void stage_copy(const PassShared &S, void *dst, const void *src, uint32_t bytes) {
@@ -38,7 +40,7 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, H = P.H;
   PK_PROSTAMP(0);
   // one copy per row, each issued by its own lane of the first warp
-  if (threadIdx.x == 0) stage_begin(S, (uint32_t)(M * H * 4));
+  if (threadIdx.x == 0) stage_begin(S, (uint32_t)(M * H * 4), false);
   if (warp == 0) {
     __syncwarp();
     if (lane < M) {
@@ -99,7 +101,7 @@ __device__ __noinline__ void swiglu_prologue(const PassParams &P, int M, const P
   const SlabSpan sp = slab_span(S, W, kind);
   const int ks4 = sp.KS / 4, ldgu = 2 * P.I, total = sp.count * M * ks4;
   // two copies (gate values, up values) per (slab, row) i = sl * M + m, spread over the lanes of the first warp
-  if (threadIdx.x == 0) stage_begin(S, (uint32_t)(sp.count * M * 2 * sp.KS * 4));
+  if (threadIdx.x == 0) stage_begin(S, (uint32_t)(sp.count * M * 2 * sp.KS * 4), false);
   if (threadIdx.x < 32) {
     __syncwarp();
     fence_proxy_async_global();
