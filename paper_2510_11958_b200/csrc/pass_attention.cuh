@@ -54,7 +54,8 @@ constexpr int PK_PA_TILES_END = PK_PA_NEW + 2 * PK_MAX_ROWS * PK_D * 4;
 constexpr int PK_PA_OS = 0;                                   // after the tiles are consumed: [warps][16][PK_OROW] floats
 constexpr int PK_PA_RED = PK_WARPS * PK_QR * PK_OROW * 4;     // running max [warps][16], then sum / merge factor [warps][16]
 constexpr int PK_PA_ROWS = PK_PA_RED + 2 * PK_WARPS * PK_QR * 4;   // the pass's q | k | v vectors of one kv head, fp32, per row
-constexpr int PK_PA_END = PK_PA_ROWS + PK_MAX_ROWS * PK_AT_ROW_FLOATS * 4;
+constexpr int PK_PA_W = PK_PA_ROWS + PK_MAX_ROWS * PK_AT_ROW_FLOATS * 4;   // q-norm, k-norm weights (floats), rotary frequencies (doubles)
+constexpr int PK_PA_END = PK_PA_W + 2 * PK_D * 4 + (PK_D / 2) * 8;
 static_assert(PK_PA_TILES_END <= PK_PA_RED, "attention scratch overlaps");
 static_assert(PK_PA_END <= PK_SCRATCH_BYTES, "attention scratch does not fit");
 
@@ -95,6 +96,8 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = P.nq / P.nkv, nQ = R * G;
   const float *rows = reinterpret_cast<const float *>(sc + PK_PA_ROWS);
+  const float *w_q = reinterpret_cast<const float *>(sc + PK_PA_W), *w_k = w_q + PK_D;
+  const double *inv_freq = reinterpret_cast<const double *>(sc + PK_PA_W + 2 * PK_D * 4);
   const float scale = rsqrtf((float)PK_D);
 #pragma unroll 1
   for (int task = warp; task < nQ + 2 * R; task += PK_WARPS) {
@@ -111,13 +114,13 @@ __device__ __forceinline__ void attn_new_rows(const PassParams &P, const PassLay
       float ss = v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
       ss = warp_sum(ss);
       const float inv = rsqrtf(ss / (float)PK_D + P.eps) * (kind == 0 ? scale : 1.f);
-      const float *w = kind == 0 ? Ly.w_qn : Ly.w_kn;
+      const float *w = kind == 0 ? w_q : w_k;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) v[j] = v[j] * inv * __ldg(w + lane + 32 * j);
+      for (int j = 0; j < 4; ++j) v[j] = v[j] * inv * w[lane + 32 * j];
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         // angle reduced to [-pi, pi] in double, then the fast sine and cosine
-        double a = (double)pos * P.inv_freq[lane + 32 * j];
+        double a = (double)pos * inv_freq[lane + 32 * j];
         a -= 6.283185307179586 * rint(a * 0.15915494309189535);
         float sn, cs;
         __sincosf((float)a, &sn, &cs);
@@ -351,18 +354,28 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     };
     PK_SUBSTAMP(0);
     pk_sync();                                            // the previous item is done with the scratch
-    if (threadIdx.x == 0) {
-      // the pass's own q | k | v vectors of this kv head: three bulk copies per row
-      const int ldq = (P.nq + 2 * P.nkv) * PK_D;
-      stage_begin(S, (uint32_t)(R * (G + 2) * PK_D * 4));
+    // the pass's own q | k | v vectors of this kv head, the two norm weights and the rotary frequencies:
+    // asynchronous 16-byte copies by all threads, a group of their own so that the rows can be waited for while
+    // the cached tile is still on its way.  (Bulk copies by one thread need a cross-proxy fence after the grid
+    // barrier first and are issued one after the other: 0.9 us before the request was out.)
+    {
+      const int ldq = (P.nq + 2 * P.nkv) * PK_D, per_row = (G + 2) * (PK_D / 4), n_rows_units = R * per_row;
+      const uint32_t sc_u32 = smem_u32(sc);
 #pragma unroll 1
-      for (int r = 0; r < R; ++r) {
-        const float *src = P.qkv + (size_t)(b * R + r) * ldq;
-        float *dst = reinterpret_cast<float *>(sc + PK_PA_ROWS) + r * PK_AT_ROW_FLOATS;
-        stage_copy(S, dst, src + kvh * G * PK_D, (uint32_t)(G * PK_D * 4));
-        stage_copy(S, dst + G * PK_D, src + (P.nq + kvh) * PK_D, PK_D * 4);
-        stage_copy(S, dst + (G + 1) * PK_D, src + (P.nq + P.nkv + kvh) * PK_D, PK_D * 4);
+      for (int c = threadIdx.x; c < n_rows_units + 96; c += PK_THREADS) {
+        if (c < n_rows_units) {
+          const int r = c / per_row, u = c - r * per_row, hd = u >> 5, part = u & 31;
+          const int col = hd < G ? (kvh * G + hd) * PK_D : hd == G ? (P.nq + kvh) * PK_D : (P.nq + P.nkv + kvh) * PK_D;
+          cp_async16(sc_u32 + PK_PA_ROWS + (r * PK_AT_ROW_FLOATS + hd * PK_D) * 4 + part * 16,
+                     P.qkv + (size_t)(b * R + r) * ldq + col + part * 4);
+        } else {
+          const int w = c - n_rows_units;                     // 32 + 32 units of norm weights, 32 of frequencies
+          const void *src = w < 32 ? (const void *)(Ly.w_qn + w * 4) : w < 64 ? (const void *)(Ly.w_kn + (w - 32) * 4)
+                                                                              : (const void *)(P.inv_freq + (w - 64) * 2);
+          cp_async16(sc_u32 + PK_PA_W + w * 16, src);
+        }
       }
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
     PK_SUBSTAMP(1);
     fetch_cached(0);                                      // in flight while the pass's own rows arrive
@@ -370,7 +383,8 @@ __device__ __noinline__ void attention_stage(const PassParams &P, const PassLaye
     // query rows beyond nQ are zero (the previous item's partial outputs lay over the Q tiles)
 #pragma unroll 1
     for (int i = threadIdx.x; i < 2 * PK_QR * PK_QROW / 16; i += PK_THREADS) sts128(qh_tile + i * 16, make_uint4(0u, 0u, 0u, 0u));
-    stage_wait(P, S);
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 1;" ::: "memory");   // the rows' group; the tile's may still be open
+    pk_sync();
     PK_SUBSTAMP(3);
     attn_new_rows<Op>(P, Ly, sc, b, kvh, R, pos0, split == 0);
     PK_SUBSTAMP(4);
