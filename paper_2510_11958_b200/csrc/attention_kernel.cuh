@@ -310,15 +310,44 @@ __device__ __forceinline__ void attn_combine_store_w(AttnAccW &A, unsigned char 
 }
 
 
-constexpr int ATTN_TC_SMEM = PK_AT_ROWS;         // tiles, Q, partial-output overlay, reduction arrays
+constexpr int ATTN_TC_NEW = PK_AT_ROWS;          // fused form: K rows of the pass [ATTN_TC_MAX_NEW][128] (cache type), then V rows
+constexpr int ATTN_TC_MAX_NEW = 15;              // new positions per sequence the fused form takes (more: the prefill kernel)
+constexpr int ATTN_TC_SMEM = ATTN_TC_NEW + 2 * ATTN_TC_MAX_NEW * PK_D * 2;   // tiles, Q, partial-output overlay, reduction arrays, new rows
+static_assert(2 * (ATTN_TC_SMEM + 1024) <= 228 * 1024, "two blocks per SM");
+
+// What the fused form of attn_tc_kernel needs for step a3 (QK-norm, rotary embedding, KV append): with these the
+// kernel reads the raw q | k | v rows of the QKV projection itself; every block normalises and rotates its own
+// query rows and the new K rows that fall into its key slice (a few rows, recomputed by the blocks that share
+// them), and the block that owns a position appends its K and V rows to the cache.  w_qn == nullptr: the rows in
+// qkv are finished already and the new K / V rows are in the cache (the stand-alone attention call).
+struct AttnFuse {
+  const float *w_qn, *w_kn;        // QK-norm weights [128]
+  const float2 *table;             // (cos, sin) of the pass's positions [R][64]
+  float eps;
+};
+// QK-norm and rotary embedding of one head vector, one value per lane and quarter (v[j] = element lane + 32 j).
+__device__ __forceinline__ void head_norm_rope_table(const float *w, const float2 *cs_row, float eps, int lane, float (&v)[4]) {
+  float ss = v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
+  ss = warp_sum(ss);
+  const float inv = rsqrtf(ss / (float)PK_D + eps);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) v[j] = v[j] * inv * w[lane + 32 * j];
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const float2 cs = cs_row[lane + 32 * j];
+    const float a = v[j], bb = v[j + 2];
+    v[j] = a * cs.x - bb * cs.y;
+    v[j + 2] = bb * cs.x + a * cs.y;
+  }
+}
 
 // qkv [B*R][ldq]: q heads already normalised and rotated (not scaled); K and V of the new rows
 // already in the cache.  Cache [b][kv head][max_seq][128] bf16.
-template <class Op>
+template <class Op, bool FUSED = false>
 __global__ void __launch_bounds__(PK_THREADS, 2)      // 16-bit cache: two blocks per SM overlap load and math
 attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ kc, const void *__restrict__ vc, int max_seq,
                int nq, int nkv, int R, int RB, int CH, const int *__restrict__ pos0_ptr, float *__restrict__ part_o,
-               float *__restrict__ part_ml, int nsplit) {
+               float *__restrict__ part_ml, int nsplit, AttnFuse F = AttnFuse{nullptr, nullptr, nullptr, 0.f}) {
   extern __shared__ __align__(1024) unsigned char sc[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int G = nq / nkv, n_rb = (R + RB - 1) / RB;
@@ -343,22 +372,48 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
   for (int qi = warp; qi < nQ; qi += PK_WARPS) {
     const float *src = qkv + (size_t)(b * R + r0 + qi / G) * ldq + (size_t)(kvh * G + qi % G) * PK_D;
     typename Op::T *qh = reinterpret_cast<typename Op::T *>(sc + PK_AT_QH + qi * PK_QROW);
+    float v[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float v = src[lane + 32 * j] * scale;
-      qh[lane + 32 * j] = Op::from_float(v);
-    }
+    for (int j = 0; j < 4; ++j) v[j] = src[lane + 32 * j];
+    if (FUSED) head_norm_rope_table(F.w_qn, F.table + (size_t)(r0 + qi / G) * (PK_D / 2), F.eps, lane, v);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) qh[lane + 32 * j] = Op::from_float(v[j] * scale);
   }
   const size_t head_off = ((size_t)b * nkv + kvh) * max_seq * PK_D;
   const int n_keys = j1 - j0;
+  // fused form: the pass's rows r_lo .. r_hi - 1 sit at positions inside this block's key slice; their K and V
+  // come from the projection's output, not from the cache
+  const int r_lo = FUSED ? max(0, j0 - pos0) : 0, r_hi = FUSED ? max(r_lo, min(r1, j1 - pos0)) : 0;
+  if (FUSED) {
+    typename Op::T *new_k = reinterpret_cast<typename Op::T *>(sc + ATTN_TC_NEW);
+    typename Op::T *new_v = new_k + ATTN_TC_MAX_NEW * PK_D;
+    for (int task = warp; task < 2 * (r_hi - r_lo); task += PK_WARPS) {
+      const int r = r_lo + (task >> 1), is_v = task & 1;
+      const float *src = qkv + (size_t)(b * R + r) * ldq + (size_t)(nq + (is_v ? nkv : 0) + kvh) * PK_D;
+      float v[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v[j] = src[lane + 32 * j];
+      if (!is_v) head_norm_rope_table(F.w_kn, F.table + (size_t)r * (PK_D / 2), F.eps, lane, v);
+      typename Op::T *row = (is_v ? new_v : new_k) + (r - r_lo) * PK_D;
+      typename Op::T *cache = const_cast<typename Op::T *>(reinterpret_cast<const typename Op::T *>(is_v ? vc : kc)) + head_off +
+                              (size_t)(pos0 + r) * PK_D;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const typename Op::T h = Op::from_float(v[j]);
+        row[lane + 32 * j] = h;
+        if (r >= r0) cache[lane + 32 * j] = h;           // the row block that owns the position appends it
+      }
+    }
+  }
   // bf16 cache: two tile buffers (the lo-part areas are free here), tile i+1 in flight while
   // tile i is multiplied
   const typename Op::T *kb = reinterpret_cast<const typename Op::T *>(kc) + head_off;
   const typename Op::T *vb = reinterpret_cast<const typename Op::T *>(vc) + head_off;
   auto fetch = [&](int tile0, int buf) {
     const int n_t = min(PK_TK, n_keys - tile0);
+    const int n_c = FUSED ? max(0, min(n_t, pos0 - (j0 + tile0))) : n_t;       // rows of the tile that come from the cache
     const uint32_t k_t = smem_u32(sc + (buf ? PK_AT_KL : PK_AT_KH)), v_t = smem_u32(sc + (buf ? PK_AT_VL : PK_AT_VH));
-    for (int c = threadIdx.x; c < n_t * 32; c += PK_THREADS) {
+    for (int c = threadIdx.x; c < n_c * 32; c += PK_THREADS) {
       const int row = c >> 5, part = c & 31;
       const uint32_t dst = part < 16 ? k_t + row * PK_KROW + part * 16 : v_t + row * PK_VROW + (part - 16) * 16;
       cp_async16(dst, (part < 16 ? kb : vb) + (size_t)(j0 + tile0 + row) * PK_D + (part & 15) * 8);
@@ -367,6 +422,19 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
     for (int c = threadIdx.x; c < (n16 - n_t) * 16; c += PK_THREADS)      // P = 0 times stale bits must stay 0
       sts128(v_t + (n_t + (c >> 4)) * PK_VROW + (c & 15) * 16, make_uint4(0u, 0u, 0u, 0u));
     asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  // fused form: the pass's own rows of a tile, from the new-row area (written before the barrier in front of the
+  // tile's multiplication; the tile buffer is free: the tile two trips back has been consumed)
+  auto place_new = [&](int tile0, int buf) {
+    if (!FUSED) return;
+    const int n_t = min(PK_TK, n_keys - tile0);
+    const int first = max(0, pos0 - (j0 + tile0));                             // first row of the tile that is a new row
+    const uint32_t k_t = smem_u32(sc + (buf ? PK_AT_KL : PK_AT_KH)), v_t = smem_u32(sc + (buf ? PK_AT_VL : PK_AT_VH));
+    for (int c = threadIdx.x + first * 32; c < n_t * 32; c += PK_THREADS) {
+      const int row = c >> 5, part = c & 31, r = j0 + tile0 + row - pos0 - r_lo;
+      const uint4 val = *reinterpret_cast<const uint4 *>(sc + ATTN_TC_NEW + ((part < 16 ? 0 : ATTN_TC_MAX_NEW) + r) * PK_D * 2 + (part & 15) * 16);
+      sts128(part < 16 ? k_t + row * PK_KROW + part * 16 : v_t + row * PK_VROW + (part - 16) * 16, val);
+    }
   };
   fetch(0, 0);
   int buf = 0;
@@ -386,6 +454,8 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
       } else {
         asm volatile("cp.async.wait_group 0;" ::: "memory");
       }
+      if (FUSED && tile0 == 0) __syncthreads();         // the new-row area is written
+      place_new(tile0, buf);
       __syncthreads();                                  // tile (and, the first time, Q) visible to all
       if (tile0 == 0) {
 #pragma unroll
@@ -411,6 +481,8 @@ attn_tc_kernel(const float *__restrict__ qkv, int ldq, const void *__restrict__ 
     } else {
       asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
+    if (FUSED && tile0 == 0) __syncthreads();           // the new-row area is written
+    place_new(tile0, buf);
     __syncthreads();                                    // tile (and, the first time, Q) visible to all
     if (tile0 == 0) {
 #pragma unroll

@@ -83,6 +83,7 @@ struct dmtd_ctx {
 
   // options
   bool use_graph = true, literal_sum = false, use_fused = true, use_tc_attention = true;
+  bool fuse_qk_rope = true;                 // QK-norm, RoPE and the KV append inside the tensor-core attention kernel
   float temperature = 0.f;                  // > 0: tokens are drawn from softmax(logits / temperature); 0: greedy
   uint64_t sample_seed = 0;
 
@@ -367,10 +368,15 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
   KVT *kc = static_cast<KVT *>(c->kc) + (size_t)layer * c->kv_layer_elems;
   KVT *vc = static_cast<KVT *>(c->vc) + (size_t)layer * c->kv_layer_elems;
   const LayerDev &lw = c->layers[layer];
-  qk_norm_rope_append_kernel<D, KVT><<<dim3(M, (heads + 3) / 4), 128, 0, c->stream>>>(
-      c->qkv, c->ldqkv, s.n_q_heads, s.n_kv_heads, R, lw.w_qn, lw.w_kn, s.rms_eps, c->rope_tab, pos0, kc, vc,
-      c->max_seq);
-  LAUNCH_OK(c, "qk_norm_rope_append_kernel");
+  // a3 inside the attention kernel (16-bit cache, head_dim 128, decode-sized chunks): one launch less per layer
+  const bool fused_a3 = D == PK_D && !std::is_same<KVT, float>::value && c->use_tc_attention && c->fuse_qk_rope && !flash &&
+                        R <= ATTN_TC_MAX_NEW;
+  if (!fused_a3) {
+    qk_norm_rope_append_kernel<D, KVT><<<dim3(M, (heads + 3) / 4), 128, 0, c->stream>>>(
+        c->qkv, c->ldqkv, s.n_q_heads, s.n_kv_heads, R, lw.w_qn, lw.w_kn, s.rms_eps, c->rope_tab, pos0, kc, vc,
+        c->max_seq);
+    LAUNCH_OK(c, "qk_norm_rope_append_kernel");
+  }
   if constexpr (D == PK_D && !std::is_same<KVT, float>::value) {
     if (flash) {
       // a chunk of many positions per sequence (the prefill): the causal kernel, rows straight into `act`
@@ -390,8 +396,13 @@ dmtd_status launch_attention_t(dmtd_ctx *c, int layer, int B, int R, const int *
           c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
     } else {
       using Op = typename std::conditional<std::is_same<KVT, __half>::value, OpF16, OpBf16>::type;
-      attn_tc_kernel<Op><<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
-          c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
+      if (fused_a3)
+        attn_tc_kernel<Op, true><<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
+            c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit,
+            AttnFuse{lw.w_qn, lw.w_kn, c->rope_tab, s.rms_eps});
+      else
+        attn_tc_kernel<Op><<<dim3(nsplit, s.n_kv_heads * n_rb, B), PK_THREADS, ATTN_TC_SMEM, c->stream>>>(
+            c->qkv, c->ldqkv, kc, vc, c->max_seq, s.n_q_heads, s.n_kv_heads, R, RB, c->CH, pos0, c->part_o, c->part_ml, nsplit);
     }
   } else {
   size_t smem = (size_t)ATTN_WARPS * ATTN_QR * D * sizeof(float);
@@ -534,6 +545,8 @@ dmtd_status configure_kernels(dmtd_ctx *c) {
   CUDA_TRY(c, cudaFuncSetAttribute(attn_f32_kernel, dyn, ATTN_F32_SMEM));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<OpBf16>, dyn, ATTN_TC_SMEM));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<OpF16>, dyn, ATTN_TC_SMEM));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<OpBf16, true>, dyn, ATTN_TC_SMEM));
+  CUDA_TRY(c, cudaFuncSetAttribute(attn_tc_kernel<OpF16, true>, dyn, ATTN_TC_SMEM));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_prefill_kernel<OpBf16>, dyn, ATTN_PF_SMEM));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_prefill_kernel<OpF16>, dyn, ATTN_PF_SMEM));
   CUDA_TRY(c, cudaFuncSetAttribute(attn_partial_kernel<64, __half>, dyn, 64 * 1024));
@@ -1196,6 +1209,7 @@ dmtd_status dmtd_set_option(dmtd_ctx *c, const char *name, int64_t value) {
   if (!strcmp(name, "cuda_graph")) { c->use_graph = value != 0; return DMTD_OK; }
   if (!strcmp(name, "literal_sum")) { c->literal_sum = value != 0; drop_graphs(c); return DMTD_OK; }
   if (!strcmp(name, "fused_pass")) { c->use_fused = value != 0; return DMTD_OK; }
+  if (!strcmp(name, "fused_qk_rope")) { c->fuse_qk_rope = value != 0; drop_graphs(c); return DMTD_OK; }
   if (!strcmp(name, "tcgen05_gemm")) { c->use_umma = value != 0; drop_graphs(c); return DMTD_OK; }
   if (!strcmp(name, "tc_attention")) { c->use_tc_attention = value != 0; drop_graphs(c); return DMTD_OK; }
   return fail(c, DMTD_ERR_INVALID_ARG, "unknown option %s", name);

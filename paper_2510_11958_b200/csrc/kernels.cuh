@@ -624,9 +624,30 @@ __global__ void argmax_slices_kernel(const float *__restrict__ logits, int ldl, 
   float best = -INFINITY;
   int bi = 0x7fffffff;
   const int position = st->n_known;                  // where the picked token will sit
-  for (int i = i0 + threadIdx.x; i < i1; i += blockDim.x) {
-    float v = pick_value(z[i], i, position, b, sp);
-    if (v > best) { best = v; bi = i; }
+  if (per % 4 == 0 && ldl % 4 == 0) {
+    // four logits per load (the slice starts on a 16-byte boundary); indices rise within a thread, so the
+    // first of equal values stays
+    for (int i = i0 + 4 * threadIdx.x; i < i1; i += 4 * blockDim.x) {
+      if (i + 4 <= i1) {
+        const float4 q = *reinterpret_cast<const float4 *>(z + i);
+        const float e[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float v = pick_value(e[j], i + j, position, b, sp);
+          if (v > best) { best = v; bi = i + j; }
+        }
+      } else {
+        for (int j = i; j < i1; ++j) {
+          const float v = pick_value(z[j], j, position, b, sp);
+          if (v > best) { best = v; bi = j; }
+        }
+      }
+    }
+  } else {
+    for (int i = i0 + threadIdx.x; i < i1; i += blockDim.x) {
+      float v = pick_value(z[i], i, position, b, sp);
+      if (v > best) { best = v; bi = i; }
+    }
   }
   __shared__ float sv[256];
   __shared__ int si[256];
