@@ -60,30 +60,47 @@ __device__ __noinline__ void norm_prologue(const PassParams &P, const float *x, 
   PK_PROSTAMP(1);
   stage_wait(P, S);
   PK_PROSTAMP(2);
-#pragma unroll 1
-  for (int m = 0; m < M; ++m) {
-    float ss = 0.f;
+  // the rows' sums of squares side by side (independent chains through the loads and the warp reductions)
+  {
+    float ss[PK_MAX_ROWS];
+#pragma unroll
+    for (int m = 0; m < PK_MAX_ROWS; ++m) ss[m] = 0.f;
 #pragma unroll 1
     for (int k4 = threadIdx.x; k4 < H / 4; k4 += PK_THREADS) {
-      const float4 v = reinterpret_cast<const float4 *>(S.xs)[m * (H / 4) + k4];
-      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+#pragma unroll
+      for (int m = 0; m < PK_MAX_ROWS; ++m) {
+        if (m < M) {
+          const float4 v = reinterpret_cast<const float4 *>(S.xs)[m * (H / 4) + k4];
+          ss[m] += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
+      }
     }
-    ss = warp_sum(ss);
-    if (lane == 0) S.red[warp * PK_MAX_ROWS + m] = ss;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+      for (int m = 0; m < PK_MAX_ROWS; ++m) ss[m] += __shfl_xor_sync(0xffffffffu, ss[m], o);
+    }
+    if (lane < PK_MAX_ROWS) {
+      float mine = ss[0];
+#pragma unroll
+      for (int m = 1; m < PK_MAX_ROWS; ++m) mine = lane == m ? ss[m] : mine;
+      S.red[warp * PK_MAX_ROWS + lane] = mine;
+    }
   }
   pk_sync();
   PK_PROSTAMP(3);
+  const float inv_h = 1.f / (float)H;
 #pragma unroll 1
   for (int m = 0; m < M; ++m) {
     float v = 0.f;
 #pragma unroll
     for (int w = 0; w < PK_WARPS; ++w) v += S.red[w * PK_MAX_ROWS + m];
-    const float inv = rsqrtf(v / (float)H + P.eps);
+    const float inv = rsqrtf(v * inv_h + P.eps);
 #pragma unroll
     for (int j = 0; j < PK_SPAN_UNITS; ++j) {
       const int u = threadIdx.x + j * PK_THREADS;
       if (u < nu) {
-        const int sl = u / ks4, kl = (u - sl * ks4) * 4;
+        const int sl = u >= ks4 ? 1 : 0, kl = (u - sl * ks4) * 4;         // a block's share touches at most two slabs
         float4 a = reinterpret_cast<const float4 *>(S.xs)[(m * H + (sp.first + sl) * sp.KS + kl) / 4];
         a.x *= inv * wv[j].x; a.y *= inv * wv[j].y; a.z *= inv * wv[j].z; a.w *= inv * wv[j].w;
         store_act4(S.bstage + (size_t)sl * 8 * sp.row_bytes, sp.row_bytes, m, kl, a);
