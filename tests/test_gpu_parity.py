@@ -99,6 +99,29 @@ def test_graph_replay_matches_plain_launches(dmtd):
     assert (outs[0] == outs[1]).all()
 
 
+def test_qk_norm_rope_inside_attention_matches_separate_kernel(dmtd):
+    """Step a3 (Section 3.1's QK-norm, RoPE, KV append) run inside the tensor-core attention kernel and as a
+    launch of its own: the same generated tokens on the per-step path (5 sequences: more rows than the pass kernel takes)."""
+    shape = SHAPES["mid"]
+    w = to_cuda(make_weights(shape, seed=0))
+    prompts = torch.from_numpy(make_prompts(shape.vocab, 5, 21, seed=1).numpy()).cuda()
+    outs, launches = [], []
+    for fused in (0, 1):
+        eng = _engine(dmtd, shape, w, 2, 3, 5, 64)
+        eng.set_option("fused_qk_rope", fused)
+        eng.set_option("cuda_graph", 0)
+        eng.prefill(prompts)
+        before = eng.launch_count()
+        toks = []
+        for _ in range(4):
+            rc, n, out = eng.decode_cycle(3)
+            toks.append(out[:, :n].clone())
+        outs.append(torch.cat(toks, 1).cpu())
+        launches.append(eng.launch_count() - before)
+    assert (outs[0] == outs[1]).all()
+    assert launches[1] < launches[0]                   # one launch less per layer and pass
+
+
 def test_prefill_longer_than_one_chunk(dmtd):
     """A prompt that does not fit the workspace in one go is fed in causal chunks."""
     shape = SHAPES["tiny"].with_(dtype="bf16")
