@@ -237,7 +237,7 @@ dmtd_status dmtd_set_sampling(dmtd_ctx *ctx, float temperature, uint64_t seed);
  *   "literal_sum"  0/1  upper-layer input of a full pass = embedding + lower-stack output, the
  *                       literal sum of Eq. 4, instead of the lower-stack output alone (default 0)
  *   "fused_pass"   0/1  run each decode pass as one persistent kernel where the model and batch
- *                       allow it (bf16 weights, bf16 or fp32 KV, head_dim 128, at most 4 rows per pass);
+ *                       allow it (bf16 weights, head_dim 128, at most 4 rows per pass);
  *                       0 = always the per-step kernels (default 1)
  *   "encoding_layers" x  the ExDy variant (Section 2.1, the paragraph after Eq. 4; Section 3.3): the
  *                       short passes run the first x encoding layers as well as the last L_d
@@ -252,6 +252,11 @@ dmtd_status dmtd_set_sampling(dmtd_ctx *ctx, float temperature, uint64_t seed);
  *                       tensor cores; bf16 contexts whose hidden, query and intermediate sizes
  *                       are multiples of 64 hold the second weight copy it reads, which doubles
  *                       the weight memory of the context (default 1)
+ *   "tcgen05_gemm_stages" n  pipeline stages of a block of that GEMM, 2..6; 0 = chosen per launch as
+ *                       what keeps the most weight blocks in flight per SM (default 0)
+ *   "fused_qk_rope" 0/1 QK-norm, rotary embedding and the KV append (Section 3.1's Qwen3 block) inside
+ *                       the tensor-core attention kernel of the per-step path (16-bit cache, head_dim
+ *                       128, chunks of fewer than 16 positions) instead of a launch of their own (default 1)
  * Errors: INVALID_ARG for an unknown name or value; SHAPE / STATE for encoding_layers as above. */
 dmtd_status dmtd_set_option(dmtd_ctx *ctx, const char *name, int64_t value);
 
