@@ -592,6 +592,13 @@ dmtd_status setup_fused(dmtd_ctx *c) {
         !fused_matrix_ok(ld.down, c->n_sms))
       return DMTD_OK;
     if ((ld.o.aps * 32) % PK_D) return DMTD_OK;
+    // the kernel works out every block's share of a matrix once per launch, from the first layer of the pass:
+    // all layers must have the same four shapes (they do: one hidden and one intermediate size per model)
+    const LayerDev &l0 = c->layers[0];
+    auto same = [](const PackedMat &a, const PackedMat &b) {
+      return a.N == b.N && a.K == b.K && a.n_tiles == b.n_tiles && a.aps == b.aps && a.n_slabs == b.n_slabs;
+    };
+    if (!same(ld.qkv, l0.qkv) || !same(ld.o, l0.o) || !same(ld.gu, l0.gu) || !same(ld.down, l0.down)) return DMTD_OK;
   }
   std::vector<PassLayer> h(s.n_layers);
   for (int l = 0; l < s.n_layers; ++l) {
